@@ -1,0 +1,171 @@
+/*
+ * flexiq.h -- C ABI of the B200 (sm_100a) FlexiQ hot path: the channel-wise mixed
+ * 4/8-bit quantized GEMM and implicit-GEMM convolution with run-time low-bit ratio.
+ *
+ * Conventions (all entry points)
+ *   - Return value: FLEXIQ_OK (0) or a negative FLEXIQ_ERR_* code.  Nothing aborts or
+ *     throws across the ABI.  flexiq_last_error() returns a thread-local message for
+ *     the last failing call on this thread.
+ *   - "_dev" pointers are device (global) memory owned by the caller, contiguous and
+ *     16-byte aligned; "_host" pointers are ordinary host memory.  The library owns
+ *     only the opaque layer handles it creates, and frees them in flexiq_layer_destroy.
+ *   - Device work is enqueued on the caller's stream (a cudaStream_t passed as void*,
+ *     NULL = legacy default stream).  Only flexiq_layer_create_* synchronises.  The
+ *     steady-state calls allocate nothing.
+ *   - There is no CPU fallback: on a device that is not sm_100 the calls return
+ *     FLEXIQ_ERR_UNSUPPORTED.
+ *   - Every device-side wait is bounded.  If one expires the kernel raises a status
+ *     word that flexiq_check_status() reports as FLEXIQ_ERR_TIMEOUT; the context
+ *     stays usable.
+ *
+ * Notation (the paper's): K input-feature channels, split into n_g = K / G channel
+ * groups of G channels; K_lo = max_4bit_ch = n_low * G channels are computed from
+ * 4-bit values, the remaining K_hi = K - K_lo at 8 bits.  "Slab order" is the channel
+ * order after the layout post-processing of Sec. 5: slab group j holds original group
+ * group_perm[j]; channels keep their order inside a group; low-bit groups are a prefix
+ * at every ratio (nested selection, Sec. 4.2).
+ */
+#ifndef FLEXIQ_H_
+#define FLEXIQ_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FLEXIQ_OK 0
+#define FLEXIQ_ERR_INVALID_ARG (-1)
+#define FLEXIQ_ERR_UNSUPPORTED (-2)
+#define FLEXIQ_ERR_CUDA (-3)
+#define FLEXIQ_ERR_TIMEOUT (-4)
+
+/* x_dtype of flexiq_quantize_lower */
+#define FLEXIQ_DTYPE_F32 0
+#define FLEXIQ_DTYPE_F16 1
+#define FLEXIQ_DTYPE_BF16 2
+#define FLEXIQ_DTYPE_I8 3 /* already quantized by Eq. 1: only lowered and gathered */
+
+/* out_mode of flexiq_mixed_gemm / flexiq_mixed_conv */
+#define FLEXIQ_OUT_ACC_I32 0    /* raw int32 accumulators                       */
+#define FLEXIQ_OUT_REQUANT_I8 1 /* int8, re-quantized with y_scale (Eq. 1)      */
+#define FLEXIQ_OUT_DEQUANT_F32 2 /* fp32, de-quantized                          */
+
+/* How the low-bit slice travels from the prologue to the mainloop (layer property).
+ * PACKED : two 4-bit values per byte (half the bytes); the mainloop widens them to the
+ *          tensor cores' 8-bit integer operands in shared memory.
+ * MASKED : one int8 per value holding the 4-bit value already shifted back to its
+ *          extraction position (x4 << sx); the mainloop is a plain 8-bit integer GEMM.
+ * Both give bit-identical accumulators. */
+#define FLEXIQ_LOWBIT_MASKED_I8 0
+#define FLEXIQ_LOWBIT_PACKED_U4 1
+
+typedef struct flexiq_layer *flexiq_layer_t;
+
+/* Linear layer handle.  Implements the static part of the method: the layout
+ * post-processing of Sec. 5 (input channels permuted so that same-bitwidth channels are
+ * contiguous for every ratio), the per-(channel group, output channel) weight extraction
+ * positions of Sec. 4.1 / Fig. 4, and the cached 4-bit weights of Sec. 7 ("Resource
+ * Consumption").
+ *   Wq_dev          [K][N] row-major int8, ORIGINAL channel order (8-bit model, Eq. 1)
+ *   w_scale_dev     [N] fp32 per-output-channel weight scales
+ *   bias_dev        [N] fp32 or NULL
+ *   group_perm_host [K/G] original group stored at each slab position (a permutation)
+ *   x_shift_host    [K/G] static activation extraction position (0..4) of each ORIGINAL
+ *                   group (Sec. 4.1); NULL = all zero
+ * K % G == 0, G in {16, 32, 64}, N % 16 == 0.  The inputs are read during the call (it
+ * synchronises `stream`); they may be freed afterwards.  Starts at ratio 0. */
+int flexiq_layer_create_linear(flexiq_layer_t *out, int K, int N, int group_size,
+                               const int8_t *Wq_dev, const float *w_scale_dev,
+                               const float *bias_dev, const int32_t *group_perm_host,
+                               const uint8_t *x_shift_host, void *stream);
+
+/* Convolution layer handle (Fig. 4): Wq_dev [Cout][R][S][Cin] int8, NHWC activations,
+ * zero padding; channel groups run over Cin only, a group's extraction positions do not
+ * depend on the tap.  Cin % G == 0, Cout % 16 == 0.  Otherwise as above. */
+int flexiq_layer_create_conv(flexiq_layer_t *out, int Cin, int Cout, int R, int S, int stride,
+                             int pad, int group_size, const int8_t *Wq_dev,
+                             const float *w_scale_dev, const float *bias_dev,
+                             const int32_t *group_perm_host, const uint8_t *x_shift_host,
+                             void *stream);
+
+int flexiq_layer_destroy(flexiq_layer_t layer);
+
+/* Chooses FLEXIQ_LOWBIT_MASKED_I8 (default) or FLEXIQ_LOWBIT_PACKED_U4 for the layer.
+ * Must be the same for a flexiq_quantize_lower call and the mixed_* call that consumes
+ * its slabs. */
+int flexiq_layer_set_lowbit_path(flexiq_layer_t layer, int lowbit_path);
+
+/* Run-time ratio switch (Sec. 7, "Low-bitwidth Ratio Adjustment"): sets
+ * max_4bit_ch = K_lo = ceil(ratio * n_g - 1e-4) * G, clamped to [0, K].  Host-only, one
+ * integer, no data movement.  Takes effect for calls enqueued afterwards.
+ * ratio outside [0, 1] or NaN: FLEXIQ_ERR_INVALID_ARG. */
+int flexiq_set_lowbit_ratio(flexiq_layer_t layer, float ratio);
+int flexiq_get_max_4bit_ch(flexiq_layer_t layer, int *K_lo);
+
+/* Row pitch in bytes of the low-bit slab for a given K_lo under the layer's path:
+ * PACKED: K_lo / 2 rounded up to a multiple of 16;  MASKED: K_lo. */
+int flexiq_x4_pitch(flexiq_layer_t layer, int K_lo, int64_t *pitch_bytes);
+
+/* Activation prologue (Sec. 2.1 Eq. 1, Sec. 4.1 bit-lowering, Sec. 5 layout):
+ *   q  = clip(round_half_even(x / x_scale), -128, 127)          (skipped for I8 input)
+ *   slab group j <  n_low : x4 = clamp(q >> sx[j], -8, 7)   -> X4_dev
+ *   slab group j >= n_low : q                               -> X8_dev
+ * with channels gathered into slab order.
+ *   X_dev    [M][K] row-major (linear) or NHWC with M = Nb*H*W pixels (conv), x_dtype
+ *   X4_dev   [M][pitch] bytes, pitch = flexiq_x4_pitch(K_lo).  PACKED: byte t of a row
+ *            holds slab channel 2t in bits 0-3 and 2t+1 in bits 4-7 (two's complement).
+ *            MASKED: int8 (x4 << sx[j]).  May be NULL when K_lo == 0.
+ *   X8_dev   [M][K_hi] int8.  May be NULL when K_hi == 0.
+ *   dynamic_pos != 0: the run-time extraction positions of Sec. 4.1 -- a bitwise OR over
+ *            all values of a channel group in this call (negatives folded by ~) finds
+ *            the highest used bit -- replace the static ones; they are written to
+ *            x_shift_out_dev [K/G] (slab order, uint8) and must be handed to the mixed_*
+ *            call.  scratch_dev must then point to K/G uint32 words of device scratch.
+ * M == 0 is a successful no-op. */
+int flexiq_quantize_lower(flexiq_layer_t layer, const void *X_dev, int x_dtype, int64_t M,
+                          float x_scale, int dynamic_pos, uint8_t *X4_dev, int8_t *X8_dev,
+                          uint8_t *x_shift_out_dev, uint32_t *scratch_dev, void *stream);
+
+/* Mixed-precision GEMM (Sec. 7; objective of Sec. 2.3):
+ *   acc[m][n] = sum_{j <  n_low} ( sum_i x4[m][j,i] * w4[j,i][n] ) << (sx[j] + sw[j][n])
+ *             + sum_{j >= n_low}   sum_i x8[m][j,i] * w8[j,i][n]            (exact int32)
+ * followed by the per-output-channel epilogue
+ *   ACC_I32    : acc
+ *   REQUANT_I8 : clip(round_half_even(fma(float(acc), (x_scale*w_scale[n])/y_scale,
+ *                                        bias[n]/y_scale)), -128, 127)
+ *   DEQUANT_F32: fma(float(acc), x_scale*w_scale[n], bias[n])
+ *   X4_dev/X8_dev  slabs written by flexiq_quantize_lower at the layer's current ratio
+ *   x_shift_dev    [K/G] uint8 slab-order activation positions (dynamic mode) or NULL for
+ *                  the layer's static ones.  Only the PACKED path reads it; on the MASKED
+ *                  path the positions are already folded into the slab.
+ *   Y_dev          [M][N] row-major of the out_mode's type. */
+int flexiq_mixed_gemm(flexiq_layer_t layer, const uint8_t *X4_dev, const int8_t *X8_dev,
+                      const uint8_t *x_shift_dev, int64_t M, float x_scale, float y_scale,
+                      int out_mode, void *Y_dev, void *stream);
+
+/* Mixed-precision convolution as an implicit GEMM (Fig. 4): m = (image, p, q),
+ * k = (r, s, c), x[image][p*stride + r - pad][q*stride + s - pad][c], zero outside; the
+ * slabs are NHWC with the channel dimension split as in flexiq_quantize_lower
+ * (X4_dev [Nb][H][W][pitch], X8_dev [Nb][H][W][C_hi]); Y_dev [Nb][P][Q][Cout]. */
+int flexiq_mixed_conv(flexiq_layer_t layer, const uint8_t *X4_dev, const int8_t *X8_dev,
+                      const uint8_t *x_shift_dev, int Nb, int H, int W, float x_scale,
+                      float y_scale, int out_mode, void *Y_dev, void *stream);
+
+/* Test hooks: copy the layer's derived tables to host buffers (any may be NULL).
+ *   sw_host [K/G][N] uint8 weight extraction positions (slab order),
+ *   w8_host [N][Kw] int8 slab-order weights, w4_host [N][Kw/2] packed 4-bit weights,
+ * Kw = K (linear) or R*S*Cin with k = (r*S + s)*Cin + c (conv). */
+int flexiq_layer_export(flexiq_layer_t layer, uint8_t *sw_host, int8_t *w8_host,
+                        uint8_t *w4_host);
+
+/* Reads and clears the device status word raised by a bounded wait that expired.
+ * Synchronises `stream`. */
+int flexiq_check_status(void *stream);
+
+const char *flexiq_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLEXIQ_H_ */

@@ -1,0 +1,240 @@
+"""ctypes binding of libflexiq.so: argument marshalling only.
+
+Every function named ``flexiq_*`` here forwards to the C entry point of the same name
+(see ``include/flexiq.h``); ``Layer`` is a small convenience wrapper that owns a handle
+and allocates the slabs with torch.  Nothing here computes: every step of the path runs
+in the CUDA kernels of the library.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_DIR, "libflexiq.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4
+DTYPE_F32, DTYPE_F16, DTYPE_BF16, DTYPE_I8 = 0, 1, 2, 3
+OUT_ACC_I32, OUT_REQUANT_I8, OUT_DEQUANT_F32 = 0, 1, 2
+LOWBIT_MASKED_I8, LOWBIT_PACKED_U4 = 0, 1
+
+EXPORTS = [
+    "flexiq_layer_create_linear", "flexiq_layer_create_conv", "flexiq_layer_destroy",
+    "flexiq_layer_set_lowbit_path", "flexiq_set_lowbit_ratio", "flexiq_get_max_4bit_ch",
+    "flexiq_x4_pitch", "flexiq_quantize_lower", "flexiq_mixed_gemm", "flexiq_mixed_conv",
+    "flexiq_layer_export", "flexiq_check_status", "flexiq_last_error",
+]
+
+_lib = None
+
+
+class FlexiqError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"flexiq error {code}: {msg}")
+        self.code = code
+
+
+def lib():
+    """Loads the CUDA library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} is missing: build it with __graft_entry__.build() "
+                "(python -m paper_2510_02822_b200.build); there is no CPU fallback")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, f32 = C.c_void_p, C.c_int, C.c_int64, C.c_float
+        L.flexiq_last_error.restype = C.c_char_p
+        L.flexiq_layer_create_linear.argtypes = [C.POINTER(vp), i32, i32, i32, vp, vp, vp, vp, vp, vp]
+        L.flexiq_layer_create_conv.argtypes = [C.POINTER(vp), i32, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+        L.flexiq_layer_destroy.argtypes = [vp]
+        L.flexiq_layer_set_lowbit_path.argtypes = [vp, i32]
+        L.flexiq_set_lowbit_ratio.argtypes = [vp, f32]
+        L.flexiq_get_max_4bit_ch.argtypes = [vp, C.POINTER(i32)]
+        L.flexiq_x4_pitch.argtypes = [vp, i32, C.POINTER(i64)]
+        L.flexiq_quantize_lower.argtypes = [vp, vp, i32, i64, f32, i32, vp, vp, vp, vp, vp]
+        L.flexiq_mixed_gemm.argtypes = [vp, vp, vp, vp, i64, f32, f32, i32, vp, vp]
+        L.flexiq_mixed_conv.argtypes = [vp, vp, vp, vp, i32, i32, i32, f32, f32, i32, vp, vp]
+        L.flexiq_layer_export.argtypes = [vp, vp, vp, vp]
+        L.flexiq_check_status.argtypes = [vp]
+        _lib = L
+    return _lib
+
+
+def last_error() -> str:
+    return lib().flexiq_last_error().decode()
+
+
+def _check(rc: int):
+    if rc != OK:
+        raise FlexiqError(rc, last_error())
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    import torch
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+# ---- one function per C entry point ------------------------------------------------
+def flexiq_layer_create_linear(K, N, G, Wq_dev, w_scale_dev, bias_dev, perm_host, x_shift_host):
+    h = C.c_void_p()
+    _check(lib().flexiq_layer_create_linear(C.byref(h), K, N, G, _ptr(Wq_dev), _ptr(w_scale_dev), _ptr(bias_dev),
+                                            perm_host.ctypes.data_as(C.c_void_p),
+                                            None if x_shift_host is None else x_shift_host.ctypes.data_as(C.c_void_p),
+                                            _stream()))
+    return h
+
+
+def flexiq_layer_create_conv(Cin, Cout, R, S, stride, pad, G, Wq_dev, w_scale_dev, bias_dev, perm_host, x_shift_host):
+    h = C.c_void_p()
+    _check(lib().flexiq_layer_create_conv(C.byref(h), Cin, Cout, R, S, stride, pad, G, _ptr(Wq_dev), _ptr(w_scale_dev),
+                                          _ptr(bias_dev), perm_host.ctypes.data_as(C.c_void_p),
+                                          None if x_shift_host is None else x_shift_host.ctypes.data_as(C.c_void_p),
+                                          _stream()))
+    return h
+
+
+def flexiq_layer_destroy(h):
+    _check(lib().flexiq_layer_destroy(h))
+
+
+def flexiq_layer_set_lowbit_path(h, path):
+    _check(lib().flexiq_layer_set_lowbit_path(h, path))
+
+
+def flexiq_set_lowbit_ratio(h, ratio):
+    _check(lib().flexiq_set_lowbit_ratio(h, ratio))
+
+
+def flexiq_get_max_4bit_ch(h) -> int:
+    v = C.c_int()
+    _check(lib().flexiq_get_max_4bit_ch(h, C.byref(v)))
+    return v.value
+
+
+def flexiq_x4_pitch(h, K_lo) -> int:
+    v = C.c_int64()
+    _check(lib().flexiq_x4_pitch(h, K_lo, C.byref(v)))
+    return v.value
+
+
+def flexiq_quantize_lower(h, X_dev, x_dtype, M, x_scale, dynamic_pos, X4_dev, X8_dev, x_shift_out_dev=None,
+                          scratch_dev=None):
+    _check(lib().flexiq_quantize_lower(h, _ptr(X_dev), x_dtype, M, x_scale, int(dynamic_pos), _ptr(X4_dev), _ptr(X8_dev),
+                                       _ptr(x_shift_out_dev), _ptr(scratch_dev), _stream()))
+
+
+def flexiq_mixed_gemm(h, X4_dev, X8_dev, x_shift_dev, M, x_scale, y_scale, out_mode, Y_dev):
+    _check(lib().flexiq_mixed_gemm(h, _ptr(X4_dev), _ptr(X8_dev), _ptr(x_shift_dev), M, x_scale, y_scale, out_mode,
+                                   _ptr(Y_dev), _stream()))
+
+
+def flexiq_mixed_conv(h, X4_dev, X8_dev, x_shift_dev, Nb, H, W, x_scale, y_scale, out_mode, Y_dev):
+    _check(lib().flexiq_mixed_conv(h, _ptr(X4_dev), _ptr(X8_dev), _ptr(x_shift_dev), Nb, H, W, x_scale, y_scale,
+                                   out_mode, _ptr(Y_dev), _stream()))
+
+
+def flexiq_layer_export(h, sw_host=None, w8_host=None, w4_host=None):
+    def hp(a):
+        return None if a is None else a.ctypes.data_as(C.c_void_p)
+    _check(lib().flexiq_layer_export(h, hp(sw_host), hp(w8_host), hp(w4_host)))
+
+
+def flexiq_check_status():
+    _check(lib().flexiq_check_status(_stream()))
+
+
+# ---- convenience wrapper ------------------------------------------------------------
+_TORCH_DTYPE = {}
+
+
+def _dtype_code(t):
+    import torch
+    if not _TORCH_DTYPE:
+        _TORCH_DTYPE.update({torch.float32: DTYPE_F32, torch.float16: DTYPE_F16, torch.bfloat16: DTYPE_BF16,
+                             torch.int8: DTYPE_I8})
+    return _TORCH_DTYPE[t.dtype]
+
+
+class Layer:
+    """Owns one flexiq layer handle plus reusable slab buffers (torch device memory)."""
+
+    def __init__(self, Wq, w_scale, bias, perm, x_shift, G=16, conv=None):
+        import numpy as np
+        self.G = G
+        self.conv = conv  # None or (stride, pad)
+        perm = np.ascontiguousarray(perm, np.int32)
+        x_shift = None if x_shift is None else np.ascontiguousarray(x_shift, np.uint8)
+        if conv is None:
+            self.K, self.N = Wq.shape
+            self.h = flexiq_layer_create_linear(self.K, self.N, G, Wq, w_scale, bias, perm, x_shift)
+        else:
+            self.N, self.R, self.S, self.K = Wq.shape
+            self.h = flexiq_layer_create_conv(self.K, self.N, self.R, self.S, conv[0], conv[1], G, Wq, w_scale, bias,
+                                              perm, x_shift)
+        self.device = Wq.device
+        self._slabs = {}
+
+    def close(self):
+        if self.h is not None:
+            flexiq_layer_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_lowbit_path(self, path):
+        flexiq_layer_set_lowbit_path(self.h, path)
+
+    def set_lowbit_ratio(self, ratio):
+        flexiq_set_lowbit_ratio(self.h, ratio)
+
+    @property
+    def K_lo(self):
+        return flexiq_get_max_4bit_ch(self.h)
+
+    def alloc_slabs(self, M):
+        """Slab buffers sized for any ratio (allocated once per M, reused)."""
+        import torch
+        if M not in self._slabs:
+            x4 = torch.empty(max(M, 1) * self.K + 16, dtype=torch.uint8, device=self.device)
+            x8 = torch.empty(max(M, 1) * self.K + 16, dtype=torch.int8, device=self.device)
+            self._slabs[M] = (x4, x8)
+        return self._slabs[M]
+
+    def quantize_lower(self, X, x_scale, dynamic=False, slabs=None):
+        import torch
+        M = X.numel() // self.K
+        x4, x8 = slabs if slabs is not None else self.alloc_slabs(M)
+        shifts = scratch = None
+        if dynamic:
+            shifts = torch.empty(self.K // self.G, dtype=torch.uint8, device=self.device)
+            scratch = torch.empty(self.K // self.G, dtype=torch.int32, device=self.device)
+        flexiq_quantize_lower(self.h, X, _dtype_code(X), M, x_scale, dynamic, x4, x8, shifts, scratch)
+        return x4, x8, shifts
+
+    def mixed_gemm(self, x4, x8, M, x_scale, y_scale, out_mode, Y=None, x_shift=None):
+        import torch
+        if Y is None:
+            dt = {OUT_ACC_I32: torch.int32, OUT_REQUANT_I8: torch.int8, OUT_DEQUANT_F32: torch.float32}[out_mode]
+            Y = torch.empty((M, self.N), dtype=dt, device=self.device)
+        flexiq_mixed_gemm(self.h, x4, x8, x_shift, M, x_scale, y_scale, out_mode, Y)
+        return Y
+
+    def mixed_conv(self, x4, x8, Nb, H, W, x_scale, y_scale, out_mode, Y=None, x_shift=None):
+        import torch
+        stride, pad = self.conv
+        P = (H + 2 * pad - self.R) // stride + 1
+        Q = (W + 2 * pad - self.S) // stride + 1
+        if Y is None:
+            dt = {OUT_ACC_I32: torch.int32, OUT_REQUANT_I8: torch.int8, OUT_DEQUANT_F32: torch.float32}[out_mode]
+            Y = torch.empty((Nb, P, Q, self.N), dtype=dt, device=self.device)
+        flexiq_mixed_conv(self.h, x4, x8, x_shift, Nb, H, W, x_scale, y_scale, out_mode, Y)
+        return Y

@@ -1,0 +1,45 @@
+"""Offline preparation that feeds the hot path (host side, runs once per layer).
+
+From a calibration batch: per-channel ranges of the quantized activations, the static
+extraction position of every channel group (Sec. 4.1), the error-estimation score
+(activation range x largest weight range, Sec. 4.2) and the greedy nested group order
+whose prefixes are the low-bit sets of every ratio (Sec. 4.2 / Sec. 5).  Written with
+torch tensor ops; it is independent of the test oracle.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+
+def quantize_reference(x: torch.Tensor, scale: float) -> torch.Tensor:
+    """Eq. 1 on the host (calibration only): fp32 division, round-half-even, clip."""
+    s = torch.tensor(scale, dtype=torch.float32)
+    return torch.clamp(torch.round(x.to(torch.float32) / s), -128, 127).to(torch.int8)
+
+
+def _used_bits(lo: torch.Tensor, hi: torch.Tensor) -> torch.Tensor:
+    # magnitude bits needed for [lo, hi]: bit length of hi and of ~lo
+    m = torch.maximum(hi.clamp(min=0), (-lo - 1).clamp(min=0)).to(torch.int64)
+    bits = torch.zeros_like(m)
+    for b in range(8):
+        bits = torch.where(m >= (1 << b), torch.full_like(m, b + 1), bits)
+    return bits
+
+
+def static_preparation(Xcal_q: torch.Tensor, Wq: torch.Tensor, G: int, conv: bool = False):
+    """Returns (group_perm int32 [n_g], x_shift uint8 [n_g] per ORIGINAL group).
+
+    Xcal_q: int8 calibration activations [..., C]; Wq: int8 [K, N] (linear) or
+    [Cout, R, S, Cin] (conv)."""
+    C = Xcal_q.shape[-1]
+    q = Xcal_q.reshape(-1, C).to(torch.int32)
+    lo = q.min(0).values.clamp(max=0)
+    hi = q.max(0).values.clamp(min=0)
+    bits = _used_bits(lo, hi).reshape(-1, G).max(1).values
+    x_shift = (bits - 3).clamp(min=0).to(torch.uint8)
+    w = Wq.to(torch.int32).abs()
+    wmax = w.reshape(-1, C).max(0).values if conv else w.max(1).values
+    score = (torch.maximum(hi, -lo).to(torch.int64) * wmax.to(torch.int64)).reshape(-1, G).max(1).values
+    perm = torch.sort(score, stable=True).indices.to(torch.int32)
+    return np.ascontiguousarray(perm.numpy()), np.ascontiguousarray(x_shift.numpy())

@@ -1,0 +1,80 @@
+// Internal declarations shared by the translation units of libflexiq (host side).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda.h>
+#include <stdint.h>
+#include <stdarg.h>
+
+#include "flexiq.h"
+
+namespace flexiq {
+
+// Layer handle: everything the static part of the method produces (layout
+// post-processing, weight extraction positions, cached 4-bit weights) plus the one
+// run-time knob, max_4bit_ch.
+struct Layer {
+    uint32_t magic;
+    int is_conv;
+    int C;        // input-feature channels (K for a linear layer, Cin for a conv)
+    int N;        // output channels
+    int G;        // channel-group size
+    int n_g;      // C / G
+    int R, S, stride, pad;  // taps (1,1,1,0 for linear)
+    int Kw;       // R*S*C: row length of the slab-order weight matrices
+    int K_lo;     // max_4bit_ch, multiple of G
+    int lowbit_path;
+    int device;
+    // device tables
+    int8_t *w8;      // [N][Kw] slab-order int8 weights
+    int8_t *w8m;     // [N][Kw] (w >> sw) << sw : 4-bit weights at their extraction position
+    uint8_t *w4;     // [N][Kw/2] packed 4-bit weights (w >> sw)
+    uint8_t *sw;     // [n_g][N] weight extraction positions
+    uint8_t *sx;     // [n_g] static activation positions, slab order
+    int32_t *perm;   // [n_g]
+    float *w_scale;  // [N]
+    float *bias;     // [N] or nullptr
+    // host copies
+    int32_t *perm_host;
+    uint8_t *sx_host;
+    // tensor maps over the weights (encoded once)
+    CUtensorMap map_w8[3], map_w8m[3], map_w4[3];  // box rows 64 / 128 / 256
+    int w4_pitch;    // row pitch of w4 in bytes: Kw/2 rounded up to 16
+};
+
+constexpr uint32_t kLayerMagic = 0x464c5851u;  // "FLXQ"
+
+int set_error(int code, const char *fmt, ...);
+int check_device_sm100();
+Layer *as_layer(flexiq_layer_t h);
+
+// driver entry point for tensor-map encoding, resolved through the runtime
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                   const cuuint64_t *, const cuuint64_t *, const int *, const int *,
+                                   cuuint32_t, cuuint32_t, const cuuint32_t *,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn get_encode_tiled();
+EncodeIm2colFn get_encode_im2col();
+
+// 2-D byte tensor map: rows x row_bytes (pitch_bytes between rows), box box_rows x box_bytes.
+int make_map_2d(CUtensorMap *map, const void *base, uint64_t row_bytes, uint64_t rows,
+                uint64_t pitch_bytes, uint32_t box_bytes, uint32_t box_rows, int swizzle_bytes);
+
+int choose_bn(long long m_tiles, int N, int sms);
+int choose_bk(const Layer *L);
+int encode_weight_maps(Layer *L);
+
+
+#define FLEXIQ_CUDA_TRY(expr)                                                         \
+    do {                                                                              \
+        cudaError_t e__ = (expr);                                                     \
+        if (e__ != cudaSuccess)                                                       \
+            return ::flexiq::set_error(FLEXIQ_ERR_CUDA, "%s failed: %s", #expr,       \
+                                       cudaGetErrorString(e__));                      \
+    } while (0)
+
+}  // namespace flexiq

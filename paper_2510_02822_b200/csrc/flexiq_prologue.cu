@@ -1,0 +1,234 @@
+// Activation prologue: quantize (Sec. 2.1, Eq. 1), bit-lower (Sec. 4.1, Fig. 3) and
+// gather the channel groups into slab order (Sec. 5), writing the low-bit slab and the
+// 8-bit slab that the mainloop consumes.  HBM-bound: one pass over X (two in the dynamic
+// extraction-position mode), 128-bit loads and stores, one 16-channel chunk per thread.
+#include "flexiq_internal.h"
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+namespace flexiq {
+
+// Loads the 16 channels starting at p and quantizes them with Eq. 1:
+// q = clip(round_half_even(x / S), -128, 127); IEEE division, no fast-math.
+template <int DTYPE>
+__device__ __forceinline__ void load_quantize16(const void *p, float S, int q[16])
+{
+    if (DTYPE == FLEXIQ_DTYPE_F32) {
+        const float4 *v = reinterpret_cast<const float4 *>(p);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float4 f = __ldg(v + i);
+            q[4 * i + 0] = __float2int_rn(__fdiv_rn(f.x, S));
+            q[4 * i + 1] = __float2int_rn(__fdiv_rn(f.y, S));
+            q[4 * i + 2] = __float2int_rn(__fdiv_rn(f.z, S));
+            q[4 * i + 3] = __float2int_rn(__fdiv_rn(f.w, S));
+        }
+    } else if (DTYPE == FLEXIQ_DTYPE_F16 || DTYPE == FLEXIQ_DTYPE_BF16) {
+        const uint4 *v = reinterpret_cast<const uint4 *>(p);
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const uint4 u = __ldg(v + i);
+            const unsigned w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                float lo, hi;
+                if (DTYPE == FLEXIQ_DTYPE_F16) {
+                    const __half2 h = *reinterpret_cast<const __half2 *>(&w[k]);
+                    lo = __low2float(h);
+                    hi = __high2float(h);
+                } else {  // bf16 widens exactly: the 16 bits are the top half of an fp32
+                    lo = __uint_as_float(w[k] << 16);
+                    hi = __uint_as_float(w[k] & 0xffff0000u);
+                }
+                q[8 * i + 2 * k] = __float2int_rn(__fdiv_rn(lo, S));
+                q[8 * i + 2 * k + 1] = __float2int_rn(__fdiv_rn(hi, S));
+            }
+        }
+    } else {  // already int8
+        const uint4 u = __ldg(reinterpret_cast<const uint4 *>(p));
+        const unsigned w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+#pragma unroll
+            for (int b = 0; b < 4; ++b) q[4 * k + b] = (int)(signed char)((w[k] >> (8 * b)) & 0xff);
+    }
+    if (DTYPE != FLEXIQ_DTYPE_I8) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) q[i] = max(-128, min(127, q[i]));
+    }
+}
+
+template <int DTYPE>
+__device__ __forceinline__ size_t elem_bytes()
+{
+    return DTYPE == FLEXIQ_DTYPE_F32 ? 4 : (DTYPE == FLEXIQ_DTYPE_I8 ? 1 : 2);
+}
+
+__device__ __forceinline__ int position_from_or(unsigned o)
+{
+    const int used = 32 - __clz(o);  // highest bit in use among the folded values
+    return used > 3 ? used - 3 : 0;
+}
+
+// Phase 1 of the dynamic mode (Sec. 4.1): OR of the sign-folded quantized values of each
+// slab group over all rows.  A thread keeps one chunk column and walks rows; lanes that
+// hold the same group merge with a warp reduction, then one shared and one global atomic.
+template <int DTYPE>
+__global__ void group_or_kernel(const void *__restrict__ X, long long M, int K, int G, float S,
+                                const int32_t *__restrict__ perm, unsigned *__restrict__ or_words)
+{
+    extern __shared__ unsigned or_s[];
+    const int n_c16 = K / 16, c_per_g = G / 16, n_g = K / G;
+    for (int i = threadIdx.x; i < n_g; i += blockDim.x) or_s[i] = 0;
+    __syncthreads();
+    // grid-wide thread count is a multiple of n_c16, so each thread keeps its chunk column
+    const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long nthreads = (long long)gridDim.x * blockDim.x;
+    const long long rows_per_pass = nthreads / n_c16;
+    const int c16 = (int)(tid % n_c16);
+    const int j = c16 / c_per_g;
+    unsigned o = 0;
+    if (tid < rows_per_pass * n_c16) {
+        const int src_c = perm[j] * G + (c16 % c_per_g) * 16;
+        for (long long m = tid / n_c16; m < M; m += rows_per_pass) {
+            int q[16];
+            load_quantize16<DTYPE>(reinterpret_cast<const char *>(X) + ((size_t)m * K + src_c) * elem_bytes<DTYPE>(), S, q);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) o |= (unsigned)(q[i] ^ (q[i] >> 31));  // q >= 0 ? q : ~q
+        }
+    }
+    const unsigned peers = __match_any_sync(0xffffffffu, j);
+    const unsigned merged = __reduce_or_sync(peers, o);
+    if ((threadIdx.x & 31) == (__ffs(peers) - 1) && merged) atomicOr(&or_s[j], merged);
+    __syncthreads();
+    for (int i = threadIdx.x; i < n_g; i += blockDim.x)
+        if (or_s[i]) atomicOr(&or_words[i], or_s[i]);
+}
+
+// Quantize + lower + gather.  Thread <-> (row m, 16-channel slab chunk c16).
+//   sx != nullptr : static positions (slab order);  else positions from or_words.
+template <int DTYPE, int PACKED>
+__global__ void quantize_lower_kernel(const void *__restrict__ X, long long M, int K, int G, int K_lo, float S,
+                                      const int32_t *__restrict__ perm, const uint8_t *__restrict__ sx,
+                                      const unsigned *__restrict__ or_words, uint8_t *__restrict__ X4,
+                                      long long x4_pitch, int8_t *__restrict__ X8, uint8_t *__restrict__ sx_out)
+{
+    const int n_c16 = K / 16, c_per_g = G / 16, lo_c16 = K_lo / 16;
+    const int K_hi = K - K_lo;
+    const long long total = M * n_c16;
+    if (sx_out != nullptr && blockIdx.x == 0)
+        for (int j = threadIdx.x; j < K / G; j += blockDim.x) sx_out[j] = (uint8_t)position_from_or(or_words[j]);
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const long long m = idx / n_c16;
+        const int c16 = (int)(idx - m * n_c16);
+        const int j = c16 / c_per_g;
+        const int src_c = perm[j] * G + (c16 % c_per_g) * 16;
+        int q[16];
+        load_quantize16<DTYPE>(reinterpret_cast<const char *>(X) + ((size_t)m * K + src_c) * elem_bytes<DTYPE>(), S, q);
+        if (c16 < lo_c16) {
+            const int s = sx ? (int)sx[j] : position_from_or(or_words[j]);
+            int v[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] = max(-8, min(7, q[i] >> s));  // arithmetic shift, saturate
+            if (PACKED) {
+                unsigned w[2];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    unsigned acc = 0;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) acc |= (unsigned)(v[8 * h + i] & 15) << (4 * i);
+                    w[h] = acc;
+                }
+                *reinterpret_cast<uint2 *>(X4 + m * x4_pitch + (size_t)c16 * 8) = make_uint2(w[0], w[1]);
+            } else {
+                unsigned w[4];
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    unsigned acc = 0;
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc |= (unsigned)((v[4 * h + i] << s) & 0xff) << (8 * i);
+                    w[h] = acc;
+                }
+                *reinterpret_cast<uint4 *>(X4 + m * x4_pitch + (size_t)c16 * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+        } else {
+            unsigned w[4];
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                unsigned acc = 0;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc |= (unsigned)(q[4 * h + i] & 0xff) << (8 * i);
+                w[h] = acc;
+            }
+            *reinterpret_cast<uint4 *>(X8 + m * (long long)K_hi + (size_t)(c16 - lo_c16) * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+    }
+}
+
+template <int DTYPE>
+static int launch_prologue(const Layer *L, const void *X, long long M, float S, int dynamic, uint8_t *X4,
+                           long long pitch, int8_t *X8, uint8_t *sx_out, unsigned *scratch, cudaStream_t st)
+{
+    const int K = L->C, G = L->G;
+    const int n_c16 = K / 16;
+    int sms = 148;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, L->device);
+    const int threads = 256;
+    if (dynamic) {
+        FLEXIQ_CUDA_TRY(cudaMemsetAsync(scratch, 0, sizeof(unsigned) * L->n_g, st));
+        long long want = (M * n_c16 + threads - 1) / threads;
+        long long blocks = want < (long long)sms * 8 ? want : (long long)sms * 8;
+        // thread count must cover at least one full row of chunks
+        while (blocks * threads < n_c16) ++blocks;
+        group_or_kernel<DTYPE><<<(unsigned)blocks, threads, sizeof(unsigned) * L->n_g, st>>>(X, M, K, G, S, L->perm, scratch);
+        FLEXIQ_CUDA_TRY(cudaGetLastError());
+    }
+    long long want = (M * n_c16 + threads - 1) / threads;
+    long long blocks = want < (long long)sms * 16 ? want : (long long)sms * 16;
+    const uint8_t *sx = dynamic ? nullptr : L->sx;
+    if (L->lowbit_path == FLEXIQ_LOWBIT_PACKED_U4)
+        quantize_lower_kernel<DTYPE, 1><<<(unsigned)blocks, threads, 0, st>>>(X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, dynamic ? sx_out : nullptr);
+    else
+        quantize_lower_kernel<DTYPE, 0><<<(unsigned)blocks, threads, 0, st>>>(X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, dynamic ? sx_out : nullptr);
+    FLEXIQ_CUDA_TRY(cudaGetLastError());
+    return FLEXIQ_OK;
+}
+
+}  // namespace flexiq
+
+using namespace flexiq;
+
+extern "C" int flexiq_quantize_lower(flexiq_layer_t layer, const void *X_dev, int x_dtype, int64_t M, float x_scale,
+                                     int dynamic_pos, uint8_t *X4_dev, int8_t *X8_dev, uint8_t *x_shift_out_dev,
+                                     uint32_t *scratch_dev, void *stream)
+{
+    Layer *L = as_layer(layer);
+    if (!L) return set_error(FLEXIQ_ERR_INVALID_ARG, "not a live flexiq layer handle");
+    if (M < 0) return set_error(FLEXIQ_ERR_INVALID_ARG, "M = %lld is negative", (long long)M);
+    if (x_dtype < FLEXIQ_DTYPE_F32 || x_dtype > FLEXIQ_DTYPE_I8)
+        return set_error(FLEXIQ_ERR_INVALID_ARG, "unknown x_dtype %d", x_dtype);
+    if (x_dtype != FLEXIQ_DTYPE_I8 && !(x_scale > 0.0f))
+        return set_error(FLEXIQ_ERR_INVALID_ARG, "x_scale %g must be positive", (double)x_scale);
+    if (M == 0) return FLEXIQ_OK;
+    const int K_lo = L->K_lo, K_hi = L->C - K_lo;
+    if (!X_dev) return set_error(FLEXIQ_ERR_INVALID_ARG, "X_dev is NULL");
+    if (K_lo > 0 && !X4_dev) return set_error(FLEXIQ_ERR_INVALID_ARG, "X4_dev is NULL but K_lo = %d", K_lo);
+    if (K_hi > 0 && !X8_dev) return set_error(FLEXIQ_ERR_INVALID_ARG, "X8_dev is NULL but K_hi = %d", K_hi);
+    if (dynamic_pos && (!x_shift_out_dev || !scratch_dev))
+        return set_error(FLEXIQ_ERR_INVALID_ARG, "dynamic_pos needs x_shift_out_dev and scratch_dev");
+    if ((reinterpret_cast<uintptr_t>(X_dev) | reinterpret_cast<uintptr_t>(X4_dev) | reinterpret_cast<uintptr_t>(X8_dev)) & 15)
+        return set_error(FLEXIQ_ERR_INVALID_ARG, "X_dev, X4_dev and X8_dev must be 16-byte aligned");
+    int rc = check_device_sm100();
+    if (rc) return rc;
+    int64_t pitch = 0;
+    flexiq_x4_pitch(layer, K_lo, &pitch);
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    switch (x_dtype) {
+        case FLEXIQ_DTYPE_F32: return launch_prologue<FLEXIQ_DTYPE_F32>(L, X_dev, M, x_scale, dynamic_pos, X4_dev, pitch, X8_dev, x_shift_out_dev, scratch_dev, st);
+        case FLEXIQ_DTYPE_F16: return launch_prologue<FLEXIQ_DTYPE_F16>(L, X_dev, M, x_scale, dynamic_pos, X4_dev, pitch, X8_dev, x_shift_out_dev, scratch_dev, st);
+        case FLEXIQ_DTYPE_BF16: return launch_prologue<FLEXIQ_DTYPE_BF16>(L, X_dev, M, x_scale, dynamic_pos, X4_dev, pitch, X8_dev, x_shift_out_dev, scratch_dev, st);
+        default: return launch_prologue<FLEXIQ_DTYPE_I8>(L, X_dev, M, x_scale, dynamic_pos, X4_dev, pitch, X8_dev, x_shift_out_dev, scratch_dev, st);
+    }
+}
