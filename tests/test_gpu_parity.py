@@ -1,0 +1,222 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the
+same seeded inputs.  Integer results (slabs, int32 accumulators, int8 outputs) must be
+bit-exact; dequantized fp32 outputs within 1e-6 relative."""
+import numpy as np
+import pytest
+import torch
+
+import helpers
+import oracle
+from paper_2510_02822_b200 import binding as fx
+from paper_2510_02822_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+F32_RTOL = 1e-6
+
+
+@pytest.fixture(scope="module")
+def dev():
+    return torch.device("cuda:0")
+
+
+def _layer(case, dev, perm, sx_group, conv=False, path=fx.LOWBIT_MASKED_I8):
+    L = fx.Layer(torch.from_numpy(case.Wq).to(dev), torch.from_numpy(case.w_scale).to(dev),
+                 torch.from_numpy(case.bias).to(dev), perm, sx_group, case.G,
+                 conv=(case.stride, case.pad) if conv else None)
+    L.set_lowbit_path(path)
+    return L
+
+
+def _check_outputs(L, case, x4, x8, acc_e, dev, conv=False, x_shift=None):
+    shape = acc_e.shape
+    for mode, dt in ((fx.OUT_ACC_I32, torch.int32), (fx.OUT_REQUANT_I8, torch.int8), (fx.OUT_DEQUANT_F32, torch.float32)):
+        Y, guard_ok = helpers.with_guard(torch, shape, dt, dev)
+        if conv:
+            L.mixed_conv(x4, x8, case.Nb, case.H, case.W, case.x_scale, case.y_scale, mode, Y=Y, x_shift=x_shift)
+        else:
+            L.mixed_gemm(x4, x8, shape[0], case.x_scale, case.y_scale, mode, Y=Y, x_shift=x_shift)
+        torch.cuda.synchronize()
+        fx.flexiq_check_status()
+        guard_ok()
+        got = Y.cpu().numpy()
+        if mode == fx.OUT_ACC_I32:
+            assert np.array_equal(got, acc_e)
+        elif mode == fx.OUT_REQUANT_I8:
+            assert np.array_equal(got, oracle.epilogue_i8(acc_e, case.x_scale, case.w_scale, case.bias, case.y_scale))
+        else:
+            exp = oracle.epilogue_f32(acc_e, case.x_scale, case.w_scale, case.bias)
+            assert np.all(np.abs(got - exp) <= F32_RTOL * np.abs(exp))
+
+
+def _run_linear(case, dev, ratios, shifts=None, x_dtype=torch.float32, path=fx.LOWBIT_MASKED_I8, dynamic=False):
+    perm, sxg, sxs, sw = helpers.prepare_linear(case, shifts)
+    L = _layer(case, dev, perm, sxg, path=path)
+    X = torch.from_numpy(case.X).to(dev).to(x_dtype)
+    q = oracle.quantize(X.float().cpu().numpy(), case.x_scale) if x_dtype != torch.int8 else X.cpu().numpy()
+    for r in ratios:
+        L.set_lowbit_ratio(r)
+        nl = oracle.n_low(r, case.K // case.G)
+        K_lo = nl * case.G
+        assert L.K_lo == K_lo
+        x4, x8, shifts_dev = L.quantize_lower(X, case.x_scale, dynamic=dynamic)
+        torch.cuda.synchronize()
+        sx_use = sxs
+        if dynamic:
+            sx_use = oracle.dynamic_positions(q, case.G, perm)
+            assert np.array_equal(shifts_dev.cpu().numpy(), sx_use)
+        e4, e8 = oracle.make_slabs(q, case.G, perm, sx_use, nl)
+        if K_lo:
+            pitch = fx.flexiq_x4_pitch(L.h, K_lo)
+            g4 = x4[:case.M * pitch].view(case.M, pitch).cpu().numpy()
+            if path == fx.LOWBIT_MASKED_I8:
+                assert np.array_equal(g4.view(np.int8), helpers.masked_slab(e4, case.G, sx_use, nl))
+            else:
+                assert np.array_equal(g4[:, :K_lo // 2], e4[:, :K_lo // 2])
+        if case.K - K_lo:
+            assert np.array_equal(x8[:case.M * (case.K - K_lo)].view(case.M, -1).cpu().numpy(), e8)
+        acc_e = oracle.mixed_gemm_acc(q, case.Wq, case.G, perm, sx_use, sw, nl)
+        _check_outputs(L, case, x4, x8, acc_e, dev, x_shift=shifts_dev)
+    L.close()
+
+
+def test_layer_tables(dev):
+    case = inputs.ranged_linear("t", 64, 192, 80, 32, seed=1, group_structured=True)
+    perm, sxg, sxs, sw = helpers.prepare_linear(case)
+    L = _layer(case, dev, perm, sxg)
+    sw_g = np.empty_like(sw)
+    w8 = np.empty((80, 192), np.int8)
+    w4 = np.empty((80, 96), np.uint8)
+    fx.flexiq_layer_export(L.h, sw_g, w8, w4)
+    assert np.array_equal(sw_g, sw)
+    cols = np.concatenate([np.arange(g * 32, (g + 1) * 32) for g in perm])
+    ws = case.Wq[cols].T.astype(np.int16)
+    assert np.array_equal(w8, ws)
+    sh = np.repeat(sw, 32, axis=0).T.astype(np.int16)
+    n4 = (ws >> sh) & 15
+    assert np.array_equal(w4, (n4[:, 0::2] | (n4[:, 1::2] << 4)).astype(np.uint8))
+    L.close()
+
+
+def test_config1_single_gemm_all_ratios(dev):
+    _run_linear(inputs.config1(), dev, inputs.RATIOS)
+
+
+def test_config1_int8_input_gives_identical_slabs(dev):
+    case = inputs.config1()
+    case.X = oracle.quantize(case.X, case.x_scale)  # the int8 X of the configuration
+    _run_linear(case, dev, [0.5], x_dtype=torch.int8)
+
+
+@pytest.mark.parametrize("M,K,N,G", [(1, 128, 16, 16), (129, 256, 48, 16), (300, 128, 272, 32), (197, 384, 384, 16),
+                                     (515, 192, 144, 64), (257, 64, 64, 16), (1000, 1024, 80, 16)])
+def test_ragged_shapes_with_saturating_positions(dev, M, K, N, G):
+    case = inputs.ranged_linear("r", M, K, N, G, seed=M + K, group_structured=True)
+    rng = np.random.default_rng(K + N)
+    shifts = rng.integers(0, 5, K // G).astype(np.uint8)  # arbitrary positions: some values saturate
+    _run_linear(case, dev, [0.0, 0.5, 1.0, 1.0 / (K // G)], shifts=shifts)
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+def test_half_precision_inputs(dev, dtype):
+    _run_linear(inputs.ranged_linear("h", 200, 256, 64, 16, seed=6, group_structured=True), dev, [0.5], x_dtype=dtype)
+
+
+def test_dynamic_positions(dev):
+    case = inputs.ranged_linear("dyn", 333, 384, 96, 16, seed=21, group_structured=True)
+    _run_linear(case, dev, [0.5, 1.0], dynamic=True)
+    case = inputs.ranged_linear("dyn2", 77, 64, 32, 32, seed=22, group_structured=True)  # fewer groups than lanes
+    _run_linear(case, dev, [1.0], dynamic=True)
+
+
+def test_deit_small_batch_shapes(dev):
+    for case in inputs.config4(batch=1):
+        _run_linear(case, dev, [0.0, 0.25, 0.5, 0.75, 1.0])
+
+
+def test_empty_batch_and_argument_errors(dev):
+    case = inputs.ranged_linear("e", 16, 128, 32, 16, seed=3)
+    perm, sxg, sxs, sw = helpers.prepare_linear(case)
+    L = _layer(case, dev, perm, sxg)
+    L.set_lowbit_ratio(0.5)
+    fx.flexiq_quantize_lower(L.h, None, fx.DTYPE_F32, 0, 1.0, 0, None, None)  # M == 0: no-op
+    fx.flexiq_mixed_gemm(L.h, None, None, None, 0, 1.0, 1.0, fx.OUT_ACC_I32, None)
+    x4, x8 = L.alloc_slabs(16)
+    with pytest.raises(fx.FlexiqError) as e:
+        fx.flexiq_mixed_gemm(L.h, None, x8, None, 16, 1.0, 1.0, fx.OUT_ACC_I32, x8)
+    assert e.value.code == fx.ERR_INVALID_ARG
+    with pytest.raises(fx.FlexiqError):
+        fx.flexiq_set_lowbit_ratio(L.h, 1.5)
+    with pytest.raises(fx.FlexiqError):
+        fx.flexiq_mixed_conv(L.h, x4, x8, None, 1, 4, 4, 1.0, 1.0, fx.OUT_ACC_I32, x8)
+    with pytest.raises(fx.FlexiqError):
+        fx.flexiq_mixed_gemm(L.h, x4[1:], x8, None, 16, 1.0, 1.0, fx.OUT_ACC_I32, x8)  # misaligned
+    L.close()
+
+
+def test_ratio_switch_is_host_only_and_nested(dev):
+    case = inputs.config1()
+    perm, sxg, sxs, sw = helpers.prepare_linear(case)
+    L = _layer(case, dev, perm, sxg)
+    seen = []
+    for r in (0.0, 0.25, 0.5, 0.75, 1.0, 0.5, 0.0):
+        L.set_lowbit_ratio(r)
+        seen.append(L.K_lo)
+    assert seen == [0, 96, 192, 288, 384, 192, 0]
+    L.close()
+
+
+# ---------------------------------------------------------------- convolution
+def _run_conv(case, dev, ratios, shifts=None):
+    perm, sxg, sxs, sw = helpers.prepare_conv(case, shifts)
+    L = _layer(case, dev, perm, sxg, conv=True)
+    X = torch.from_numpy(case.X).to(dev)
+    q = oracle.quantize(case.X, case.x_scale)
+    for r in ratios:
+        L.set_lowbit_ratio(r)
+        nl = oracle.n_low(r, case.C // case.G)
+        x4, x8, _ = L.quantize_lower(X, case.x_scale)
+        acc_e = oracle.mixed_conv_acc(q, case.Wq, case.stride, case.pad, case.G, perm, sxs, sw, nl)
+        _check_outputs(L, case, x4, x8, acc_e, dev, conv=True)
+    L.close()
+
+
+@pytest.mark.parametrize("Nb,H,C,Cout,R,stride", [(2, 14, 128, 64, 3, 1), (3, 28, 64, 64, 3, 1), (5, 7, 256, 128, 3, 1),
+                                                  (2, 14, 128, 64, 3, 2), (2, 14, 128, 256, 1, 1), (1, 9, 192, 48, 3, 1)])
+def test_conv_shapes(dev, Nb, H, C, Cout, R, stride):
+    case = inputs.resnet_conv("c", Nb, H, C, Cout, R, seed=H + C, stride=stride)
+    rng = np.random.default_rng(H * C)
+    shifts = rng.integers(0, 5, C // case.G).astype(np.uint8)
+    _run_conv(case, dev, [0.0, 0.25, 0.5, 1.0], shifts=shifts)
+
+
+def test_resnet50_conv_full_size_56(dev):
+    # full-size 3x3 C=64 @56x56 at batch 4 (the bench runs batch 32; rows are independent)
+    case = inputs.resnet_conv("c56", 4, 56, 64, 64, 3, seed=3000)
+    _run_conv(case, dev, [0.0, 0.5, 1.0])
+
+
+# ---------------------------------------------------------------- full-size, sampled rows
+@pytest.mark.parametrize("layer", [0, 3])
+def test_vit_b_full_size_sampled_rows(dev, layer):
+    name, K, N = inputs.VIT_B_LAYERS[layer]
+    case = inputs.vit_linear(f"cfg2_{name}", 64 * 197, K, N, 16, seed=2000 + layer)
+    perm, sxg, sxs, sw = helpers.prepare_linear(case)
+    L = _layer(case, dev, perm, sxg)
+    X = torch.from_numpy(case.X).to(dev)
+    rows = np.unique(np.concatenate([np.arange(0, case.M, 97), np.arange(case.M - 70, case.M), np.arange(120, 136)])).astype(np.int64)
+    q_rows = oracle.quantize(case.X[rows], case.x_scale)
+    for r in (0.0, 0.5, 1.0):
+        L.set_lowbit_ratio(r)
+        nl = oracle.n_low(r, K // 16)
+        x4, x8, _ = L.quantize_lower(X, case.x_scale)
+        acc_e = oracle.mixed_gemm_acc(q_rows, case.Wq, 16, perm, sxs, sw, nl)
+        acc = L.mixed_gemm(x4, x8, case.M, case.x_scale, case.y_scale, fx.OUT_ACC_I32)
+        y8 = L.mixed_gemm(x4, x8, case.M, case.x_scale, case.y_scale, fx.OUT_REQUANT_I8)
+        torch.cuda.synchronize()
+        fx.flexiq_check_status()
+        assert np.array_equal(acc.cpu().numpy()[rows], acc_e)
+        assert np.array_equal(y8.cpu().numpy()[rows], oracle.epilogue_i8(acc_e, case.x_scale, case.w_scale, case.bias, case.y_scale))
+        # property that holds at any size: results are bit-identical run to run
+        acc2 = L.mixed_gemm(x4, x8, case.M, case.x_scale, case.y_scale, fx.OUT_ACC_I32)
+        assert torch.equal(acc, acc2)
+    L.close()
