@@ -51,8 +51,8 @@ class ClockSampler:
         self.samples = []
         self.proc = None
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "50",
-                                          "-i", str(gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "20",
+                                          "-i", str(gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -80,7 +80,10 @@ class ClockSampler:
             for n, v in zip(names, f[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(sm)}
+        out = {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(sm)}
+        if not sm:
+            out["note"] = (self.samples[-1][1] if self.samples else "no output from nvidia-smi")[:160]
+        return out
 
 
 def layer_ops(case):
@@ -108,6 +111,7 @@ def run_ours(args):
     fx.lib()  # fails loudly when the CUDA library is missing
 
     cases = inputs.config2(batch=64)
+    sampler = ClockSampler(local_rank) if rank == 0 else None  # started early: nvidia-smi takes a while to report
     layers, Xd, Xh, slabs, Yd, Yh = [], [], [], [], [], []
     for c in cases:
         qcal = calib.quantize_reference(torch.from_numpy(c.Xcal), c.x_scale)
@@ -150,7 +154,6 @@ def run_ours(args):
     torch.cuda.synchronize()
     fx.flexiq_check_status()
 
-    sampler = ClockSampler(local_rank) if rank == 0 else None
     # ---- timed region: K steps, device-resident inputs --------------------------------
     dist.barrier()
     torch.cuda.synchronize()

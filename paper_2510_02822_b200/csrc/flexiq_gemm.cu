@@ -8,8 +8,7 @@
 // registers for the shift.  A persistent, warp-specialised CTA per SM:
 //   warp 0      TMA producer (tiled loads for linear layers, im2col loads for convs)
 //   warp 1      TMEM allocation + single-thread MMA issue
-//   warps 2..5  epilogue: tcgen05.ld, scale / bias / round / clip, 128-bit stores
-//   warps 6..9  (packed low-bit path only) widen 4-bit slabs to 8-bit operands in smem
+//   warps 2..9  epilogue: tcgen05.ld, scale / bias / round / clip, staged coalesced stores
 // Two TMEM accumulators let the epilogue of tile i overlap the mainloop of tile i+1.
 // Every wait is bounded; an expired wait raises the status word and the CTA drains.
 #include "flexiq_internal.h"
@@ -20,9 +19,15 @@ namespace flexiq {
 __device__ unsigned int g_status_word = 0;
 
 constexpr int BM = 128;
-constexpr int kNumEpiWarps = 4;
-constexpr int kThreadsMasked = 32 * (2 + kNumEpiWarps);
+constexpr int kNumEpiWarps = 8;                       // two per TMEM lane quadrant
+constexpr int kThreads = 32 * (2 + kNumEpiWarps);
 constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr int kABytes = BM * 128;                     // A stage (BK <= 128 bytes per row)
+constexpr int kStageRegion = 196608;                  // shared memory given to the operand ring
+constexpr int kStagingPerWarp = 2048;                 // 32 rows x 64 B output staging per epilogue warp
+constexpr int kFactorsPerWarp = 256;                  // alpha[32], beta[32] of the current column chunk
+constexpr int kMaxStages = 8;
+constexpr int kSmemBytes = kStageRegion + kNumEpiWarps * (kStagingPerWarp + kFactorsPerWarp) + 256 + 1024;
 
 struct GemmParams {
     long long M;         // rows of the implicit GEMM (tokens or output pixels)
@@ -31,37 +36,28 @@ struct GemmParams {
     int C_lo, C_hi;      // max_4bit_ch and the rest
     int T, S;            // taps R*S and S
     int BK;              // K bytes per stage: 128 or 64
+    int BN;              // tile width: 64, 128, 192 or 256
+    int stages;          // depth of the operand ring
     int nb_lo, nb_hi;    // k-blocks per tap in the low / high slab
     int im2col;          // A operand through im2col-mode TMA
     int P, Q, stride, pad;
     int out_mode;
-    float x_scale, y_scale;
-    const float *w_scale;
-    const float *bias;
+    const float *alpha;  // [N] per-output-channel multiplier of this call
+    const float *beta;   // [N] per-output-channel addend of this call
     void *Y;
     int m_tiles, n_tiles;
-};
-
-template <int BN>
-struct Cfg {
-    static constexpr int kStages = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
-    static constexpr int kABytes = BM * 128;
-    static constexpr int kBBytes = BN * 128;
-    static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kTmemCols = 2 * BN;
-    // stages | alpha/beta [2][BN] each | barriers | tmem ptr, abort flag
-    static constexpr int kSmemBytes = kStages * kStageBytes + 4 * BN * 4 + (2 * kStages + 4) * 8 + 16 + 1024;
 };
 
 // Bounded wait.  Returns false after the limit or when another role already gave up;
 // the caller then leaves its loops and the CTA drains.
 __device__ __forceinline__ bool wait_bounded(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int where)
 {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
         if (ptx::mbar_try_wait(bar, parity)) return true;
-        if (it > 64) {
+        if (it > 256) {
             if (*abort_flag) return false;
-            __nanosleep(it > 4096 ? 256 : 32);
+            __nanosleep(it > 8192 ? 256 : 20);
         }
     }
     *abort_flag = 1;
@@ -69,70 +65,100 @@ __device__ __forceinline__ bool wait_bounded(uint64_t *bar, uint32_t parity, vol
     return false;
 }
 
-// All epilogue threads agree on whether the wait succeeded, so that no warp runs ahead
-// to the next tile's barrier while another one has left the loop.
-__device__ __forceinline__ bool epilogue_vote(bool ok)
+// Walks the K blocks of one output tile in the order both the producer and the MMA
+// issuer use: the low slab (all taps, all channel blocks), then the high slab.
+struct KBlockIter {
+    int part, tap, cb, tap_r, tap_s;
+    __device__ __forceinline__ void reset(const GemmParams &p)
+    {
+        part = p.nb_lo > 0 ? 0 : 1;
+        tap = cb = tap_r = tap_s = 0;
+    }
+    __device__ __forceinline__ void next(const GemmParams &p)
+    {
+        const int nb = part == 0 ? p.nb_lo : p.nb_hi;
+        if (++cb == nb) {
+            cb = 0;
+            if (++tap_s == p.S) { tap_s = 0; ++tap_r; }
+            if (++tap == p.T) { tap = tap_r = tap_s = 0; ++part; }
+        }
+    }
+};
+
+// two int32 -> two saturated int8 in the low half, upper half taken from c's low half
+__device__ __forceinline__ unsigned pack2_sat_s8(int hi, int lo, unsigned c)
 {
-    uint32_t all;
-    asm volatile(
-        "{\n"
-        ".reg .pred p, q;\n"
-        "setp.ne.u32 p, %1, 0;\n"
-        "bar.red.and.pred q, 2, %2, p;\n"
-        "selp.u32 %0, 1, 0, q;\n"
-        "}\n"
-        : "=r"(all)
-        : "r"((uint32_t)ok), "n"(32 * kNumEpiWarps)
-        : "memory");
-    return all != 0;
+    unsigned d;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(hi), "r"(lo), "r"(c));
+    return d;
+}
+// round-half-even, saturate to int8, pack little-endian (y0 in the lowest byte)
+__device__ __forceinline__ unsigned requant4(float y0, float y1, float y2, float y3)
+{
+    const unsigned top = pack2_sat_s8(__float2int_rn(y3), __float2int_rn(y2), 0u);
+    return pack2_sat_s8(__float2int_rn(y1), __float2int_rn(y0), top);
 }
 
-__device__ __forceinline__ unsigned pack4_sat_i8(float y0, float y1, float y2, float y3)
+// Staging buffer of one epilogue warp: 32 rows x 64 B, 16-byte units XOR-swizzled so that
+// both the row-per-lane writes and the two-rows-per-quarter-warp reads avoid bank conflicts.
+__device__ __forceinline__ uint4 *staging_unit(uint8_t *stg, int row, int unit)
 {
-    const int a = max(-128, min(127, __float2int_rn(y0)));
-    const int b = max(-128, min(127, __float2int_rn(y1)));
-    const int c = max(-128, min(127, __float2int_rn(y2)));
-    const int d = max(-128, min(127, __float2int_rn(y3)));
-    return (unsigned)(a & 0xff) | ((unsigned)(b & 0xff) << 8) | ((unsigned)(c & 0xff) << 16) | ((unsigned)d << 24);
+    return reinterpret_cast<uint4 *>(stg + row * 64 + ((unit ^ ((row >> 1) & 3)) << 4));
 }
 
-template <int BN>
-__global__ void __launch_bounds__(kThreadsMasked, 1)
+// Coalesced copy of the staged rows to global memory: `upr` (2 or 4) 16-byte units per row.
+__device__ __forceinline__ void flush_staging(uint8_t *stg, int upr, uint8_t *gbase, long long row_pitch_bytes,
+                                              int rows_valid, int units_valid, int lane)
+{
+    __syncwarp();
+    const int sh = upr == 4 ? 2 : 1;
+    for (int u = lane; u < 32 * upr; u += 32) {
+        const int row = u >> sh, j = u & (upr - 1);
+        if (row < rows_valid && j < units_valid)
+            *reinterpret_cast<uint4 *>(gbase + row * row_pitch_bytes + j * 16) = *staging_unit(stg, row, j);
+    }
+    __syncwarp();
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
 mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_constant__ CUtensorMap mapA_hi,
                   const __grid_constant__ CUtensorMap mapB_lo, const __grid_constant__ CUtensorMap mapB_hi,
                   const GemmParams p)
 {
-    using C = Cfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t *stage_base = smem;
-    float *alpha_s = reinterpret_cast<float *>(smem + C::kStages * C::kStageBytes);  // [2][BN]
-    float *beta_s = alpha_s + 2 * BN;                                               // [2][BN]
-    uint64_t *full_bar = reinterpret_cast<uint64_t *>(beta_s + 2 * BN);
-    uint64_t *empty_bar = full_bar + C::kStages;
-    uint64_t *tmem_full = empty_bar + C::kStages;
+    uint8_t *staging = smem + kStageRegion;
+    uint8_t *factors = staging + kNumEpiWarps * kStagingPerWarp;
+    uint64_t *full_bar = reinterpret_cast<uint64_t *>(factors + kNumEpiWarps * kFactorsPerWarp);
+    uint64_t *empty_bar = full_bar + kMaxStages;
+    uint64_t *tmem_full = empty_bar + kMaxStages;
     uint64_t *tmem_empty = tmem_full + 2;
     uint32_t *tmem_ptr_s = reinterpret_cast<uint32_t *>(tmem_empty + 2);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_ptr_s + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int BN = p.BN;
+    const int stage_bytes = kABytes + BN * 128;
     const int num_tiles = p.m_tiles * p.n_tiles;
-    const int kb_lo = p.T * p.nb_lo, kb_total = p.T * (p.nb_lo + p.nb_hi);
+    const int kb_total = p.T * (p.nb_lo + p.nb_hi);
+    const uint32_t tmem_cols = BN <= 64 ? 128u : (BN <= 128 ? 256u : 512u);
+    const uint32_t buf_stride = tmem_cols / 2;  // column offset of the second accumulator
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < C::kStages; ++s) {
+        for (int s = 0; s < p.stages; ++s) {
             ptx::mbar_init(&full_bar[s], 1);
             ptx::mbar_init(&empty_bar[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(&tmem_full[b], 1);
-            ptx::mbar_init(&tmem_empty[b], 32 * kNumEpiWarps);
+            ptx::mbar_init(&tmem_empty[b], kNumEpiWarps);
         }
         *abort_flag = 0;
         ptx::fence_mbar_init();
     }
     if (warp == 1) {
-        ptx::tmem_alloc(tmem_ptr_s, C::kTmemCols);
+        ptx::tmem_alloc(tmem_ptr_s, tmem_cols);
         ptx::tmem_relinquish();
     }
     ptx::tc_fence_before_sync();
@@ -164,37 +190,35 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                     pix_h = (rem / p.Q) * p.stride - p.pad;
                     pix_w = (rem % p.Q) * p.stride - p.pad;
                 }
-                for (int kb = 0; kb < kb_total; ++kb) {
+                KBlockIter it;
+                it.reset(p);
+                for (int kb = 0; kb < kb_total; ++kb, it.next(p)) {
                     if (!wait_bounded(&empty_bar[stage], phase ^ 1, abort_flag, 1)) { ok = false; break; }
-                    const bool low = kb < kb_lo;
-                    const int kk = low ? kb : kb - kb_lo;
-                    const int nb = low ? p.nb_lo : p.nb_hi;
-                    const int tap = kk / nb, cb = kk - tap * nb;
-                    uint8_t *sa = stage_base + stage * C::kStageBytes;
-                    uint8_t *sb = sa + C::kABytes;
+                    const bool low = it.part == 0;
+                    uint8_t *sa = stage_base + stage * stage_bytes;
                     ptx::mbar_expect_tx(&full_bar[stage], tx_bytes);
                     const CUtensorMap *ma = low ? &mapA_lo : &mapA_hi;
                     if (p.im2col)
-                        ptx::tma_load_im2col_4d(sa, ma, &full_bar[stage], cb * p.BK, pix_w, pix_h, pix_n,
-                                                (uint16_t)(tap % p.S), (uint16_t)(tap / p.S));
+                        ptx::tma_load_im2col_4d(sa, ma, &full_bar[stage], it.cb * p.BK, pix_w, pix_h, pix_n,
+                                                (uint16_t)it.tap_s, (uint16_t)it.tap_r);
                     else
-                        ptx::tma_load_2d(sa, ma, &full_bar[stage], cb * p.BK, (int)m0);
+                        ptx::tma_load_2d(sa, ma, &full_bar[stage], it.cb * p.BK, (int)m0);
                     // weights: slab-order [N][T*C]; the low slab's forms start each tap at channel 0,
                     // the 8-bit form of the high groups at channel C_lo
-                    ptx::tma_load_2d(sb, low ? &mapB_lo : &mapB_hi, &full_bar[stage],
-                                     tap * p.C + (low ? 0 : p.C_lo) + cb * p.BK, n0);
+                    ptx::tma_load_2d(sa + kABytes, low ? &mapB_lo : &mapB_hi, &full_bar[stage],
+                                     it.tap * p.C + (low ? 0 : p.C_lo) + it.cb * p.BK, n0);
                     ++issued;
-                    if (++stage == C::kStages) { stage = 0; phase ^= 1; }
+                    if (++stage == p.stages) { stage = 0; phase ^= 1; }
                 }
             }
             if (!ok) {
                 // drain: let the copies already in flight land before the CTA retires
-                const int n_back = issued < C::kStages ? (int)issued : C::kStages;
+                const int n_back = issued < p.stages ? (int)issued : p.stages;
                 int s = stage;
                 uint32_t ph = phase;
                 for (int i = 0; i < n_back; ++i) {
-                    if (--s < 0) { s = C::kStages - 1; ph ^= 1; }
-                    for (uint32_t it = 0; it < (1u << 16); ++it) {
+                    if (--s < 0) { s = p.stages - 1; ph ^= 1; }
+                    for (uint32_t w = 0; w < (1u << 16); ++w) {
                         if (ptx::mbar_try_wait(&full_bar[s], ph)) break;
                         __nanosleep(64);
                     }
@@ -205,6 +229,9 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
         // ------------------------------------------------------------- MMA issuer
         if (lane == 0) {
             const uint32_t idesc = ptx::idesc_i8(BM, BN);
+            const uint64_t adesc0 = ptx::smem_desc(ptx::smem_u32(stage_base), p.BK);
+            const uint64_t bdesc0 = ptx::smem_desc(ptx::smem_u32(stage_base + kABytes), p.BK);
+            const uint64_t stage_step = (uint64_t)(stage_bytes >> 4);
             int stage = 0;
             uint32_t phase = 0;
             int buf = 0;
@@ -213,23 +240,23 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 if (!wait_bounded(&tmem_empty[buf], buf_phase ^ 1, abort_flag, 2)) break;
                 ptx::tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-                for (int kb = 0; kb < kb_total; ++kb) {
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * buf_stride;
+                KBlockIter it;
+                it.reset(p);
+                uint32_t accumulate = 0;
+                for (int kb = 0; kb < kb_total; ++kb, it.next(p)) {
                     if (!wait_bounded(&full_bar[stage], phase, abort_flag, 3)) { ok = false; break; }
-                    ptx::tc_fence_after_sync();
-                    const bool low = kb < kb_lo;
-                    const int kk = low ? kb : kb - kb_lo;
-                    const int nb = low ? p.nb_lo : p.nb_hi;
-                    const int cb = kk % nb;
-                    const int valid = min(p.BK, (low ? p.C_lo : p.C_hi) - cb * p.BK);
-                    const int ksteps = (valid + 31) >> 5;
-                    const uint32_t sa = ptx::smem_u32(stage_base + stage * C::kStageBytes);
-                    const uint64_t adesc = ptx::smem_desc(sa, p.BK);
-                    const uint64_t bdesc = ptx::smem_desc(sa + C::kABytes, p.BK);
-                    for (int k = 0; k < ksteps; ++k)  // 32 bytes of K per instruction: +2 in 16-byte units
-                        ptx::mma_i8(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0);
+                    const int nb = it.part == 0 ? p.nb_lo : p.nb_hi;
+                    int ksteps = p.BK >> 5;
+                    if (it.cb == nb - 1) ksteps = ((it.part == 0 ? p.C_lo : p.C_hi) - it.cb * p.BK + 31) >> 5;
+                    const uint64_t adesc = adesc0 + stage_step * stage;
+                    const uint64_t bdesc = bdesc0 + stage_step * stage;
+                    for (int k = 0; k < ksteps; ++k) {  // 32 bytes of K per instruction: +2 in 16-byte units
+                        ptx::mma_i8(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, accumulate);
+                        accumulate = 1;
+                    }
                     ptx::mma_commit(&empty_bar[stage]);
-                    if (++stage == C::kStages) { stage = 0; phase ^= 1; }
+                    if (++stage == p.stages) { stage = 0; phase ^= 1; }
                 }
                 if (ok) ptx::mma_commit(&tmem_full[buf]);
                 if ((buf ^= 1) == 0) buf_phase ^= 1;
@@ -237,79 +264,106 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
         }
     } else {
         // ------------------------------------------------------------- epilogue
-        const int quad = warp & 3;  // TMEM lane quadrant this warp may read
-        const int et = threadIdx.x - 64;
+        // warp e owns TMEM lane quadrant (warp & 3) and one half of the tile's columns;
+        // the warps do not synchronise with one another.
+        const int e = warp - 2;
+        const int quad = warp & 3;
+        const int half = e >> 2;
+        const int cols_per_warp = BN >> 1;           // 32, 64, 96 or 128
+        const int n_chunks = cols_per_warp >> 5;
+        uint8_t *stg = staging + e * kStagingPerWarp;
+        float *fac = reinterpret_cast<float *>(factors + e * kFactorsPerWarp);  // alpha[32] | beta[32]
+        const bool scaled = p.out_mode != FLEXIQ_OUT_ACC_I32;
         int buf = 0;
         uint32_t buf_phase = 0;
         for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
             const int m_blk = tile / p.n_tiles, n_blk = tile - m_blk * p.n_tiles;
-            const int n0 = n_blk * BN;
-            // per-output-channel factors of this tile: alpha = (S_x * S_w) / S_y, beta = bias / S_y
-            for (int c = et; c < BN; c += 32 * kNumEpiWarps) {
-                const int n = n0 + c;
-                float a = 0.f, b = 0.f;
-                if (n < p.N) {
-                    const float sxw = __fmul_rn(p.x_scale, p.w_scale[n]);
-                    const float bv = p.bias ? p.bias[n] : 0.f;
-                    if (p.out_mode == FLEXIQ_OUT_REQUANT_I8) {
-                        a = __fdiv_rn(sxw, p.y_scale);
-                        b = __fdiv_rn(bv, p.y_scale);
-                    } else {
-                        a = sxw;
-                        b = bv;
-                    }
-                }
-                alpha_s[buf * BN + c] = a;
-                beta_s[buf * BN + c] = b;
-            }
-            asm volatile("bar.sync 1, %0;" ::"n"(32 * kNumEpiWarps) : "memory");
-            if (!epilogue_vote(wait_bounded(&tmem_full[buf], buf_phase, abort_flag, 4))) break;
+            const int nw = n_blk * BN + half * cols_per_warp;  // first output channel of this warp
+            const long long row0 = (long long)m_blk * BM + quad * 32;
+            const int rows_valid = (int)min(32LL, p.M - row0);  // may be <= 0
+            // this lane's factor of the first chunk, fetched while the accumulator is still being produced
+            float a_next = 0.f, b_next = 0.f;
+            if (scaled && nw + lane < p.N) { a_next = __ldg(p.alpha + nw + lane); b_next = __ldg(p.beta + nw + lane); }
+            const bool ok = wait_bounded(&tmem_full[buf], buf_phase, abort_flag, 4);
+            if (!__all_sync(0xffffffffu, ok)) break;
             ptx::tc_fence_after_sync();
-            const long long m = (long long)m_blk * BM + quad * 32 + lane;
-            const bool row_ok = m < p.M;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN);
-            const float *al = alpha_s + buf * BN, *be = beta_s + buf * BN;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)buf * buf_stride + (uint32_t)(half * cols_per_warp);
+            uint32_t ra[32], rb[32];
+            ptx::tmem_ld_32x32(taddr, ra);
+            bool arrived = false;
 #pragma unroll 1
-            for (int c = 0; c < BN; c += 32) {
-                uint32_t r[32];
-                ptx::tmem_ld_32x32(taddr + c, r);
-                ptx::tmem_ld_wait();
-                const int n = n0 + c;
-                if (row_ok && n < p.N) {
-                    const bool second = n + 16 < p.N;  // N is a multiple of 16
+            for (int ch = 0; ch < n_chunks; ch += 2) {
+#pragma unroll
+                for (int sub = 0; sub < 2; ++sub) {
+                    const int c = ch + sub;
+                    if (c >= n_chunks) break;
+                    uint32_t *r = sub == 0 ? ra : rb;
+                    ptx::tmem_ld_wait();
+                    const bool last = c + 1 == n_chunks;
+                    if (!last) ptx::tmem_ld_32x32(taddr + 32 * (c + 1), sub == 0 ? rb : ra);
+                    const int n = nw + 32 * c;                 // first output channel of this chunk
+                    const bool live = n < p.N && rows_valid > 0;
+                    if (scaled) {
+                        __syncwarp();
+                        fac[lane] = a_next;
+                        fac[32 + lane] = b_next;
+                        __syncwarp();
+                        a_next = b_next = 0.f;
+                        if (!last && n + 32 + lane < p.N) { a_next = __ldg(p.alpha + n + 32 + lane); b_next = __ldg(p.beta + n + 32 + lane); }
+                    }
+                    if (last) {
+                        // every TMEM read of this tile has landed: hand the accumulator back to the MMA warp
+                        ptx::tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(&tmem_empty[buf]);
+                        arrived = true;
+                    }
+                    if (!live) continue;
+                    const float4 *fa = reinterpret_cast<const float4 *>(fac), *fb = reinterpret_cast<const float4 *>(fac + 32);
                     if (p.out_mode == FLEXIQ_OUT_REQUANT_I8) {
                         unsigned w[8];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            w[i] = pack4_sat_i8(fmaf((float)(int)r[4 * i + 0], al[c + 4 * i + 0], be[c + 4 * i + 0]),
-                                                fmaf((float)(int)r[4 * i + 1], al[c + 4 * i + 1], be[c + 4 * i + 1]),
-                                                fmaf((float)(int)r[4 * i + 2], al[c + 4 * i + 2], be[c + 4 * i + 2]),
-                                                fmaf((float)(int)r[4 * i + 3], al[c + 4 * i + 3], be[c + 4 * i + 3]));
-                        uint4 *dst = reinterpret_cast<uint4 *>(static_cast<int8_t *>(p.Y) + m * p.N + n);
-                        dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-                        if (second) dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
-                    } else if (p.out_mode == FLEXIQ_OUT_DEQUANT_F32) {
-                        float4 *dst = reinterpret_cast<float4 *>(static_cast<float *>(p.Y) + m * p.N + n);
-#pragma unroll
                         for (int i = 0; i < 8; ++i) {
-                            if (i >= 4 && !second) break;
-                            dst[i] = make_float4(fmaf((float)(int)r[4 * i + 0], al[c + 4 * i + 0], be[c + 4 * i + 0]),
-                                                 fmaf((float)(int)r[4 * i + 1], al[c + 4 * i + 1], be[c + 4 * i + 1]),
-                                                 fmaf((float)(int)r[4 * i + 2], al[c + 4 * i + 2], be[c + 4 * i + 2]),
-                                                 fmaf((float)(int)r[4 * i + 3], al[c + 4 * i + 3], be[c + 4 * i + 3]));
+                            const float4 a = fa[i], b = fb[i];
+                            w[i] = requant4(fmaf((float)(int)r[4 * i + 0], a.x, b.x), fmaf((float)(int)r[4 * i + 1], a.y, b.y),
+                                            fmaf((float)(int)r[4 * i + 2], a.z, b.z), fmaf((float)(int)r[4 * i + 3], a.w, b.w));
+                        }
+                        const int u0 = 2 * (c & 1);            // 64 staged bytes per row hold two chunks
+                        *staging_unit(stg, lane, u0) = make_uint4(w[0], w[1], w[2], w[3]);
+                        *staging_unit(stg, lane, u0 + 1) = make_uint4(w[4], w[5], w[6], w[7]);
+                        if ((c & 1) || last) {
+                            const int nf = n - 32 * (c & 1);
+                            flush_staging(stg, (c & 1) ? 4 : 2, static_cast<uint8_t *>(p.Y) + row0 * p.N + nf, (long long)p.N,
+                                          rows_valid, (p.N - nf) >> 4, lane);
                         }
                     } else {
-                        uint4 *dst = reinterpret_cast<uint4 *>(static_cast<int32_t *>(p.Y) + m * p.N + n);
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            if (i >= 4 && !second) break;
-                            dst[i] = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+                        for (int h = 0; h < 2; ++h) {          // 16 columns x 4 bytes = 64 staged bytes per row
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                const int q = 4 * h + i;
+                                uint4 v = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
+                                if (p.out_mode == FLEXIQ_OUT_DEQUANT_F32) {
+                                    const float4 a = fa[q], b = fb[q];
+                                    v.x = __float_as_uint(fmaf((float)(int)r[4 * q + 0], a.x, b.x));
+                                    v.y = __float_as_uint(fmaf((float)(int)r[4 * q + 1], a.y, b.y));
+                                    v.z = __float_as_uint(fmaf((float)(int)r[4 * q + 2], a.z, b.z));
+                                    v.w = __float_as_uint(fmaf((float)(int)r[4 * q + 3], a.w, b.w));
+                                }
+                                *staging_unit(stg, lane, i) = v;
+                            }
+                            const int nf = n + 16 * h;
+                            flush_staging(stg, 4, static_cast<uint8_t *>(p.Y) + (row0 * p.N + nf) * 4, (long long)p.N * 4,
+                                          rows_valid, (p.N - nf) >> 2, lane);
                         }
                     }
                 }
             }
-            ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(&tmem_empty[buf]);
+            if (!arrived) {  // not reached: n_chunks >= 1 always marks a last chunk
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&tmem_empty[buf]);
+            }
             if ((buf ^= 1) == 0) buf_phase ^= 1;
         }
     }
@@ -318,24 +372,37 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
     __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc(tmem_base, C::kTmemCols);
+        ptx::tmem_dealloc(tmem_base, tmem_cols);
     }
+}
+
+// Per-output-channel factors of a call: REQUANT alpha = (S_x * S_w[n]) / S_y, beta = bias[n] / S_y;
+// DEQUANT alpha = S_x * S_w[n], beta = bias[n].  Each operation rounds once, in fp32.
+__global__ void scale_vectors_kernel(int N, float x_scale, float y_scale, int requant, const float *__restrict__ w_scale,
+                                     const float *__restrict__ bias, float *__restrict__ alpha, float *__restrict__ beta)
+{
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= N) return;
+    const float sxw = __fmul_rn(x_scale, w_scale[n]);
+    const float bv = bias ? bias[n] : 0.f;
+    alpha[n] = requant ? __fdiv_rn(sxw, y_scale) : sxw;
+    beta[n] = requant ? __fdiv_rn(bv, y_scale) : bv;
 }
 
 // ------------------------------------------------------------------------------------
 // host side
 
-static int bn_index(int bn) { return bn == 64 ? 0 : (bn == 128 ? 1 : 2); }
+static int bn_index(int bn) { return bn / 64 - 1; }
 
 // Tile width: fewest machine-waves weighted by how well a tile of that width feeds the
 // tensor pipe (narrow tiles re-read A from shared memory more often per MMA).
 int choose_bn(long long m_tiles, int N, int sms)
 {
-    const int bns[3] = {256, 128, 64};
-    const double penalty[3] = {1.0, 1.15, 1.6};
+    const int bns[4] = {256, 192, 128, 64};
+    const double penalty[4] = {1.0, 1.05, 1.15, 1.6};
     int best = 256;
     double best_cost = 1e300;
-    for (int i = 0; i < 3; ++i) {
+    for (int i = 0; i < 4; ++i) {
         const long long n_tiles = (N + bns[i] - 1) / bns[i];
         const long long tiles = m_tiles * n_tiles;
         const long long waves = (tiles + sms - 1) / sms;
@@ -366,20 +433,19 @@ static int make_map_im2col(CUtensorMap *map, const void *base, int Cpart, long l
     return FLEXIQ_OK;
 }
 
-template <int BN>
-static int launch_bn(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const CUtensorMap &b_lo, const CUtensorMap &b_hi,
-                     const GemmParams &p, int sms, cudaStream_t st)
+static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const CUtensorMap &b_lo, const CUtensorMap &b_hi,
+                         const GemmParams &p, int sms, cudaStream_t st)
 {
     static bool attr_set[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 64 && !attr_set[dev]) {
-        FLEXIQ_CUDA_TRY(cudaFuncSetAttribute(mixed_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::kSmemBytes));
+        FLEXIQ_CUDA_TRY(cudaFuncSetAttribute(mixed_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
         attr_set[dev] = true;
     }
     const long long tiles = (long long)p.m_tiles * p.n_tiles;
     const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-    mixed_gemm_kernel<BN><<<grid, kThreadsMasked, Cfg<BN>::kSmemBytes, st>>>(a_lo, a_hi, b_lo, b_hi, p);
+    mixed_gemm_kernel<<<grid, kThreads, kSmemBytes, st>>>(a_lo, a_hi, b_lo, b_hi, p);
     FLEXIQ_CUDA_TRY(cudaGetLastError());
     return FLEXIQ_OK;
 }
@@ -418,11 +484,23 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
         p.P = (H + 2 * L->pad - L->R) / L->stride + 1;
         p.Q = (W + 2 * L->pad - L->S) / L->stride + 1;
     }
-    p.out_mode = out_mode; p.x_scale = x_scale; p.y_scale = y_scale;
-    p.w_scale = L->w_scale; p.bias = L->bias; p.Y = Y;
+    p.out_mode = out_mode; p.Y = Y;
+    p.alpha = L->alpha; p.beta = L->beta;
     p.m_tiles = (int)((M + BM - 1) / BM);
     const int bn = choose_bn(p.m_tiles, L->N, sms);
+    p.BN = bn;
     p.n_tiles = (L->N + bn - 1) / bn;
+    p.stages = kStageRegion / (kABytes + bn * 128);
+    if (p.stages > kMaxStages) p.stages = kMaxStages;
+    // the per-output-channel factors depend on the call's scales: recomputed (one tiny launch,
+    // stream-ordered before the GEMM) only when they differ from the previous call's
+    if (out_mode != FLEXIQ_OUT_ACC_I32 &&
+        !(L->cache_mode == out_mode && L->cache_xs == x_scale && (out_mode == FLEXIQ_OUT_DEQUANT_F32 || L->cache_ys == y_scale))) {
+        scale_vectors_kernel<<<(L->N + 255) / 256, 256, 0, st>>>(L->N, x_scale, y_scale, out_mode == FLEXIQ_OUT_REQUANT_I8,
+                                                                 L->w_scale, L->bias, L->alpha, L->beta);
+        FLEXIQ_CUDA_TRY(cudaGetLastError());
+        L->cache_mode = out_mode; L->cache_xs = x_scale; L->cache_ys = y_scale;
+    }
 
     // activation maps (per call: they depend on the caller's buffers, M and the ratio);
     // an empty slab borrows the other one's map and is never addressed
@@ -439,11 +517,7 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     if (C_lo == 0) a_lo = a_hi;
     if (C_hi == 0) a_hi = a_lo;
     const int bi = bn_index(bn);
-    switch (bn) {
-        case 256: return launch_bn<256>(a_lo, a_hi, L->map_w8m[bi], L->map_w8[bi], p, sms, st);
-        case 128: return launch_bn<128>(a_lo, a_hi, L->map_w8m[bi], L->map_w8[bi], p, sms, st);
-        default: return launch_bn<64>(a_lo, a_hi, L->map_w8m[bi], L->map_w8[bi], p, sms, st);
-    }
+    return launch_kernel(a_lo, a_hi, L->map_w8m[bi], L->map_w8[bi], p, sms, st);
 }
 
 }  // namespace flexiq

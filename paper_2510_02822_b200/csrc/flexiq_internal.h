@@ -37,7 +37,11 @@ struct Layer {
     int32_t *perm_host;
     uint8_t *sx_host;
     // tensor maps over the weights (encoded once)
-    CUtensorMap map_w8[3], map_w8m[3], map_w4[3];  // box rows 64 / 128 / 256
+    CUtensorMap map_w8[4], map_w8m[4], map_w4[4];  // box rows 64 / 128 / 192 / 256
+    // per-output-channel epilogue factors of the most recent call and what they were computed for
+    float *alpha, *beta;
+    float cache_xs, cache_ys;
+    int cache_mode;
     int w4_pitch;    // row pitch of w4 in bytes: Kw/2 rounded up to 16
 };
 

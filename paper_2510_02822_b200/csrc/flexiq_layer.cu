@@ -171,7 +171,7 @@ static void free_layer(Layer *L)
 {
     if (!L) return;
     cudaFree(L->w8); cudaFree(L->w8m); cudaFree(L->w4); cudaFree(L->sw); cudaFree(L->sx);
-    cudaFree(L->perm); cudaFree(L->w_scale); cudaFree(L->bias);
+    cudaFree(L->perm); cudaFree(L->w_scale); cudaFree(L->bias); cudaFree(L->alpha); cudaFree(L->beta);
     free(L->perm_host); free(L->sx_host);
     L->magic = 0;
     free(L);
@@ -180,8 +180,8 @@ static void free_layer(Layer *L)
 int encode_weight_maps(Layer *L)
 {
     const int bk = choose_bk(L);
-    const int bns[3] = {64, 128, 256};
-    for (int i = 0; i < 3; ++i) {
+    const int bns[4] = {64, 128, 192, 256};
+    for (int i = 0; i < 4; ++i) {
         int rc = make_map_2d(&L->map_w8[i], L->w8, (uint64_t)L->Kw, (uint64_t)L->N, (uint64_t)L->Kw, bk, bns[i], bk);
         if (rc) return rc;
         rc = make_map_2d(&L->map_w8m[i], L->w8m, (uint64_t)L->Kw, (uint64_t)L->N, (uint64_t)L->Kw, bk, bns[i], bk);
@@ -238,6 +238,9 @@ static int create_common(flexiq_layer_t *out, int is_conv, int C, int N, int R, 
     TRY_OR_FREE(cudaMalloc(&L->perm, sizeof(int32_t) * n_g));
     TRY_OR_FREE(cudaMalloc(&L->w_scale, sizeof(float) * N));
     if (bias) TRY_OR_FREE(cudaMalloc(&L->bias, sizeof(float) * N));
+    TRY_OR_FREE(cudaMalloc(&L->alpha, sizeof(float) * N));
+    TRY_OR_FREE(cudaMalloc(&L->beta, sizeof(float) * N));
+    L->cache_mode = -1;
     TRY_OR_FREE(cudaMemcpyAsync(L->perm, L->perm_host, sizeof(int32_t) * n_g, cudaMemcpyHostToDevice, stream));
     TRY_OR_FREE(cudaMemcpyAsync(L->sx, L->sx_host, n_g, cudaMemcpyHostToDevice, stream));
     TRY_OR_FREE(cudaMemcpyAsync(L->w_scale, w_scale, sizeof(float) * N, cudaMemcpyDeviceToDevice, stream));
