@@ -159,6 +159,11 @@ int flexiq_mixed_conv(flexiq_layer_t layer, const uint8_t *X4_dev, const int8_t 
 int flexiq_layer_export(flexiq_layer_t layer, uint8_t *sw_host, int8_t *w8_host,
                         uint8_t *w4_host);
 
+/* Test hook: forces the mainloop's tile shape for every later mixed_* call of the process
+ * (cta_group 1 or 2 CTAs per tile, tile_n in {64, 128, 192, 256}; cta_group 2 needs
+ * tile_n >= 128).  cta_group 0 restores the automatic choice.  The paper has no counterpart. */
+int flexiq_force_tile(int cta_group, int tile_n);
+
 /* Reads and clears the device status word raised by a bounded wait that expired.
  * Synchronises `stream`. */
 int flexiq_check_status(void *stream);

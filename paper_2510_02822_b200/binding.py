@@ -22,7 +22,7 @@ EXPORTS = [
     "flexiq_layer_create_linear", "flexiq_layer_create_conv", "flexiq_layer_destroy",
     "flexiq_layer_set_lowbit_path", "flexiq_set_lowbit_ratio", "flexiq_get_max_4bit_ch",
     "flexiq_x4_pitch", "flexiq_quantize_lower", "flexiq_mixed_gemm", "flexiq_mixed_conv",
-    "flexiq_layer_export", "flexiq_check_status", "flexiq_last_error",
+    "flexiq_layer_export", "flexiq_force_tile", "flexiq_check_status", "flexiq_last_error",
 ]
 
 _lib = None
@@ -142,6 +142,10 @@ def flexiq_layer_export(h, sw_host=None, w8_host=None, w4_host=None):
     def hp(a):
         return None if a is None else a.ctypes.data_as(C.c_void_p)
     _check(lib().flexiq_layer_export(h, hp(sw_host), hp(w8_host), hp(w4_host)))
+
+
+def flexiq_force_tile(cta_group, tile_n):
+    _check(lib().flexiq_force_tile(cta_group, tile_n))
 
 
 def flexiq_check_status():

@@ -18,16 +18,30 @@ namespace flexiq {
 
 __device__ unsigned int g_status_word = 0;
 
+// Optional role timers (build with -DFLEXIQ_PROFILE): cycles CTA 0 spends waiting per role.
+#ifdef FLEXIQ_PROFILE
+__device__ long long g_prof[16];
+#define PROF_DECL(name) long long name = 0
+#define PROF_T0(t) const long long t = clock64()
+#define PROF_ADD(name, t) name += clock64() - t
+#define PROF_STORE(i, v) do { if (blockIdx.x == 0) g_prof[i] = (v); } while (0)
+#else
+#define PROF_DECL(name)
+#define PROF_T0(t)
+#define PROF_ADD(name, t)
+#define PROF_STORE(i, v)
+#endif
+
 constexpr int BM = 128;
-constexpr int kNumEpiWarps = 8;                       // two per TMEM lane quadrant
+constexpr int kNumEpiWarps = 16;                      // four per TMEM lane quadrant
 constexpr int kThreads = 32 * (2 + kNumEpiWarps);
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kABytes = BM * 128;                     // A stage (BK <= 128 bytes per row)
 constexpr int kStageRegion = 196608;                  // shared memory given to the operand ring
 constexpr int kStagingPerWarp = 2048;                 // 32 rows x 64 B output staging per epilogue warp
-constexpr int kFactorsPerWarp = 256;                  // alpha[32], beta[32] of the current column chunk
+constexpr int kFactorsPerWarp = 128;                  // alpha[16], beta[16] of the current column chunk
 constexpr int kMaxStages = 8;
-constexpr int kSmemBytes = kStageRegion + kNumEpiWarps * (kStagingPerWarp + kFactorsPerWarp) + 256 + 1024;
+constexpr int kSmemBytes = kStageRegion + kNumEpiWarps * (kStagingPerWarp + kFactorsPerWarp) + 256;
 
 struct GemmParams {
     long long M;         // rows of the implicit GEMM (tokens or output pixels)
@@ -106,27 +120,34 @@ __device__ __forceinline__ uint4 *staging_unit(uint8_t *stg, int row, int unit)
     return reinterpret_cast<uint4 *>(stg + row * 64 + ((unit ^ ((row >> 1) & 3)) << 4));
 }
 
-// Coalesced copy of the staged rows to global memory: `upr` (2 or 4) 16-byte units per row.
+// Coalesced copy of the staged rows to global memory: `upr` (1..4) 16-byte units per row.
 __device__ __forceinline__ void flush_staging(uint8_t *stg, int upr, uint8_t *gbase, long long row_pitch_bytes,
                                               int rows_valid, int units_valid, int lane)
 {
     __syncwarp();
-    const int sh = upr == 4 ? 2 : 1;
     for (int u = lane; u < 32 * upr; u += 32) {
-        const int row = u >> sh, j = u & (upr - 1);
+        const int row = u / upr, j = u - row * upr;
         if (row < rows_valid && j < units_valid)
             *reinterpret_cast<uint4 *>(gbase + row * row_pitch_bytes + j * 16) = *staging_unit(stg, row, j);
     }
     __syncwarp();
 }
 
+// CG = 1: one CTA per 128 x BN tile.  CG = 2: a CTA pair (cluster of two) per 256 x BN tile;
+// each CTA loads its own 128 rows of A and its own half of B (no multicast), the leader
+// CTA issues cta_group::2 MMAs that read both halves, and each CTA drains the 128
+// accumulator rows held in its own TMEM.  Operand traffic from L2 per MAC drops by a third.
+template <int CG>
 __global__ void __launch_bounds__(kThreads, 1)
 mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_constant__ CUtensorMap mapA_hi,
                   const __grid_constant__ CUtensorMap mapB_lo, const __grid_constant__ CUtensorMap mapB_hi,
                   const GemmParams p)
 {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) uint8_t smem[];
+    if (ptx::smem_u32(smem) & 1023u) {  // the swizzled operand tiles need 1024-byte alignment
+        if (threadIdx.x == 0) atomicMax(&g_status_word, 0x200u);
+        return;
+    }
     uint8_t *stage_base = smem;
     uint8_t *staging = smem + kStageRegion;
     uint8_t *factors = staging + kNumEpiWarps * kStagingPerWarp;
@@ -139,8 +160,12 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int BN = p.BN;
-    const int stage_bytes = kABytes + BN * 128;
+    const int b_rows = BN / CG;                       // rows of the B tile this CTA loads
+    const int stage_bytes = kABytes + b_rows * 128;
     const int num_tiles = p.m_tiles * p.n_tiles;
+    const uint32_t cta_rank = CG == 2 ? ptx::cluster_ctarank() : 0u;
+    const bool leader = cta_rank == 0;
+    const int first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
     const int kb_total = p.T * (p.nb_lo + p.nb_hi);
     const uint32_t tmem_cols = BN <= 64 ? 128u : (BN <= 128 ? 256u : 512u);
     const uint32_t buf_stride = tmem_cols / 2;  // column offset of the second accumulator
@@ -152,36 +177,42 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(&tmem_full[b], 1);
-            ptx::mbar_init(&tmem_empty[b], kNumEpiWarps);
+            ptx::mbar_init(&tmem_empty[b], CG * kNumEpiWarps);
         }
         *abort_flag = 0;
         ptx::fence_mbar_init();
     }
     if (warp == 1) {
-        ptx::tmem_alloc(tmem_ptr_s, tmem_cols);
-        ptx::tmem_relinquish();
+        if (CG == 2) { ptx::tmem_alloc_pair(tmem_ptr_s, tmem_cols); ptx::tmem_relinquish_pair(); }
+        else { ptx::tmem_alloc(tmem_ptr_s, tmem_cols); ptx::tmem_relinquish(); }
     }
     ptx::tc_fence_before_sync();
-    __syncthreads();
+    if (CG == 2) ptx::cluster_sync_all();  // the peer's barriers are initialised before anyone signals them
+    else __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_ptr_s;
 
     if (warp == 0) {
         // ------------------------------------------------------------- TMA producer
-        if (lane == 0) {
-            ptx::prefetch_tmap(&mapA_lo);
-            ptx::prefetch_tmap(&mapA_hi);
-            ptx::prefetch_tmap(&mapB_lo);
-            ptx::prefetch_tmap(&mapB_hi);
-            const uint32_t tx_bytes = (uint32_t)(BM * p.BK + BN * p.BK);
+        // The whole warp walks the loop; one elected lane issues the copies.
+        {
+            if (ptx::elect_one()) {
+                ptx::prefetch_tmap(&mapA_lo);
+                ptx::prefetch_tmap(&mapA_hi);
+                ptx::prefetch_tmap(&mapB_lo);
+                ptx::prefetch_tmap(&mapB_hi);
+            }
+            const uint32_t tx_bytes = (uint32_t)(CG * (BM * p.BK + b_rows * p.BK));  // both CTAs' loads
             int stage = 0;
             uint32_t phase = 0;
             long long issued = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            PROF_DECL(prof_wait);
+            PROF_T0(prof_start);
+            for (int tile = first_tile; tile < num_tiles && ok; tile += tile_step) {
                 const int m_blk = tile / p.n_tiles, n_blk = tile - m_blk * p.n_tiles;
-                const long long m0 = (long long)m_blk * BM;
-                const int n0 = n_blk * BN;
+                const long long m0 = ((long long)m_blk * CG + cta_rank) * BM;
+                const int n0 = n_blk * BN + (int)cta_rank * b_rows;
                 int pix_w = 0, pix_h = 0, pix_n = 0;
                 if (p.im2col) {
                     const long long pq = (long long)p.P * p.Q;
@@ -193,25 +224,42 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                 KBlockIter it;
                 it.reset(p);
                 for (int kb = 0; kb < kb_total; ++kb, it.next(p)) {
-                    if (!wait_bounded(&empty_bar[stage], phase ^ 1, abort_flag, 1)) { ok = false; break; }
+                    PROF_T0(t0);
+                    if (!__all_sync(0xffffffffu, wait_bounded(&empty_bar[stage], phase ^ 1, abort_flag, 1))) { ok = false; break; }
+                    PROF_ADD(prof_wait, t0);
                     const bool low = it.part == 0;
                     uint8_t *sa = stage_base + stage * stage_bytes;
-                    ptx::mbar_expect_tx(&full_bar[stage], tx_bytes);
+                    if (ptx::elect_one()) {
+                    if (leader) ptx::mbar_expect_tx(&full_bar[stage], tx_bytes);
                     const CUtensorMap *ma = low ? &mapA_lo : &mapA_hi;
-                    if (p.im2col)
-                        ptx::tma_load_im2col_4d(sa, ma, &full_bar[stage], it.cb * p.BK, pix_w, pix_h, pix_n,
-                                                (uint16_t)it.tap_s, (uint16_t)it.tap_r);
-                    else
-                        ptx::tma_load_2d(sa, ma, &full_bar[stage], it.cb * p.BK, (int)m0);
+                    const CUtensorMap *mb = low ? &mapB_lo : &mapB_hi;
                     // weights: slab-order [N][T*C]; the low slab's forms start each tap at channel 0,
                     // the 8-bit form of the high groups at channel C_lo
-                    ptx::tma_load_2d(sa + kABytes, low ? &mapB_lo : &mapB_hi, &full_bar[stage],
-                                     it.tap * p.C + (low ? 0 : p.C_lo) + it.cb * p.BK, n0);
+                    const int xb = it.tap * p.C + (low ? 0 : p.C_lo) + it.cb * p.BK;
+                    if (CG == 2) {
+                        const uint32_t bar = ptx::mapa(ptx::smem_u32(&full_bar[stage]), 0);  // the leader's barrier
+                        if (p.im2col)
+                            ptx::tma_load_im2col_4d_pair(sa, ma, bar, it.cb * p.BK, pix_w, pix_h, pix_n, (uint16_t)it.tap_s, (uint16_t)it.tap_r);
+                        else
+                            ptx::tma_load_2d_pair(sa, ma, bar, it.cb * p.BK, (int)m0);
+                        ptx::tma_load_2d_pair(sa + kABytes, mb, bar, xb, n0);
+                    } else {
+                        if (p.im2col)
+                            ptx::tma_load_im2col_4d(sa, ma, &full_bar[stage], it.cb * p.BK, pix_w, pix_h, pix_n, (uint16_t)it.tap_s, (uint16_t)it.tap_r);
+                        else
+                            ptx::tma_load_2d(sa, ma, &full_bar[stage], it.cb * p.BK, (int)m0);
+                        ptx::tma_load_2d(sa + kABytes, mb, &full_bar[stage], xb, n0);
+                    }
+                    }
+                    __syncwarp();
                     ++issued;
                     if (++stage == p.stages) { stage = 0; phase ^= 1; }
                 }
             }
-            if (!ok) {
+            PROF_STORE(0, prof_wait);
+            PROF_STORE(1, clock64() - prof_start);
+            PROF_STORE(2, issued);
+            if (!ok && lane == 0) {
                 // drain: let the copies already in flight land before the CTA retires
                 const int n_back = issued < p.stages ? (int)issued : p.stages;
                 int s = stage;
@@ -219,16 +267,18 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                 for (int i = 0; i < n_back; ++i) {
                     if (--s < 0) { s = p.stages - 1; ph ^= 1; }
                     for (uint32_t w = 0; w < (1u << 16); ++w) {
-                        if (ptx::mbar_try_wait(&full_bar[s], ph)) break;
+                        if (leader && ptx::mbar_try_wait(&full_bar[s], ph)) break;
                         __nanosleep(64);
+                        if (!leader && w > 64) break;  // its loads credit the leader's barrier: give them a few microseconds
                     }
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc = ptx::idesc_i8(BM, BN);
+        // The whole warp walks the loop; one elected lane issues the MMAs and their commits.
+        if (leader) {
+            const uint32_t idesc = ptx::idesc_i8(BM * CG, BN);
             const uint64_t adesc0 = ptx::smem_desc(ptx::smem_u32(stage_base), p.BK);
             const uint64_t bdesc0 = ptx::smem_desc(ptx::smem_u32(stage_base + kABytes), p.BK);
             const uint64_t stage_step = (uint64_t)(stage_bytes >> 4);
@@ -237,60 +287,85 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             int buf = 0;
             uint32_t buf_phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-                if (!wait_bounded(&tmem_empty[buf], buf_phase ^ 1, abort_flag, 2)) break;
+            PROF_DECL(prof_wait_acc);
+            PROF_DECL(prof_wait_full);
+            PROF_T0(prof_start);
+            for (int tile = first_tile; tile < num_tiles && ok; tile += tile_step) {
+                PROF_T0(t0);
+                if (!__all_sync(0xffffffffu, wait_bounded(&tmem_empty[buf], buf_phase ^ 1, abort_flag, 2))) break;
+                PROF_ADD(prof_wait_acc, t0);
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)buf * buf_stride;
                 KBlockIter it;
                 it.reset(p);
                 uint32_t accumulate = 0;
                 for (int kb = 0; kb < kb_total; ++kb, it.next(p)) {
-                    if (!wait_bounded(&full_bar[stage], phase, abort_flag, 3)) { ok = false; break; }
+                    PROF_T0(t1);
+                    if (!__all_sync(0xffffffffu, wait_bounded(&full_bar[stage], phase, abort_flag, 3))) { ok = false; break; }
+                    PROF_ADD(prof_wait_full, t1);
                     const int nb = it.part == 0 ? p.nb_lo : p.nb_hi;
                     int ksteps = p.BK >> 5;
                     if (it.cb == nb - 1) ksteps = ((it.part == 0 ? p.C_lo : p.C_hi) - it.cb * p.BK + 31) >> 5;
                     const uint64_t adesc = adesc0 + stage_step * stage;
                     const uint64_t bdesc = bdesc0 + stage_step * stage;
-                    for (int k = 0; k < ksteps; ++k) {  // 32 bytes of K per instruction: +2 in 16-byte units
-                        ptx::mma_i8(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, accumulate);
-                        accumulate = 1;
+                    if (ptx::elect_one()) {
+                        uint32_t acc = accumulate;
+                        for (int k = 0; k < ksteps; ++k) {  // 32 bytes of K per instruction: +2 in 16-byte units
+                            if (CG == 2) ptx::mma_i8_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, acc);
+                            else ptx::mma_i8(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, acc);
+                            acc = 1;
+                        }
+                        if (CG == 2) ptx::mma_commit_pair(&empty_bar[stage], 3);  // frees the stage in both CTAs
+                        else ptx::mma_commit(&empty_bar[stage]);
                     }
-                    ptx::mma_commit(&empty_bar[stage]);
+                    __syncwarp();
+                    accumulate = 1;
                     if (++stage == p.stages) { stage = 0; phase ^= 1; }
                 }
-                if (ok) ptx::mma_commit(&tmem_full[buf]);
+                if (ok && ptx::elect_one()) {
+                    if (CG == 2) ptx::mma_commit_pair(&tmem_full[buf], 3);
+                    else ptx::mma_commit(&tmem_full[buf]);
+                }
+                __syncwarp();
                 if ((buf ^= 1) == 0) buf_phase ^= 1;
             }
+            PROF_STORE(4, prof_wait_acc);
+            PROF_STORE(5, prof_wait_full);
+            PROF_STORE(6, clock64() - prof_start);
         }
     } else {
         // ------------------------------------------------------------- epilogue
-        // warp e owns TMEM lane quadrant (warp & 3) and one half of the tile's columns;
-        // the warps do not synchronise with one another.
+        // warp e owns TMEM lane quadrant (warp & 3) and one quarter of the tile's columns,
+        // processed 16 columns at a time; the warps do not synchronise with one another.
         const int e = warp - 2;
         const int quad = warp & 3;
-        const int half = e >> 2;
-        const int cols_per_warp = BN >> 1;           // 32, 64, 96 or 128
-        const int n_chunks = cols_per_warp >> 5;
+        const int part = e >> 2;
+        const int cols_per_warp = BN >> 2;           // 16, 32, 48 or 64
+        const int n_chunks = cols_per_warp >> 4;
         uint8_t *stg = staging + e * kStagingPerWarp;
-        float *fac = reinterpret_cast<float *>(factors + e * kFactorsPerWarp);  // alpha[32] | beta[32]
+        float *fac = reinterpret_cast<float *>(factors + e * kFactorsPerWarp);  // alpha[16] | beta[16]
         const bool scaled = p.out_mode != FLEXIQ_OUT_ACC_I32;
+        const float *fsrc = lane < 16 ? p.alpha : p.beta;                       // lanes 0-15 fetch alpha, 16-31 beta
         int buf = 0;
         uint32_t buf_phase = 0;
-        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
+        PROF_DECL(prof_wait);
+        PROF_T0(prof_start);
+        for (int tile = first_tile; tile < num_tiles; tile += tile_step) {
             const int m_blk = tile / p.n_tiles, n_blk = tile - m_blk * p.n_tiles;
-            const int nw = n_blk * BN + half * cols_per_warp;  // first output channel of this warp
-            const long long row0 = (long long)m_blk * BM + quad * 32;
+            const int nw = n_blk * BN + part * cols_per_warp;  // first output channel of this warp
+            const long long row0 = ((long long)m_blk * CG + cta_rank) * BM + quad * 32;
             const int rows_valid = (int)min(32LL, p.M - row0);  // may be <= 0
             // this lane's factor of the first chunk, fetched while the accumulator is still being produced
-            float a_next = 0.f, b_next = 0.f;
-            if (scaled && nw + lane < p.N) { a_next = __ldg(p.alpha + nw + lane); b_next = __ldg(p.beta + nw + lane); }
+            float f_next = 0.f;
+            if (scaled && nw + (lane & 15) < p.N) f_next = __ldg(fsrc + nw + (lane & 15));
+            PROF_T0(t0);
             const bool ok = wait_bounded(&tmem_full[buf], buf_phase, abort_flag, 4);
+            PROF_ADD(prof_wait, t0);
             if (!__all_sync(0xffffffffu, ok)) break;
             ptx::tc_fence_after_sync();
-            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)buf * buf_stride + (uint32_t)(half * cols_per_warp);
-            uint32_t ra[32], rb[32];
-            ptx::tmem_ld_32x32(taddr, ra);
-            bool arrived = false;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)buf * buf_stride + (uint32_t)(part * cols_per_warp);
+            uint32_t ra[16], rb[16];
+            ptx::tmem_ld_32x16(taddr, ra);
 #pragma unroll 1
             for (int ch = 0; ch < n_chunks; ch += 2) {
 #pragma unroll
@@ -300,79 +375,69 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                     uint32_t *r = sub == 0 ? ra : rb;
                     ptx::tmem_ld_wait();
                     const bool last = c + 1 == n_chunks;
-                    if (!last) ptx::tmem_ld_32x32(taddr + 32 * (c + 1), sub == 0 ? rb : ra);
-                    const int n = nw + 32 * c;                 // first output channel of this chunk
+                    if (!last) ptx::tmem_ld_32x16(taddr + 16 * (c + 1), sub == 0 ? rb : ra);
+                    const int n = nw + 16 * c;                 // first output channel of this chunk
                     const bool live = n < p.N && rows_valid > 0;
                     if (scaled) {
                         __syncwarp();
-                        fac[lane] = a_next;
-                        fac[32 + lane] = b_next;
+                        fac[lane] = f_next;
                         __syncwarp();
-                        a_next = b_next = 0.f;
-                        if (!last && n + 32 + lane < p.N) { a_next = __ldg(p.alpha + n + 32 + lane); b_next = __ldg(p.beta + n + 32 + lane); }
+                        f_next = 0.f;
+                        if (!last && n + 16 + (lane & 15) < p.N) f_next = __ldg(fsrc + n + 16 + (lane & 15));
                     }
                     if (last) {
                         // every TMEM read of this tile has landed: hand the accumulator back to the MMA warp
                         ptx::tc_fence_before_sync();
                         __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(&tmem_empty[buf]);
-                        arrived = true;
+                        if (lane == 0) {
+                            if (CG == 2) ptx::mbar_arrive_cluster(ptx::mapa(ptx::smem_u32(&tmem_empty[buf]), 0));
+                            else ptx::mbar_arrive(&tmem_empty[buf]);
+                        }
                     }
                     if (!live) continue;
-                    const float4 *fa = reinterpret_cast<const float4 *>(fac), *fb = reinterpret_cast<const float4 *>(fac + 32);
+                    const float4 *fa = reinterpret_cast<const float4 *>(fac), *fb = reinterpret_cast<const float4 *>(fac + 16);
                     if (p.out_mode == FLEXIQ_OUT_REQUANT_I8) {
-                        unsigned w[8];
+                        unsigned w[4];
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) {
+                        for (int i = 0; i < 4; ++i) {
                             const float4 a = fa[i], b = fb[i];
                             w[i] = requant4(fmaf((float)(int)r[4 * i + 0], a.x, b.x), fmaf((float)(int)r[4 * i + 1], a.y, b.y),
                                             fmaf((float)(int)r[4 * i + 2], a.z, b.z), fmaf((float)(int)r[4 * i + 3], a.w, b.w));
                         }
-                        const int u0 = 2 * (c & 1);            // 64 staged bytes per row hold two chunks
-                        *staging_unit(stg, lane, u0) = make_uint4(w[0], w[1], w[2], w[3]);
-                        *staging_unit(stg, lane, u0 + 1) = make_uint4(w[4], w[5], w[6], w[7]);
-                        if ((c & 1) || last) {
-                            const int nf = n - 32 * (c & 1);
-                            flush_staging(stg, (c & 1) ? 4 : 2, static_cast<uint8_t *>(p.Y) + row0 * p.N + nf, (long long)p.N,
-                                          rows_valid, (p.N - nf) >> 4, lane);
-                        }
+                        *staging_unit(stg, lane, c) = make_uint4(w[0], w[1], w[2], w[3]);  // 16 output bytes of this row
+                        if (last || n + 16 >= p.N)                                        // no live chunk follows
+                            flush_staging(stg, c + 1, static_cast<uint8_t *>(p.Y) + row0 * p.N + nw, (long long)p.N,
+                                          rows_valid, (p.N - nw) >> 4, lane);
                     } else {
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {          // 16 columns x 4 bytes = 64 staged bytes per row
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-                                const int q = 4 * h + i;
-                                uint4 v = make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
-                                if (p.out_mode == FLEXIQ_OUT_DEQUANT_F32) {
-                                    const float4 a = fa[q], b = fb[q];
-                                    v.x = __float_as_uint(fmaf((float)(int)r[4 * q + 0], a.x, b.x));
-                                    v.y = __float_as_uint(fmaf((float)(int)r[4 * q + 1], a.y, b.y));
-                                    v.z = __float_as_uint(fmaf((float)(int)r[4 * q + 2], a.z, b.z));
-                                    v.w = __float_as_uint(fmaf((float)(int)r[4 * q + 3], a.w, b.w));
-                                }
-                                *staging_unit(stg, lane, i) = v;
+                        for (int i = 0; i < 4; ++i) {              // 16 columns x 4 bytes = 64 staged bytes per row
+                            uint4 v = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+                            if (p.out_mode == FLEXIQ_OUT_DEQUANT_F32) {
+                                const float4 a = fa[i], b = fb[i];
+                                v.x = __float_as_uint(fmaf((float)(int)r[4 * i + 0], a.x, b.x));
+                                v.y = __float_as_uint(fmaf((float)(int)r[4 * i + 1], a.y, b.y));
+                                v.z = __float_as_uint(fmaf((float)(int)r[4 * i + 2], a.z, b.z));
+                                v.w = __float_as_uint(fmaf((float)(int)r[4 * i + 3], a.w, b.w));
                             }
-                            const int nf = n + 16 * h;
-                            flush_staging(stg, 4, static_cast<uint8_t *>(p.Y) + (row0 * p.N + nf) * 4, (long long)p.N * 4,
-                                          rows_valid, (p.N - nf) >> 2, lane);
+                            *staging_unit(stg, lane, i) = v;
                         }
+                        flush_staging(stg, 4, static_cast<uint8_t *>(p.Y) + (row0 * p.N + n) * 4, (long long)p.N * 4,
+                                      rows_valid, (p.N - n) >> 2, lane);
                     }
                 }
             }
-            if (!arrived) {  // not reached: n_chunks >= 1 always marks a last chunk
-                ptx::tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&tmem_empty[buf]);
-            }
             if ((buf ^= 1) == 0) buf_phase ^= 1;
         }
+        if (e == 0 && lane == 0) { PROF_STORE(8, prof_wait); PROF_STORE(9, clock64() - prof_start); }
     }
 
     ptx::tc_fence_before_sync();
-    __syncthreads();
+    if (CG == 2) ptx::cluster_sync_all();  // neither CTA frees TMEM or retires while its peer still works
+    else __syncthreads();
     if (warp == 1) {
         ptx::tc_fence_after_sync();
-        ptx::tmem_dealloc(tmem_base, tmem_cols);
+        if (CG == 2) ptx::tmem_dealloc_pair(tmem_base, tmem_cols);
+        else ptx::tmem_dealloc(tmem_base, tmem_cols);
     }
 }
 
@@ -392,23 +457,28 @@ __global__ void scale_vectors_kernel(int N, float x_scale, float y_scale, int re
 // ------------------------------------------------------------------------------------
 // host side
 
-static int bn_index(int bn) { return bn / 64 - 1; }
-
-// Tile width: fewest machine-waves weighted by how well a tile of that width feeds the
-// tensor pipe (narrow tiles re-read A from shared memory more often per MMA).
-int choose_bn(long long m_tiles, int N, int sms)
+// Tile shape.  Operand traffic from L2 bounds the mainloop on this part, so the cost of a
+// tile is the larger of its operand bytes per SM and its MMA time (both per byte of K),
+// times the number of machine waves; cg = 2 pairs two CTAs on a 256-row tile.
+struct TileChoice { int cg, bn; };
+static TileChoice g_forced_tile{0, 0};  // test hook: 0 = choose automatically
+static TileChoice choose_tile(long long M, int N, int sms)
 {
     const int bns[4] = {256, 192, 128, 64};
-    const double penalty[4] = {1.0, 1.05, 1.15, 1.6};
-    int best = 256;
+    TileChoice best{1, 256};
     double best_cost = 1e300;
-    for (int i = 0; i < 4; ++i) {
-        const long long n_tiles = (N + bns[i] - 1) / bns[i];
-        const long long tiles = m_tiles * n_tiles;
-        const long long waves = (tiles + sms - 1) / sms;
-        const double cost = (double)waves * bns[i] * penalty[i];
-        if (cost < best_cost - 1e-9) { best_cost = cost; best = bns[i]; }
-    }
+    for (int cg = 1; cg <= 2; ++cg)
+        for (int i = 0; i < 4; ++i) {
+            const int bn = bns[i];
+            if (cg == 2 && bn < 128) continue;
+            const long long m_tiles = (M + (long long)BM * cg - 1) / ((long long)BM * cg);
+            const long long n_tiles = (N + bn - 1) / bn;
+            const long long slots = sms / cg;
+            const long long waves = (m_tiles * n_tiles + slots - 1) / slots;
+            const double l2 = (128.0 + (double)bn / cg) / 36.0, mma = bn / 64.0;
+            const double cost = (double)waves * (l2 > mma ? l2 : mma);
+            if (cost < best_cost - 1e-9) { best_cost = cost; best = TileChoice{cg, bn}; }
+        }
     return best;
 }
 
@@ -433,6 +503,7 @@ static int make_map_im2col(CUtensorMap *map, const void *base, int Cpart, long l
     return FLEXIQ_OK;
 }
 
+template <int CG>
 static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const CUtensorMap &b_lo, const CUtensorMap &b_hi,
                          const GemmParams &p, int sms, cudaStream_t st)
 {
@@ -440,13 +511,25 @@ static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 64 && !attr_set[dev]) {
-        FLEXIQ_CUDA_TRY(cudaFuncSetAttribute(mixed_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        FLEXIQ_CUDA_TRY(cudaFuncSetAttribute(mixed_gemm_kernel<CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
         attr_set[dev] = true;
     }
     const long long tiles = (long long)p.m_tiles * p.n_tiles;
-    const unsigned grid = (unsigned)(tiles < sms ? tiles : sms);
-    mixed_gemm_kernel<<<grid, kThreads, kSmemBytes, st>>>(a_lo, a_hi, b_lo, b_hi, p);
-    FLEXIQ_CUDA_TRY(cudaGetLastError());
+    const long long slots = sms / CG;
+    const unsigned grid = (unsigned)((tiles < slots ? tiles : slots) * CG);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CG;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    FLEXIQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, mixed_gemm_kernel<CG>, a_lo, a_hi, b_lo, b_hi, p));
     return FLEXIQ_OK;
 }
 
@@ -486,11 +569,12 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     }
     p.out_mode = out_mode; p.Y = Y;
     p.alpha = L->alpha; p.beta = L->beta;
-    p.m_tiles = (int)((M + BM - 1) / BM);
-    const int bn = choose_bn(p.m_tiles, L->N, sms);
+    const TileChoice tc = g_forced_tile.cg ? g_forced_tile : choose_tile(M, L->N, sms);
+    const int bn = tc.bn, cg = tc.cg;
+    p.m_tiles = (int)((M + (long long)BM * cg - 1) / ((long long)BM * cg));
     p.BN = bn;
     p.n_tiles = (L->N + bn - 1) / bn;
-    p.stages = kStageRegion / (kABytes + bn * 128);
+    p.stages = kStageRegion / (kABytes + (bn / cg) * 128);
     if (p.stages > kMaxStages) p.stages = kMaxStages;
     // the per-output-channel factors depend on the call's scales: recomputed (one tiny launch,
     // stream-ordered before the GEMM) only when they differ from the previous call's
@@ -516,8 +600,9 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     }
     if (C_lo == 0) a_lo = a_hi;
     if (C_hi == 0) a_hi = a_lo;
-    const int bi = bn_index(bn);
-    return launch_kernel(a_lo, a_hi, L->map_w8m[bi], L->map_w8[bi], p, sms, st);
+    const int bi = weight_map_index(bn / cg);  // box rows = the B rows one CTA loads
+    if (cg == 2) return launch_kernel<2>(a_lo, a_hi, L->map_w8m[bi], L->map_w8[bi], p, sms, st);
+    return launch_kernel<1>(a_lo, a_hi, L->map_w8m[bi], L->map_w8[bi], p, sms, st);
 }
 
 }  // namespace flexiq
@@ -549,6 +634,25 @@ extern "C" int flexiq_mixed_conv(flexiq_layer_t layer, const uint8_t *X4_dev, co
     if (P <= 0 || Q <= 0) return set_error(FLEXIQ_ERR_INVALID_ARG, "filter does not fit the padded input");
     return run_mixed(L, X4_dev, X8_dev, x_shift_dev, (long long)Nb * P * Q, Nb, H, W, x_scale, y_scale, out_mode, Y_dev,
                      reinterpret_cast<cudaStream_t>(stream));
+}
+
+#ifdef FLEXIQ_PROFILE
+extern "C" int flexiq_profile_counters(long long *out16)
+{
+    FLEXIQ_CUDA_TRY(cudaDeviceSynchronize());
+    FLEXIQ_CUDA_TRY(cudaMemcpyFromSymbol(out16, g_prof, sizeof(long long) * 16));
+    return FLEXIQ_OK;
+}
+#endif
+
+extern "C" int flexiq_force_tile(int cta_group, int tile_n)
+{
+    if (cta_group == 0) { g_forced_tile = TileChoice{0, 0}; return FLEXIQ_OK; }
+    if ((cta_group != 1 && cta_group != 2) || (tile_n != 64 && tile_n != 128 && tile_n != 192 && tile_n != 256) ||
+        (cta_group == 2 && tile_n < 128))
+        return set_error(FLEXIQ_ERR_INVALID_ARG, "unsupported tile: cta_group %d, tile_n %d", cta_group, tile_n);
+    g_forced_tile = TileChoice{cta_group, tile_n};
+    return FLEXIQ_OK;
 }
 
 extern "C" int flexiq_check_status(void *stream)

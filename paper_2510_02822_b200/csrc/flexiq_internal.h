@@ -9,6 +9,16 @@
 
 namespace flexiq {
 
+// Box heights (rows of the B tile one CTA loads) the weight tensor maps are encoded for.
+constexpr int kNumWeightMaps = 6;
+constexpr int kWeightMapRows[kNumWeightMaps] = {32, 64, 96, 128, 192, 256};
+inline int weight_map_index(int rows)
+{
+    for (int i = 0; i < kNumWeightMaps; ++i)
+        if (kWeightMapRows[i] == rows) return i;
+    return -1;
+}
+
 // Layer handle: everything the static part of the method produces (layout
 // post-processing, weight extraction positions, cached 4-bit weights) plus the one
 // run-time knob, max_4bit_ch.
@@ -37,7 +47,7 @@ struct Layer {
     int32_t *perm_host;
     uint8_t *sx_host;
     // tensor maps over the weights (encoded once)
-    CUtensorMap map_w8[4], map_w8m[4], map_w4[4];  // box rows 64 / 128 / 192 / 256
+    CUtensorMap map_w8[kNumWeightMaps], map_w8m[kNumWeightMaps], map_w4[kNumWeightMaps];  // one per box height
     // per-output-channel epilogue factors of the most recent call and what they were computed for
     float *alpha, *beta;
     float cache_xs, cache_ys;
@@ -68,7 +78,6 @@ EncodeIm2colFn get_encode_im2col();
 int make_map_2d(CUtensorMap *map, const void *base, uint64_t row_bytes, uint64_t rows,
                 uint64_t pitch_bytes, uint32_t box_bytes, uint32_t box_rows, int swizzle_bytes);
 
-int choose_bn(long long m_tiles, int N, int sms);
 int choose_bk(const Layer *L);
 int encode_weight_maps(Layer *L);
 

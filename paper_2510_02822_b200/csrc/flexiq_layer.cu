@@ -180,8 +180,8 @@ static void free_layer(Layer *L)
 int encode_weight_maps(Layer *L)
 {
     const int bk = choose_bk(L);
-    const int bns[4] = {64, 128, 192, 256};
-    for (int i = 0; i < 4; ++i) {
+    const int *bns = kWeightMapRows;
+    for (int i = 0; i < kNumWeightMaps; ++i) {
         int rc = make_map_2d(&L->map_w8[i], L->w8, (uint64_t)L->Kw, (uint64_t)L->N, (uint64_t)L->Kw, bk, bns[i], bk);
         if (rc) return rc;
         rc = make_map_2d(&L->map_w8m[i], L->w8m, (uint64_t)L->Kw, (uint64_t)L->N, (uint64_t)L->Kw, bk, bns[i], bk);

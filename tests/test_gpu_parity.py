@@ -165,6 +165,19 @@ def test_ratio_switch_is_host_only_and_nested(dev):
     L.close()
 
 
+@pytest.mark.parametrize("cg,bn", [(1, 64), (1, 128), (1, 192), (1, 256), (2, 128), (2, 192), (2, 256)])
+def test_every_tile_shape(dev, cg, bn):
+    fx.flexiq_force_tile(cg, bn)
+    try:
+        rng = np.random.default_rng(cg * 1000 + bn)
+        case = inputs.ranged_linear("tile", 700, 384, 400, 16, seed=cg * 10 + bn, group_structured=True)
+        _run_linear(case, dev, [0.0, 0.5, 1.0], shifts=rng.integers(0, 5, 24).astype(np.uint8))
+        conv = inputs.resnet_conv("tilec", 3, 14, 128, 272, 3, seed=bn)
+        _run_conv(conv, dev, [0.5])
+    finally:
+        fx.flexiq_force_tile(0, 0)
+
+
 # ---------------------------------------------------------------- convolution
 def _run_conv(case, dev, ratios, shifts=None):
     perm, sxg, sxs, sw = helpers.prepare_conv(case, shifts)
