@@ -63,12 +63,12 @@ struct GemmParams {
 };
 
 // Bounded wait.  Returns false after the limit or when another role already gave up;
-// the caller then leaves its loops and the CTA drains.
-__device__ __forceinline__ bool wait_bounded(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int where)
+// the caller then leaves its loops and the CTA drains.  The slow path stays out of line
+// so that the hot loops remain small.
+__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int where)
 {
-    if (ptx::mbar_try_wait(bar, parity)) return true;
     for (uint32_t it = 0; it < kSpinLimit; ++it) {
-        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if (ptx::mbar_try_wait_s(bar, parity)) return true;
         if (it > 256) {
             if (*abort_flag) return false;
             __nanosleep(it > 8192 ? 256 : 20);
@@ -78,24 +78,35 @@ __device__ __forceinline__ bool wait_bounded(uint64_t *bar, uint32_t parity, vol
     atomicMax(&g_status_word, 0x100u + (unsigned)where);
     return false;
 }
+__device__ __forceinline__ bool wait_bounded(uint32_t bar, uint32_t parity, volatile int *abort_flag, int where)
+{
+    if (ptx::mbar_try_wait_s(bar, parity)) return true;
+    return wait_slow(bar, parity, abort_flag, where);
+}
+__device__ __forceinline__ bool wait_bounded(uint64_t *bar, uint32_t parity, volatile int *abort_flag, int where)
+{
+    return wait_bounded(ptx::smem_u32(bar), parity, abort_flag, where);
+}
 
-// Walks the K blocks of one output tile in the order both the producer and the MMA
-// issuer use: the low slab (all taps, all channel blocks), then the high slab.
-struct KBlockIter {
-    int part, tap, cb, tap_r, tap_s;
-    __device__ __forceinline__ void reset(const GemmParams &p)
+// Static round-robin walk over the output tiles of one CTA (or CTA pair) without divisions
+// in the loop: tile = first + i * step, decoded as (m_blk, n_blk).
+struct TileWalk {
+    int m_blk, n_blk, step_m, step_n, n_tiles, left;
+    __device__ __forceinline__ void init(int first, int step, int num_tiles, int n_tiles_)
     {
-        part = p.nb_lo > 0 ? 0 : 1;
-        tap = cb = tap_r = tap_s = 0;
+        n_tiles = n_tiles_;
+        m_blk = first / n_tiles;
+        n_blk = first - m_blk * n_tiles;
+        step_m = step / n_tiles;
+        step_n = step - step_m * n_tiles;
+        left = first < num_tiles ? (num_tiles - first + step - 1) / step : 0;
     }
-    __device__ __forceinline__ void next(const GemmParams &p)
+    __device__ __forceinline__ void next()
     {
-        const int nb = part == 0 ? p.nb_lo : p.nb_hi;
-        if (++cb == nb) {
-            cb = 0;
-            if (++tap_s == p.S) { tap_s = 0; ++tap_r; }
-            if (++tap == p.T) { tap = tap_r = tap_s = 0; ++part; }
-        }
+        --left;
+        m_blk += step_m;
+        n_blk += step_n;
+        if (n_blk >= n_tiles) { n_blk -= n_tiles; ++m_blk; }
     }
 };
 
@@ -166,7 +177,6 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
     const uint32_t cta_rank = CG == 2 ? ptx::cluster_ctarank() : 0u;
     const bool leader = cta_rank == 0;
     const int first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
-    const int kb_total = p.T * (p.nb_lo + p.nb_hi);
     const uint32_t tmem_cols = BN <= 64 ? 128u : (BN <= 128 ? 256u : 512u);
     const uint32_t buf_stride = tmem_cols / 2;  // column offset of the second accumulator
 
@@ -194,138 +204,151 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
 
     if (warp == 0) {
         // ------------------------------------------------------------- TMA producer
-        // The whole warp walks the loop; one elected lane issues the copies.
-        {
-            if (ptx::elect_one()) {
-                ptx::prefetch_tmap(&mapA_lo);
-                ptx::prefetch_tmap(&mapA_hi);
-                ptx::prefetch_tmap(&mapB_lo);
-                ptx::prefetch_tmap(&mapB_hi);
+        // The whole warp walks the loops; one elected lane issues the copies.  K blocks run
+        // low slab first (every tap, every channel block), then the high slab.
+        if (ptx::elect_one()) {
+            ptx::prefetch_tmap(&mapA_lo);
+            ptx::prefetch_tmap(&mapA_hi);
+            ptx::prefetch_tmap(&mapB_lo);
+            ptx::prefetch_tmap(&mapB_hi);
+        }
+        const uint32_t tx_bytes = (uint32_t)(CG * (BM * p.BK + b_rows * p.BK));  // both CTAs' loads
+        const uint32_t stage0 = ptx::smem_u32(stage_base);
+        const uint32_t empty0 = ptx::smem_u32(empty_bar);
+        const uint32_t full0 = ptx::smem_u32(full_bar);
+        const uint32_t full0_lead = CG == 2 ? ptx::mapa(full0, 0) : full0;  // transaction bytes go to the leader's barrier
+        uint32_t stage = 0, phase = 0;
+        long long issued = 0;
+        bool ok = true;
+        PROF_DECL(prof_wait);
+        PROF_T0(prof_start);
+        TileWalk tw;
+        for (tw.init(first_tile, tile_step, num_tiles, p.n_tiles); tw.left > 0 && ok; tw.next()) {
+            const long long m0 = ((long long)tw.m_blk * CG + cta_rank) * BM;
+            const int n0 = tw.n_blk * BN + (int)cta_rank * b_rows;
+            int pix_w = 0, pix_h = 0, pix_n = 0;
+            if (p.im2col) {
+                const long long pq = (long long)p.P * p.Q;
+                pix_n = (int)(m0 / pq);
+                const int rem = (int)(m0 - (long long)pix_n * pq);
+                pix_h = (rem / p.Q) * p.stride - p.pad;
+                pix_w = (rem % p.Q) * p.stride - p.pad;
             }
-            const uint32_t tx_bytes = (uint32_t)(CG * (BM * p.BK + b_rows * p.BK));  // both CTAs' loads
-            int stage = 0;
-            uint32_t phase = 0;
-            long long issued = 0;
-            bool ok = true;
-            PROF_DECL(prof_wait);
-            PROF_T0(prof_start);
-            for (int tile = first_tile; tile < num_tiles && ok; tile += tile_step) {
-                const int m_blk = tile / p.n_tiles, n_blk = tile - m_blk * p.n_tiles;
-                const long long m0 = ((long long)m_blk * CG + cta_rank) * BM;
-                const int n0 = n_blk * BN + (int)cta_rank * b_rows;
-                int pix_w = 0, pix_h = 0, pix_n = 0;
-                if (p.im2col) {
-                    const long long pq = (long long)p.P * p.Q;
-                    pix_n = (int)(m0 / pq);
-                    const int rem = (int)(m0 - (long long)pix_n * pq);
-                    pix_h = (rem / p.Q) * p.stride - p.pad;
-                    pix_w = (rem % p.Q) * p.stride - p.pad;
-                }
-                KBlockIter it;
-                it.reset(p);
-                for (int kb = 0; kb < kb_total; ++kb, it.next(p)) {
-                    PROF_T0(t0);
-                    if (!__all_sync(0xffffffffu, wait_bounded(&empty_bar[stage], phase ^ 1, abort_flag, 1))) { ok = false; break; }
-                    PROF_ADD(prof_wait, t0);
-                    const bool low = it.part == 0;
-                    uint8_t *sa = stage_base + stage * stage_bytes;
-                    if (ptx::elect_one()) {
-                    if (leader) ptx::mbar_expect_tx(&full_bar[stage], tx_bytes);
-                    const CUtensorMap *ma = low ? &mapA_lo : &mapA_hi;
-                    const CUtensorMap *mb = low ? &mapB_lo : &mapB_hi;
-                    // weights: slab-order [N][T*C]; the low slab's forms start each tap at channel 0,
-                    // the 8-bit form of the high groups at channel C_lo
-                    const int xb = it.tap * p.C + (low ? 0 : p.C_lo) + it.cb * p.BK;
-                    if (CG == 2) {
-                        const uint32_t bar = ptx::mapa(ptx::smem_u32(&full_bar[stage]), 0);  // the leader's barrier
-                        if (p.im2col)
-                            ptx::tma_load_im2col_4d_pair(sa, ma, bar, it.cb * p.BK, pix_w, pix_h, pix_n, (uint16_t)it.tap_s, (uint16_t)it.tap_r);
-                        else
-                            ptx::tma_load_2d_pair(sa, ma, bar, it.cb * p.BK, (int)m0);
-                        ptx::tma_load_2d_pair(sa + kABytes, mb, bar, xb, n0);
-                    } else {
-                        if (p.im2col)
-                            ptx::tma_load_im2col_4d(sa, ma, &full_bar[stage], it.cb * p.BK, pix_w, pix_h, pix_n, (uint16_t)it.tap_s, (uint16_t)it.tap_r);
-                        else
-                            ptx::tma_load_2d(sa, ma, &full_bar[stage], it.cb * p.BK, (int)m0);
-                        ptx::tma_load_2d(sa + kABytes, mb, &full_bar[stage], xb, n0);
+            for (int part = 0; part < 2 && ok; ++part) {
+                const int nb = part ? p.nb_hi : p.nb_lo;
+                if (nb == 0) continue;
+                const CUtensorMap *ma = part ? &mapA_hi : &mapA_lo;
+                const CUtensorMap *mb = part ? &mapB_hi : &mapB_lo;
+                // weights: slab-order [N][T*C]; the low forms start each tap at channel 0, the
+                // 8-bit form of the high groups at channel C_lo
+                int xb_tap = part ? p.C_lo : 0;
+                int tap_r = 0, tap_s = 0;
+                for (int tap = 0; tap < p.T && ok; ++tap) {
+                    int xa = 0, xb = xb_tap;
+                    for (int cb = 0; cb < nb; ++cb) {
+                        PROF_T0(t0);
+                        if (!__all_sync(0xffffffffu, wait_bounded(empty0 + 8 * stage, phase ^ 1, abort_flag, 1))) { ok = false; break; }
+                        PROF_ADD(prof_wait, t0);
+                        if (ptx::elect_one()) {
+                            const uint32_t sa = stage0 + stage * stage_bytes;
+                            if (leader) ptx::mbar_expect_tx_s(full0 + 8 * stage, tx_bytes);
+                            const uint32_t bar = full0_lead + 8 * stage;
+                            if (p.im2col)
+                                ptx::tma_load_im2col_4d_s<CG>(sa, ma, bar, xa, pix_w, pix_h, pix_n, (uint16_t)tap_s, (uint16_t)tap_r);
+                            else
+                                ptx::tma_load_2d_s<CG>(sa, ma, bar, xa, (int)m0);
+                            ptx::tma_load_2d_s<CG>(sa + kABytes, mb, bar, xb, n0);
+                        }
+                        __syncwarp();
+                        xa += p.BK;
+                        xb += p.BK;
+                        ++issued;
+                        if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
                     }
-                    }
-                    __syncwarp();
-                    ++issued;
-                    if (++stage == p.stages) { stage = 0; phase ^= 1; }
+                    xb_tap += p.C;
+                    if (++tap_s == p.S) { tap_s = 0; ++tap_r; }
                 }
             }
-            PROF_STORE(0, prof_wait);
-            PROF_STORE(1, clock64() - prof_start);
-            PROF_STORE(2, issued);
-            if (!ok && lane == 0) {
-                // drain: let the copies already in flight land before the CTA retires
-                const int n_back = issued < p.stages ? (int)issued : p.stages;
-                int s = stage;
-                uint32_t ph = phase;
-                for (int i = 0; i < n_back; ++i) {
-                    if (--s < 0) { s = p.stages - 1; ph ^= 1; }
-                    for (uint32_t w = 0; w < (1u << 16); ++w) {
-                        if (leader && ptx::mbar_try_wait(&full_bar[s], ph)) break;
-                        __nanosleep(64);
-                        if (!leader && w > 64) break;  // its loads credit the leader's barrier: give them a few microseconds
-                    }
+        }
+        PROF_STORE(0, prof_wait);
+        PROF_STORE(1, clock64() - prof_start);
+        PROF_STORE(2, issued);
+        if (!ok && lane == 0) {
+            // drain: let the copies already in flight land before the CTA retires
+            const int n_back = issued < p.stages ? (int)issued : p.stages;
+            int s = (int)stage;
+            uint32_t ph = phase;
+            for (int i = 0; i < n_back; ++i) {
+                if (--s < 0) { s = p.stages - 1; ph ^= 1; }
+                for (uint32_t w = 0; w < (1u << 16); ++w) {
+                    if (leader && ptx::mbar_try_wait(&full_bar[s], ph)) break;
+                    __nanosleep(64);
+                    if (!leader && w > 64) break;  // its loads credit the leader's barrier: give them a few microseconds
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------- MMA issuer
-        // The whole warp walks the loop; one elected lane issues the MMAs and their commits.
+        // The whole warp walks the loops; one elected lane issues the MMAs and their commits.
         if (leader) {
             const uint32_t idesc = ptx::idesc_i8(BM * CG, BN);
             const uint64_t adesc0 = ptx::smem_desc(ptx::smem_u32(stage_base), p.BK);
-            const uint64_t bdesc0 = ptx::smem_desc(ptx::smem_u32(stage_base + kABytes), p.BK);
-            const uint64_t stage_step = (uint64_t)(stage_bytes >> 4);
-            int stage = 0;
-            uint32_t phase = 0;
+            const uint32_t desc_hi = (uint32_t)(adesc0 >> 32);
+            const uint32_t a_lo0 = (uint32_t)adesc0;
+            const uint32_t b_lo0 = a_lo0 + (kABytes >> 4);
+            const uint32_t stage_step = (uint32_t)(stage_bytes >> 4);  // stays inside the 14-bit address field
+            const uint32_t empty0 = ptx::smem_u32(empty_bar);
+            const uint32_t full0 = ptx::smem_u32(full_bar);
+            const int ks_full = p.BK >> 5;
+            uint32_t stage = 0, phase = 0;
             int buf = 0;
             uint32_t buf_phase = 0;
             bool ok = true;
             PROF_DECL(prof_wait_acc);
             PROF_DECL(prof_wait_full);
             PROF_T0(prof_start);
-            for (int tile = first_tile; tile < num_tiles && ok; tile += tile_step) {
+            TileWalk tw;
+            for (tw.init(first_tile, tile_step, num_tiles, p.n_tiles); tw.left > 0 && ok; tw.next()) {
                 PROF_T0(t0);
                 if (!__all_sync(0xffffffffu, wait_bounded(&tmem_empty[buf], buf_phase ^ 1, abort_flag, 2))) break;
                 PROF_ADD(prof_wait_acc, t0);
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)buf * buf_stride;
-                KBlockIter it;
-                it.reset(p);
-                uint32_t accumulate = 0;
-                for (int kb = 0; kb < kb_total; ++kb, it.next(p)) {
-                    PROF_T0(t1);
-                    if (!__all_sync(0xffffffffu, wait_bounded(&full_bar[stage], phase, abort_flag, 3))) { ok = false; break; }
-                    PROF_ADD(prof_wait_full, t1);
-                    const int nb = it.part == 0 ? p.nb_lo : p.nb_hi;
-                    int ksteps = p.BK >> 5;
-                    if (it.cb == nb - 1) ksteps = ((it.part == 0 ? p.C_lo : p.C_hi) - it.cb * p.BK + 31) >> 5;
-                    const uint64_t adesc = adesc0 + stage_step * stage;
-                    const uint64_t bdesc = bdesc0 + stage_step * stage;
-                    if (ptx::elect_one()) {
-                        uint32_t acc = accumulate;
-                        for (int k = 0; k < ksteps; ++k) {  // 32 bytes of K per instruction: +2 in 16-byte units
-                            if (CG == 2) ptx::mma_i8_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, acc);
-                            else ptx::mma_i8(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, acc);
+                uint32_t acc = 0;
+                for (int part = 0; part < 2 && ok; ++part) {
+                    const int nb = part ? p.nb_hi : p.nb_lo;
+                    if (nb == 0) continue;
+                    const int ks_last = ((part ? p.C_hi : p.C_lo) - (nb - 1) * p.BK + 31) >> 5;
+                    for (int tap = 0; tap < p.T && ok; ++tap) {
+                        for (int cb = 0; cb < nb; ++cb) {
+                            PROF_T0(t1);
+                            if (!__all_sync(0xffffffffu, wait_bounded(full0 + 8 * stage, phase, abort_flag, 3))) { ok = false; break; }
+                            PROF_ADD(prof_wait_full, t1);
+                            const uint32_t a_lo = a_lo0 + stage * stage_step, b_lo = b_lo0 + stage * stage_step;
+                            const int ks = cb == nb - 1 ? ks_last : ks_full;
+                            if (ptx::elect_one()) {
+                                // 32 bytes of K per instruction: the descriptor address advances by 2 (16-byte units)
+                                if (ks == 4) {
+                                    ptx::mma_i8_s<CG>(d_tmem, a_lo, b_lo, desc_hi, idesc, acc);
+                                    ptx::mma_i8_s<CG>(d_tmem, a_lo + 2, b_lo + 2, desc_hi, idesc, 1);
+                                    ptx::mma_i8_s<CG>(d_tmem, a_lo + 4, b_lo + 4, desc_hi, idesc, 1);
+                                    ptx::mma_i8_s<CG>(d_tmem, a_lo + 6, b_lo + 6, desc_hi, idesc, 1);
+                                } else {
+                                    uint32_t a2 = acc;
+                                    for (int k = 0; k < ks; ++k) {
+                                        ptx::mma_i8_s<CG>(d_tmem, a_lo + 2 * k, b_lo + 2 * k, desc_hi, idesc, a2);
+                                        a2 = 1;
+                                    }
+                                }
+                                ptx::mma_commit_s<CG>(empty0 + 8 * stage);  // frees the stage (in both CTAs of a pair)
+                            }
+                            __syncwarp();
                             acc = 1;
+                            if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
                         }
-                        if (CG == 2) ptx::mma_commit_pair(&empty_bar[stage], 3);  // frees the stage in both CTAs
-                        else ptx::mma_commit(&empty_bar[stage]);
                     }
-                    __syncwarp();
-                    accumulate = 1;
-                    if (++stage == p.stages) { stage = 0; phase ^= 1; }
                 }
-                if (ok && ptx::elect_one()) {
-                    if (CG == 2) ptx::mma_commit_pair(&tmem_full[buf], 3);
-                    else ptx::mma_commit(&tmem_full[buf]);
-                }
+                if (ok && ptx::elect_one()) ptx::mma_commit_s<CG>(ptx::smem_u32(&tmem_full[buf]));
                 __syncwarp();
                 if ((buf ^= 1) == 0) buf_phase ^= 1;
             }
@@ -350,10 +373,10 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
         uint32_t buf_phase = 0;
         PROF_DECL(prof_wait);
         PROF_T0(prof_start);
-        for (int tile = first_tile; tile < num_tiles; tile += tile_step) {
-            const int m_blk = tile / p.n_tiles, n_blk = tile - m_blk * p.n_tiles;
-            const int nw = n_blk * BN + part * cols_per_warp;  // first output channel of this warp
-            const long long row0 = ((long long)m_blk * CG + cta_rank) * BM + quad * 32;
+        TileWalk tw;
+        for (tw.init(first_tile, tile_step, num_tiles, p.n_tiles); tw.left > 0; tw.next()) {
+            const int nw = tw.n_blk * BN + part * cols_per_warp;  // first output channel of this warp
+            const long long row0 = ((long long)tw.m_blk * CG + cta_rank) * BM + quad * 32;
             const int rows_valid = (int)min(32LL, p.M - row0);  // may be <= 0
             // this lane's factor of the first chunk, fetched while the accumulator is still being produced
             float f_next = 0.f;

@@ -158,6 +158,69 @@ __device__ __forceinline__ void tmem_ld_wait()
 }
 
 
+__device__ __forceinline__ void mma_i8_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate);
+
+// ---- variants taking 32-bit shared-memory addresses (hot loops keep them in registers) ----
+__device__ __forceinline__ bool mbar_try_wait_s(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void mbar_expect_tx_s(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+template <int CG>
+__device__ __forceinline__ void tma_load_2d_s(uint32_t dst, const CUtensorMap *m, uint32_t bar, int x, int y)
+{
+    if (CG == 2)
+        asm volatile(
+            "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+            ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(x), "r"(y) : "memory");
+    else
+        asm volatile(
+            "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+            ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+template <int CG>
+__device__ __forceinline__ void tma_load_im2col_4d_s(uint32_t dst, const CUtensorMap *m, uint32_t bar, int c, int w, int h,
+                                                     int n, uint16_t off_w, uint16_t off_h)
+{
+    if (CG == 2)
+        asm volatile(
+            "cp.async.bulk.tensor.4d.im2col.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+            ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h) : "memory");
+    else
+        asm volatile(
+            "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+            ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h) : "memory");
+}
+template <int CG>
+__device__ __forceinline__ void mma_i8_s(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc, uint32_t accumulate)
+{
+    const uint64_t adesc = ((uint64_t)desc_hi << 32) | a_lo, bdesc = ((uint64_t)desc_hi << 32) | b_lo;
+    if (CG == 2) mma_i8_pair(d_tmem, adesc, bdesc, idesc, accumulate);
+    else mma_i8(d_tmem, adesc, bdesc, idesc, accumulate);
+}
+template <int CG>
+__device__ __forceinline__ void mma_commit_s(uint32_t bar)
+{
+    if (CG == 2)
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(bar), "h"((uint16_t)3) : "memory");
+    else
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
 // ---- thread-block clusters and CTA pairs (cta_group::2) ------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank()
 {
