@@ -38,10 +38,9 @@ constexpr int kThreads = 32 * (2 + kNumEpiWarps);
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kABytes = BM * 128;                     // A stage (BK <= 128 bytes per row)
 constexpr int kStageRegion = 196608;                  // shared memory given to the operand ring
-constexpr int kStagingPerWarp = 2048;                 // 32 rows x 64 B output staging per epilogue warp
-constexpr int kFactorsPerWarp = 128;                  // alpha[16], beta[16] of the current column chunk
+constexpr int kFactorsPerWarp = 512;                  // alpha[64] | beta[64] of the warp's columns in the current tile
 constexpr int kMaxStages = 8;
-constexpr int kSmemBytes = kStageRegion + kNumEpiWarps * (kStagingPerWarp + kFactorsPerWarp) + 256;
+constexpr int kSmemBytes = kStageRegion + kNumEpiWarps * kFactorsPerWarp + 256;
 
 struct GemmParams {
     long long M;         // rows of the implicit GEMM (tokens or output pixels)
@@ -124,24 +123,134 @@ __device__ __forceinline__ unsigned requant4(float y0, float y1, float y2, float
     return pack2_sat_s8(__float2int_rn(y1), __float2int_rn(y0), top);
 }
 
-// Staging buffer of one epilogue warp: 32 rows x 64 B, 16-byte units XOR-swizzled so that
-// both the row-per-lane writes and the two-rows-per-quarter-warp reads avoid bank conflicts.
-__device__ __forceinline__ uint4 *staging_unit(uint8_t *stg, int row, int unit)
+// 16 accumulator columns of one row -> 16 output values, through the per-channel factors.
+//   REQUANT_I8 : 16 bytes (one 128-bit word);  DEQUANT_F32 / ACC_I32 : 64 bytes.
+template <int MODE>
+__device__ __forceinline__ void finish16(const uint32_t *r, const float *alpha16, const float *beta16, uint32_t *out)
 {
-    return reinterpret_cast<uint4 *>(stg + row * 64 + ((unit ^ ((row >> 1) & 3)) << 4));
+    const float4 *fa = reinterpret_cast<const float4 *>(alpha16), *fb = reinterpret_cast<const float4 *>(beta16);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        if (MODE == FLEXIQ_OUT_ACC_I32) {
+            out[4 * i + 0] = r[4 * i + 0]; out[4 * i + 1] = r[4 * i + 1]; out[4 * i + 2] = r[4 * i + 2]; out[4 * i + 3] = r[4 * i + 3];
+        } else {
+            const float4 a = fa[i], b = fb[i];
+            const float y0 = fmaf((float)(int)r[4 * i + 0], a.x, b.x), y1 = fmaf((float)(int)r[4 * i + 1], a.y, b.y);
+            const float y2 = fmaf((float)(int)r[4 * i + 2], a.z, b.z), y3 = fmaf((float)(int)r[4 * i + 3], a.w, b.w);
+            if (MODE == FLEXIQ_OUT_REQUANT_I8) {
+                out[i] = requant4(y0, y1, y2, y3);
+            } else {
+                out[4 * i + 0] = __float_as_uint(y0); out[4 * i + 1] = __float_as_uint(y1);
+                out[4 * i + 2] = __float_as_uint(y2); out[4 * i + 3] = __float_as_uint(y3);
+            }
+        }
+    }
+}
+__device__ __forceinline__ void st_global_128(void *p, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ void st_global_256(void *p, const uint32_t *w)
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
 }
 
-// Coalesced copy of the staged rows to global memory: `upr` (1..4) 16-byte units per row.
-__device__ __forceinline__ void flush_staging(uint8_t *stg, int upr, uint8_t *gbase, long long row_pitch_bytes,
-                                              int rows_valid, int units_valid, int lane)
+struct EpilogueCtx {
+    uint32_t tmem_base, buf_stride, cta_rank;
+    uint64_t *tmem_full, *tmem_empty;
+    volatile int *abort_flag;
+    float *fac;
+    int first_tile, tile_step, num_tiles;
+};
+
+// One epilogue warp: TMEM lane quadrant `quad` (32 rows, lane = row), column quarter `part`
+// (BN/4 = 16..64 columns) of every tile of this CTA.  Per tile: fetch the columns' factors,
+// read the whole slice of the accumulator into registers, hand the accumulator back, then
+// scale / round / clip and store each row's bytes straight to global memory.
+template <int CG, int MODE>
+__device__ __forceinline__ void epilogue_role(const GemmParams &p, const EpilogueCtx &x, int quad, int part, int lane)
 {
-    __syncwarp();
-    for (int u = lane; u < 32 * upr; u += 32) {
-        const int row = u / upr, j = u - row * upr;
-        if (row < rows_valid && j < units_valid)
-            *reinterpret_cast<uint4 *>(gbase + row * row_pitch_bytes + j * 16) = *staging_unit(stg, row, j);
+    constexpr bool kScaled = MODE != FLEXIQ_OUT_ACC_I32;
+    constexpr int kElem = MODE == FLEXIQ_OUT_REQUANT_I8 ? 1 : 4;  // output bytes per element
+    const int BN = p.BN;
+    const int cols = BN >> 2;                    // 16, 32, 48 or 64 columns for this warp
+    const bool y32 = (reinterpret_cast<uintptr_t>(p.Y) & 31) == 0;
+    const bool wide = y32 && (p.N & 31) == 0;    // int8 rows are 32-byte aligned: 256-bit stores
+    // lane l keeps factors 4l..4l+3 of the table alpha[64] | beta[64]
+    const float *fsrc = (lane < 16 ? p.alpha : p.beta) + 4 * (lane & 15);
+    int buf = 0;
+    uint32_t buf_phase = 0;
+    PROF_DECL(prof_wait);
+    PROF_T0(prof_start);
+    TileWalk tw;
+    for (tw.init(x.first_tile, x.tile_step, x.num_tiles, p.n_tiles); tw.left > 0; tw.next()) {
+        const int nw = tw.n_blk * BN + part * cols;  // first output channel of this warp
+        const long long row = ((long long)tw.m_blk * CG + x.cta_rank) * BM + quad * 32 + lane;
+        float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (kScaled && nw + 4 * (lane & 15) < p.N) f = __ldg(reinterpret_cast<const float4 *>(fsrc + nw));
+        PROF_T0(t0);
+        const bool ok = wait_bounded(&x.tmem_full[buf], buf_phase, x.abort_flag, 4);
+        PROF_ADD(prof_wait, t0);
+        if (!__all_sync(0xffffffffu, ok)) break;
+        ptx::tc_fence_after_sync();
+        const uint32_t taddr = x.tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)buf * x.buf_stride + (uint32_t)(part * cols);
+        uint32_t ra[32], rb[32];
+        if (cols >= 32) ptx::tmem_ld_32x32(taddr, ra); else ptx::tmem_ld_32x16(taddr, ra);
+        if (cols == 64) ptx::tmem_ld_32x32(taddr + 32, rb); else if (cols == 48) ptx::tmem_ld_32x16(taddr + 32, rb);
+        if (kScaled) {
+            __syncwarp();                                      // the previous tile's reads of the table are done
+            reinterpret_cast<float4 *>(x.fac)[lane] = f;
+            __syncwarp();
+        }
+        ptx::tmem_ld_wait();
+        // the accumulator slice is in registers: hand it back to the MMA warp before the math
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) {
+            if (CG == 2) ptx::mbar_arrive_cluster(ptx::mapa(ptx::smem_u32(&x.tmem_empty[buf]), 0));
+            else ptx::mbar_arrive(&x.tmem_empty[buf]);
+        }
+        if (row < p.M) {
+            uint8_t *yrow = static_cast<uint8_t *>(p.Y) + (row * p.N + nw) * kElem;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {                       // two halves of 32 columns
+                const uint32_t *r = h == 0 ? ra : rb;
+                const int n = nw + 32 * h;
+                if (32 * h < cols && n < p.N) {
+                    const bool second = 32 * h + 16 < cols && n + 16 < p.N;  // columns 16..31 of this half are live
+                    if (MODE == FLEXIQ_OUT_REQUANT_I8) {
+                        uint32_t w[8];
+                        finish16<MODE>(r, x.fac + 32 * h, x.fac + 64 + 32 * h, w);
+                        if (second) finish16<MODE>(r + 16, x.fac + 32 * h + 16, x.fac + 64 + 32 * h + 16, w + 4);
+                        if (second && wide && ((nw & 31) == 0)) st_global_256(yrow + 32 * h, w);  // 32-byte aligned only then
+                        else {
+                            st_global_128(yrow + 32 * h, w[0], w[1], w[2], w[3]);
+                            if (second) st_global_128(yrow + 32 * h + 16, w[4], w[5], w[6], w[7]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int g = 0; g < 2; ++g) {
+                            if (g == 0 || second) {
+                                uint32_t w[16];
+                                finish16<MODE>(r + 16 * g, x.fac + 32 * h + 16 * g, x.fac + 64 + 32 * h + 16 * g, w);
+                                uint8_t *dst = yrow + (32 * h + 16 * g) * 4;
+                                if (y32) {                      // rows of 4-byte elements with N % 16 == 0 are 64-byte aligned
+                                    st_global_256(dst, w);
+                                    st_global_256(dst + 32, w + 8);
+                                } else {
+#pragma unroll
+                                    for (int q = 0; q < 4; ++q) st_global_128(dst + 16 * q, w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+        }
+        if ((buf ^= 1) == 0) buf_phase ^= 1;
     }
-    __syncwarp();
+    if (quad == 2 && part == 0 && lane == 0) { PROF_STORE(8, prof_wait); PROF_STORE(9, clock64() - prof_start); }
 }
 
 // CG = 1: one CTA per 128 x BN tile.  CG = 2: a CTA pair (cluster of two) per 256 x BN tile;
@@ -160,8 +269,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
         return;
     }
     uint8_t *stage_base = smem;
-    uint8_t *staging = smem + kStageRegion;
-    uint8_t *factors = staging + kNumEpiWarps * kStagingPerWarp;
+    uint8_t *factors = smem + kStageRegion;
     uint64_t *full_bar = reinterpret_cast<uint64_t *>(factors + kNumEpiWarps * kFactorsPerWarp);
     uint64_t *empty_bar = full_bar + kMaxStages;
     uint64_t *tmem_full = empty_bar + kMaxStages;
@@ -358,100 +466,17 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
         }
     } else {
         // ------------------------------------------------------------- epilogue
-        // warp e owns TMEM lane quadrant (warp & 3) and one quarter of the tile's columns,
-        // processed 16 columns at a time; the warps do not synchronise with one another.
+        // warp e owns TMEM lane quadrant (warp & 3) and one quarter of the tile's columns;
+        // the warps do not synchronise with one another.
         const int e = warp - 2;
-        const int quad = warp & 3;
-        const int part = e >> 2;
-        const int cols_per_warp = BN >> 2;           // 16, 32, 48 or 64
-        const int n_chunks = cols_per_warp >> 4;
-        uint8_t *stg = staging + e * kStagingPerWarp;
-        float *fac = reinterpret_cast<float *>(factors + e * kFactorsPerWarp);  // alpha[16] | beta[16]
-        const bool scaled = p.out_mode != FLEXIQ_OUT_ACC_I32;
-        const float *fsrc = lane < 16 ? p.alpha : p.beta;                       // lanes 0-15 fetch alpha, 16-31 beta
-        int buf = 0;
-        uint32_t buf_phase = 0;
-        PROF_DECL(prof_wait);
-        PROF_T0(prof_start);
-        TileWalk tw;
-        for (tw.init(first_tile, tile_step, num_tiles, p.n_tiles); tw.left > 0; tw.next()) {
-            const int nw = tw.n_blk * BN + part * cols_per_warp;  // first output channel of this warp
-            const long long row0 = ((long long)tw.m_blk * CG + cta_rank) * BM + quad * 32;
-            const int rows_valid = (int)min(32LL, p.M - row0);  // may be <= 0
-            // this lane's factor of the first chunk, fetched while the accumulator is still being produced
-            float f_next = 0.f;
-            if (scaled && nw + (lane & 15) < p.N) f_next = __ldg(fsrc + nw + (lane & 15));
-            PROF_T0(t0);
-            const bool ok = wait_bounded(&tmem_full[buf], buf_phase, abort_flag, 4);
-            PROF_ADD(prof_wait, t0);
-            if (!__all_sync(0xffffffffu, ok)) break;
-            ptx::tc_fence_after_sync();
-            const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)buf * buf_stride + (uint32_t)(part * cols_per_warp);
-            uint32_t ra[16], rb[16];
-            ptx::tmem_ld_32x16(taddr, ra);
-#pragma unroll 1
-            for (int ch = 0; ch < n_chunks; ch += 2) {
-#pragma unroll
-                for (int sub = 0; sub < 2; ++sub) {
-                    const int c = ch + sub;
-                    if (c >= n_chunks) break;
-                    uint32_t *r = sub == 0 ? ra : rb;
-                    ptx::tmem_ld_wait();
-                    const bool last = c + 1 == n_chunks;
-                    if (!last) ptx::tmem_ld_32x16(taddr + 16 * (c + 1), sub == 0 ? rb : ra);
-                    const int n = nw + 16 * c;                 // first output channel of this chunk
-                    const bool live = n < p.N && rows_valid > 0;
-                    if (scaled) {
-                        __syncwarp();
-                        fac[lane] = f_next;
-                        __syncwarp();
-                        f_next = 0.f;
-                        if (!last && n + 16 + (lane & 15) < p.N) f_next = __ldg(fsrc + n + 16 + (lane & 15));
-                    }
-                    if (last) {
-                        // every TMEM read of this tile has landed: hand the accumulator back to the MMA warp
-                        ptx::tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) {
-                            if (CG == 2) ptx::mbar_arrive_cluster(ptx::mapa(ptx::smem_u32(&tmem_empty[buf]), 0));
-                            else ptx::mbar_arrive(&tmem_empty[buf]);
-                        }
-                    }
-                    if (!live) continue;
-                    const float4 *fa = reinterpret_cast<const float4 *>(fac), *fb = reinterpret_cast<const float4 *>(fac + 16);
-                    if (p.out_mode == FLEXIQ_OUT_REQUANT_I8) {
-                        unsigned w[4];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const float4 a = fa[i], b = fb[i];
-                            w[i] = requant4(fmaf((float)(int)r[4 * i + 0], a.x, b.x), fmaf((float)(int)r[4 * i + 1], a.y, b.y),
-                                            fmaf((float)(int)r[4 * i + 2], a.z, b.z), fmaf((float)(int)r[4 * i + 3], a.w, b.w));
-                        }
-                        *staging_unit(stg, lane, c) = make_uint4(w[0], w[1], w[2], w[3]);  // 16 output bytes of this row
-                        if (last || n + 16 >= p.N)                                        // no live chunk follows
-                            flush_staging(stg, c + 1, static_cast<uint8_t *>(p.Y) + row0 * p.N + nw, (long long)p.N,
-                                          rows_valid, (p.N - nw) >> 4, lane);
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {              // 16 columns x 4 bytes = 64 staged bytes per row
-                            uint4 v = make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
-                            if (p.out_mode == FLEXIQ_OUT_DEQUANT_F32) {
-                                const float4 a = fa[i], b = fb[i];
-                                v.x = __float_as_uint(fmaf((float)(int)r[4 * i + 0], a.x, b.x));
-                                v.y = __float_as_uint(fmaf((float)(int)r[4 * i + 1], a.y, b.y));
-                                v.z = __float_as_uint(fmaf((float)(int)r[4 * i + 2], a.z, b.z));
-                                v.w = __float_as_uint(fmaf((float)(int)r[4 * i + 3], a.w, b.w));
-                            }
-                            *staging_unit(stg, lane, i) = v;
-                        }
-                        flush_staging(stg, 4, static_cast<uint8_t *>(p.Y) + (row0 * p.N + n) * 4, (long long)p.N * 4,
-                                      rows_valid, (p.N - n) >> 2, lane);
-                    }
-                }
-            }
-            if ((buf ^= 1) == 0) buf_phase ^= 1;
-        }
-        if (e == 0 && lane == 0) { PROF_STORE(8, prof_wait); PROF_STORE(9, clock64() - prof_start); }
+        EpilogueCtx x;
+        x.tmem_base = tmem_base; x.buf_stride = buf_stride; x.cta_rank = cta_rank;
+        x.tmem_full = tmem_full; x.tmem_empty = tmem_empty; x.abort_flag = abort_flag;
+        x.fac = reinterpret_cast<float *>(factors + e * kFactorsPerWarp);  // alpha[64] | beta[64]
+        x.first_tile = first_tile; x.tile_step = tile_step; x.num_tiles = num_tiles;
+        if (p.out_mode == FLEXIQ_OUT_REQUANT_I8) epilogue_role<CG, FLEXIQ_OUT_REQUANT_I8>(p, x, warp & 3, e >> 2, lane);
+        else if (p.out_mode == FLEXIQ_OUT_DEQUANT_F32) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_F32>(p, x, warp & 3, e >> 2, lane);
+        else epilogue_role<CG, FLEXIQ_OUT_ACC_I32>(p, x, warp & 3, e >> 2, lane);
     }
 
     ptx::tc_fence_before_sync();
