@@ -208,8 +208,8 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
         ptx::tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) {
-            if (CG == 2) ptx::mbar_arrive_cluster(ptx::mapa(ptx::smem_u32(&x.tmem_empty[buf]), 0));
-            else ptx::mbar_arrive(&x.tmem_empty[buf]);
+            if (CG == 2) ptx::mbar_arrive_cluster_relaxed(ptx::mapa(ptx::smem_u32(&x.tmem_empty[buf]), 0));
+            else ptx::mbar_arrive_relaxed(&x.tmem_empty[buf]);
         }
         if (row < p.M) {
             uint8_t *yrow = static_cast<uint8_t *>(p.Y) + (row * p.N + nw) * kElem;
@@ -505,17 +505,19 @@ __global__ void scale_vectors_kernel(int N, float x_scale, float y_scale, int re
 // ------------------------------------------------------------------------------------
 // host side
 
-// Tile shape.  Operand traffic from L2 bounds the mainloop on this part, so the cost of a
-// tile is the larger of its operand bytes per SM and its MMA time (both per byte of K),
-// times the number of machine waves; cg = 2 pairs two CTAs on a 256-row tile.
+// Tile shape, from a cost model with constants measured on B200 (cycles per 128-byte K block):
+// the MMA takes 2*BN cycles, the TMA fill of the operands about (128 + BN/cg) * 128 / 97, and no
+// K block goes faster than about 420 cycles of issue overhead; the epilogue of a tile takes about
+// 2400 + 8 * BN cycles and, being overlapped, only costs when it exceeds the mainloop (ties go to the
+// configuration listed first).  cost = waves * tile time.
 struct TileChoice { int cg, bn; };
 static TileChoice g_forced_tile{0, 0};  // test hook: 0 = choose automatically
-static TileChoice choose_tile(long long M, int N, int sms)
+static TileChoice choose_tile(long long M, int N, int k_blocks, int sms)
 {
     const int bns[4] = {256, 192, 128, 64};
     TileChoice best{1, 256};
     double best_cost = 1e300;
-    for (int cg = 1; cg <= 2; ++cg)
+    for (int cg = 2; cg >= 1; --cg)  // pairs first: they halve the B traffic per SM
         for (int i = 0; i < 4; ++i) {
             const int bn = bns[i];
             if (cg == 2 && bn < 128) continue;
@@ -523,8 +525,13 @@ static TileChoice choose_tile(long long M, int N, int sms)
             const long long n_tiles = (N + bn - 1) / bn;
             const long long slots = sms / cg;
             const long long waves = (m_tiles * n_tiles + slots - 1) / slots;
-            const double l2 = (128.0 + (double)bn / cg) / 36.0, mma = bn / 64.0;
-            const double cost = (double)waves * (l2 > mma ? l2 : mma);
+            double per_kb = 2.0 * bn;
+            const double tma = (128.0 + (double)bn / cg) * 128.0 / 97.0;
+            if (tma > per_kb) per_kb = tma;
+            if (per_kb < 420.0) per_kb = 420.0;
+            const double mainloop = k_blocks * per_kb + 800.0;
+            const double epi = 2400.0 + 8.0 * bn;
+            const double cost = (double)waves * (mainloop > epi ? mainloop : epi);
             if (cost < best_cost - 1e-9) { best_cost = cost; best = TileChoice{cg, bn}; }
         }
     return best;
@@ -617,7 +624,7 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     }
     p.out_mode = out_mode; p.Y = Y;
     p.alpha = L->alpha; p.beta = L->beta;
-    const TileChoice tc = g_forced_tile.cg ? g_forced_tile : choose_tile(M, L->N, sms);
+    const TileChoice tc = g_forced_tile.cg ? g_forced_tile : choose_tile(M, L->N, p.T * (p.nb_lo + p.nb_hi), sms);
     const int bn = tc.bn, cg = tc.cg;
     p.m_tiles = (int)((M + (long long)BM * cg - 1) / ((long long)BM * cg));
     p.BN = bn;

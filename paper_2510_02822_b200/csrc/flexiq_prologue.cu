@@ -1,6 +1,6 @@
 // Activation prologue: quantize (Sec. 2.1, Eq. 1), bit-lower (Sec. 4.1, Fig. 3) and
 // gather the channel groups into slab order (Sec. 5), writing the low-bit slab and the
-// 8-bit slab that the mainloop consumes.  HBM-bound: one pass over X (two in the dynamic
+// 8-bit slab that the mainloop consumes.  One pass over X (two in the dynamic
 // extraction-position mode), 128-bit loads and stores, one 16-channel chunk per thread.
 #include "flexiq_internal.h"
 
@@ -9,22 +9,58 @@
 
 namespace flexiq {
 
-// Loads the 16 channels starting at p and quantizes them with Eq. 1:
-// q = clip(round_half_even(x / S), -128, 127); IEEE division, no fast-math.
+// Eq. 1 divides by the scale.  The scale is the same for every element, so its correctly
+// rounded reciprocal r = RN(1/S) is computed once per thread and each quotient follows from
+// two Newton corrections with exact fused residuals:
+//     t = RN(x*r);  t = RN(t + r*(x - S*t));  t = RN(t + r*(x - S*t))
+// With r correctly rounded and the first corrected t faithful, the last step yields the
+// correctly rounded quotient RN(x/S) (Markstein's theorem), i.e. the IEEE division result,
+// at five instructions per element.  (Only the final integer matters here: results in the
+// subnormal range may differ but round to 0 either way; inf / NaN inputs are excluded.)
+struct Divider {
+    float S, r;
+    __device__ __forceinline__ float operator()(float x) const
+    {
+        float t = __fmul_rn(x, r);
+        t = __fmaf_rn(__fmaf_rn(-S, t, x), r, t);
+        t = __fmaf_rn(__fmaf_rn(-S, t, x), r, t);
+        return t;
+    }
+};
+__device__ __forceinline__ Divider make_divider(float scale)
+{
+    Divider d;
+    d.S = scale;
+    d.r = __frcp_rn(scale);
+    return d;
+}
+
+// two int32 -> two saturated int8 in the low half, upper half taken from c's low half
+__device__ __forceinline__ unsigned pack2_sat_s8(int hi, int lo, unsigned c)
+{
+    unsigned d;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(hi), "r"(lo), "r"(c));
+    return d;
+}
+// clip(round_half_even(t), -128, 127) of four values, packed little-endian
+__device__ __forceinline__ unsigned quant4(float t0, float t1, float t2, float t3)
+{
+    const unsigned top = pack2_sat_s8(__float2int_rn(t3), __float2int_rn(t2), 0u);
+    return pack2_sat_s8(__float2int_rn(t1), __float2int_rn(t0), top);
+}
+
+// Loads the 16 channels starting at p as fp32 (exact widening for fp16 / bf16).
 template <int DTYPE>
-__device__ __forceinline__ void load_quantize16(const void *p, float S, int q[16])
+__device__ __forceinline__ void load16(const void *p, float x[16])
 {
     if (DTYPE == FLEXIQ_DTYPE_F32) {
         const float4 *v = reinterpret_cast<const float4 *>(p);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const float4 f = __ldg(v + i);
-            q[4 * i + 0] = __float2int_rn(__fdiv_rn(f.x, S));
-            q[4 * i + 1] = __float2int_rn(__fdiv_rn(f.y, S));
-            q[4 * i + 2] = __float2int_rn(__fdiv_rn(f.z, S));
-            q[4 * i + 3] = __float2int_rn(__fdiv_rn(f.w, S));
+            x[4 * i + 0] = f.x; x[4 * i + 1] = f.y; x[4 * i + 2] = f.z; x[4 * i + 3] = f.w;
         }
-    } else if (DTYPE == FLEXIQ_DTYPE_F16 || DTYPE == FLEXIQ_DTYPE_BF16) {
+    } else {
         const uint4 *v = reinterpret_cast<const uint4 *>(p);
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
@@ -32,30 +68,46 @@ __device__ __forceinline__ void load_quantize16(const void *p, float S, int q[16
             const unsigned w[4] = {u.x, u.y, u.z, u.w};
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                float lo, hi;
                 if (DTYPE == FLEXIQ_DTYPE_F16) {
                     const __half2 h = *reinterpret_cast<const __half2 *>(&w[k]);
-                    lo = __low2float(h);
-                    hi = __high2float(h);
-                } else {  // bf16 widens exactly: the 16 bits are the top half of an fp32
-                    lo = __uint_as_float(w[k] << 16);
-                    hi = __uint_as_float(w[k] & 0xffff0000u);
+                    x[8 * i + 2 * k] = __low2float(h);
+                    x[8 * i + 2 * k + 1] = __high2float(h);
+                } else {  // bf16: the 16 bits are the top half of an fp32
+                    x[8 * i + 2 * k] = __uint_as_float(w[k] << 16);
+                    x[8 * i + 2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
                 }
-                q[8 * i + 2 * k] = __float2int_rn(__fdiv_rn(lo, S));
-                q[8 * i + 2 * k + 1] = __float2int_rn(__fdiv_rn(hi, S));
             }
         }
-    } else {  // already int8
-        const uint4 u = __ldg(reinterpret_cast<const uint4 *>(p));
-        const unsigned w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-#pragma unroll
-            for (int b = 0; b < 4; ++b) q[4 * k + b] = (int)(signed char)((w[k] >> (8 * b)) & 0xff);
     }
-    if (DTYPE != FLEXIQ_DTYPE_I8) {
+}
+
+// The 16 channels of one slab chunk as four words of packed int8: q = Eq. 1 of the input,
+// clipped to [lo, hi] (both integers, so clipping before the rounding gives the same value
+// as clipping after it).  int8 input is only clipped.
+template <int DTYPE>
+__device__ __forceinline__ void quantize16(const void *p, const Divider &div, float lo, float hi, unsigned w[4])
+{
+    if (DTYPE == FLEXIQ_DTYPE_I8) {
+        const uint4 u = __ldg(reinterpret_cast<const uint4 *>(p));
+        const unsigned in[4] = {u.x, u.y, u.z, u.w};
+        const int ilo = (int)lo, ihi = (int)hi;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) q[i] = max(-128, min(127, q[i]));
+        for (int k = 0; k < 4; ++k) {
+            int b[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) b[j] = max(ilo, min(ihi, (int)(signed char)((in[k] >> (8 * j)) & 0xff)));
+            w[k] = pack2_sat_s8(b[1], b[0], pack2_sat_s8(b[3], b[2], 0u));
+        }
+    } else {
+        float x[16];
+        load16<DTYPE>(p, x);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            float t[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) t[j] = fminf(fmaxf(div(x[4 * k + j]), lo), hi);
+            w[k] = quant4(t[0], t[1], t[2], t[3]);
+        }
     }
 }
 
@@ -88,16 +140,22 @@ __global__ void group_or_kernel(const void *__restrict__ X, long long M, int K, 
     const long long rows_per_pass = nthreads / n_c16;
     const int c16 = (int)(tid % n_c16);
     const int j = c16 / c_per_g;
+    const Divider div = make_divider(S);
     unsigned o = 0;
     if (tid < rows_per_pass * n_c16) {
         const int src_c = perm[j] * G + (c16 % c_per_g) * 16;
         for (long long m = tid / n_c16; m < M; m += rows_per_pass) {
-            int q[16];
-            load_quantize16<DTYPE>(reinterpret_cast<const char *>(X) + ((size_t)m * K + src_c) * elem_bytes<DTYPE>(), S, q);
+            unsigned w[4];
+            quantize16<DTYPE>(reinterpret_cast<const char *>(X) + ((size_t)m * K + src_c) * elem_bytes<DTYPE>(), div, -128.f, 127.f, w);
+            // fold negatives per byte (q >= 0 ? q : ~q): xor with the byte's sign replicated
 #pragma unroll
-            for (int i = 0; i < 16; ++i) o |= (unsigned)(q[i] ^ (q[i] >> 31));  // q >= 0 ? q : ~q
+            for (int k = 0; k < 4; ++k) {
+                const unsigned sign = (w[k] >> 7) & 0x01010101u;
+                o |= w[k] ^ (sign * 0xffu);
+            }
         }
     }
+    o = (o | (o >> 8) | (o >> 16) | (o >> 24)) & 0xffu;  // OR of the four byte lanes
     const unsigned peers = __match_any_sync(0xffffffffu, j);
     const unsigned merged = __reduce_or_sync(peers, o);
     if ((threadIdx.x & 31) == (__ffs(peers) - 1) && merged) atomicOr(&or_s[j], merged);
@@ -108,6 +166,10 @@ __global__ void group_or_kernel(const void *__restrict__ X, long long M, int K, 
 
 // Quantize + lower + gather.  Thread <-> (row m, 16-channel slab chunk c16).
 //   sx != nullptr : static positions (slab order);  else positions from or_words.
+// Lowering works on the packed int8 words: q is first clipped to the range the 4-bit value
+// at position s can hold, [-2^(s+3), 2^(s+3) - 1] (identical to clamping q >> s to [-8, 7],
+// the shift being monotone); then bits s..s+3 of every byte are the two's-complement nibble
+// (packed path), and clearing the s low bits of every byte is (q >> s) << s (masked path).
 template <int DTYPE, int PACKED>
 __global__ void quantize_lower_kernel(const void *__restrict__ X, long long M, int K, int G, int K_lo, float S,
                                       const int32_t *__restrict__ perm, const uint8_t *__restrict__ sx,
@@ -117,6 +179,7 @@ __global__ void quantize_lower_kernel(const void *__restrict__ X, long long M, i
     const int n_c16 = K / 16, c_per_g = G / 16, lo_c16 = K_lo / 16;
     const int K_hi = K - K_lo;
     const long long total = M * n_c16;
+    const Divider div = make_divider(S);
     if (sx_out != nullptr && blockIdx.x == 0)
         for (int j = threadIdx.x; j < K / G; j += blockDim.x) sx_out[j] = (uint8_t)position_from_or(or_words[j]);
     for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
@@ -125,43 +188,29 @@ __global__ void quantize_lower_kernel(const void *__restrict__ X, long long M, i
         const int c16 = (int)(idx - m * n_c16);
         const int j = c16 / c_per_g;
         const int src_c = perm[j] * G + (c16 % c_per_g) * 16;
-        int q[16];
-        load_quantize16<DTYPE>(reinterpret_cast<const char *>(X) + ((size_t)m * K + src_c) * elem_bytes<DTYPE>(), S, q);
+        const void *src = reinterpret_cast<const char *>(X) + ((size_t)m * K + src_c) * elem_bytes<DTYPE>();
+        unsigned w[4];
         if (c16 < lo_c16) {
             const int s = sx ? (int)sx[j] : position_from_or(or_words[j]);
-            int v[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) v[i] = max(-8, min(7, q[i] >> s));  // arithmetic shift, saturate
+            const float bound = (float)(8 << s);
+            quantize16<DTYPE>(src, div, -bound, bound - 1.f, w);
             if (PACKED) {
-                unsigned w[2];
+                unsigned h[4];
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    unsigned acc = 0;
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) acc |= (unsigned)(v[8 * h + i] & 15) << (4 * i);
-                    w[h] = acc;
+                for (int k = 0; k < 4; ++k) {
+                    const unsigned n = (w[k] >> s) & 0x0f0f0f0fu;  // one nibble per byte
+                    h[k] = n | (n >> 4);                            // bytes 0 and 2 now hold two nibbles each
                 }
-                *reinterpret_cast<uint2 *>(X4 + m * x4_pitch + (size_t)c16 * 8) = make_uint2(w[0], w[1]);
+                *reinterpret_cast<uint2 *>(X4 + m * x4_pitch + (size_t)c16 * 8) =
+                    make_uint2(__byte_perm(h[0], h[1], 0x6420), __byte_perm(h[2], h[3], 0x6420));
             } else {
-                unsigned w[4];
-#pragma unroll
-                for (int h = 0; h < 4; ++h) {
-                    unsigned acc = 0;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) acc |= (unsigned)((v[4 * h + i] << s) & 0xff) << (8 * i);
-                    w[h] = acc;
-                }
-                *reinterpret_cast<uint4 *>(X4 + m * x4_pitch + (size_t)c16 * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+                const unsigned keep = (0xffu << s) & 0xffu;
+                const unsigned mask = keep * 0x01010101u;
+                *reinterpret_cast<uint4 *>(X4 + m * x4_pitch + (size_t)c16 * 16) =
+                    make_uint4(w[0] & mask, w[1] & mask, w[2] & mask, w[3] & mask);
             }
         } else {
-            unsigned w[4];
-#pragma unroll
-            for (int h = 0; h < 4; ++h) {
-                unsigned acc = 0;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) acc |= (unsigned)(q[4 * h + i] & 0xff) << (8 * i);
-                w[h] = acc;
-            }
+            quantize16<DTYPE>(src, div, -128.f, 127.f, w);
             *reinterpret_cast<uint4 *>(X8 + m * (long long)K_hi + (size_t)(c16 - lo_c16) * 16) = make_uint4(w[0], w[1], w[2], w[3]);
         }
     }

@@ -121,6 +121,37 @@ def test_half_precision_inputs(dev, dtype):
     _run_linear(inputs.ranged_linear("h", 200, 256, 64, 16, seed=6, group_structured=True), dev, [0.5], x_dtype=dtype)
 
 
+@pytest.mark.parametrize("S", [0.033, 0.0123457, 1.7e-3, 0.61, 3.3, 0.25])
+def test_quantization_matches_ieee_division_near_ties(dev, S):
+    # Values within a few ulps of every rounding boundary (k + 0.5) * S: the kernel's
+    # reciprocal-based quotient must round exactly like the oracle's IEEE division.
+    S = float(np.float32(S))
+    ks = np.arange(-131, 131, dtype=np.float64) + 0.5
+    base = (ks * S).astype(np.float32)
+    vals = [base]
+    for _ in range(4):
+        vals.append(np.nextafter(vals[-1], np.float32(np.inf)))
+    lo = base
+    for _ in range(4):
+        lo = np.nextafter(lo, np.float32(-np.inf))
+        vals.append(lo)
+    rng = np.random.default_rng(7)
+    x = np.concatenate(vals + [rng.uniform(-140 * S, 140 * S, 4096).astype(np.float32)])
+    K, G = 64, 16
+    M = (x.size + K - 1) // K
+    X = np.zeros((M, K), np.float32)
+    X.reshape(-1)[:x.size] = x
+    perm = np.arange(K // G, dtype=np.int32)
+    Wq = torch.zeros((K, 16), dtype=torch.int8, device=dev)
+    L = fx.Layer(Wq, torch.ones(16, device=dev), None, perm, np.zeros(K // G, np.uint8), G)
+    L.set_lowbit_ratio(0.0)
+    x4, x8, _ = L.quantize_lower(torch.from_numpy(X).to(dev), S)
+    torch.cuda.synchronize()
+    got = x8[:M * K].view(M, K).cpu().numpy()
+    assert np.array_equal(got, oracle.quantize(X, S))
+    L.close()
+
+
 def test_dynamic_positions(dev):
     case = inputs.ranged_linear("dyn", 333, 384, 96, 16, seed=21, group_structured=True)
     _run_linear(case, dev, [0.5, 1.0], dynamic=True)
