@@ -127,6 +127,29 @@ int flexiq_quantize_lower(flexiq_layer_t layer, const void *X_dev, int x_dtype, 
                           float x_scale, int dynamic_pos, uint8_t *X4_dev, int8_t *X8_dev,
                           uint8_t *x_shift_out_dev, uint32_t *scratch_dev, void *stream);
 
+/* Dynamic-position prologue for callers that must not allocate device memory.  (The paper has
+ * no counterpart; this is a convenience of this library.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a region being captured
+ * into a CUDA graph, inside a memory-pool callback or an allocator hook, in a real-time serving
+ * loop that has handed all device memory to another allocator -- and that therefore cannot set
+ * aside the K/G scratch words flexiq_quantize_lower(dynamic_pos = 1) asks its caller for.  This
+ * entry point behaves exactly like that call (same arguments otherwise, same results), but takes
+ * its scratch from a fixed array inside the library and calls no allocating routine at all.
+ *
+ * Limits and rules:
+ *   - at most 4096 channel groups per layer (K/G <= 4096); larger layers get
+ *     FLEXIQ_ERR_INVALID_ARG and should use flexiq_quantize_lower with their own scratch.
+ *     The array costs 16 KB of device memory on every GPU that loads the library, until exit.
+ *   - the first call on each device looks up the array's device address (with that device
+ *     current) and caches it; make that first call outside any stream capture.
+ *   - every call on a device shares the one array (it is cleared at the start of each call, on
+ *     `stream`): calls whose kernels may overlap on the GPU -- different streams without an
+ *     ordering between them -- race on it and give wrong positions.  Keep such calls ordered. */
+int flexiq_quantize_lower_dynamic_noalloc(flexiq_layer_t layer, const void *X_dev, int x_dtype,
+                                          int64_t M, float x_scale, uint8_t *X4_dev, int8_t *X8_dev,
+                                          uint8_t *x_shift_out_dev, void *stream);
+
 /* Mixed-precision GEMM (Sec. 7; objective of Sec. 2.3):
  *   acc[m][n] = sum_{j <  n_low} ( sum_i x4[m][j,i] * w4[j,i][n] ) << (sx[j] + sw[j][n])
  *             + sum_{j >= n_low}   sum_i x8[m][j,i] * w8[j,i][n]            (exact int32)

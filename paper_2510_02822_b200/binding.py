@@ -21,7 +21,7 @@ LOWBIT_MASKED_I8, LOWBIT_PACKED_U4 = 0, 1
 EXPORTS = [
     "flexiq_layer_create_linear", "flexiq_layer_create_conv", "flexiq_layer_destroy",
     "flexiq_layer_set_lowbit_path", "flexiq_set_lowbit_ratio", "flexiq_get_max_4bit_ch",
-    "flexiq_x4_pitch", "flexiq_quantize_lower", "flexiq_mixed_gemm", "flexiq_mixed_conv",
+    "flexiq_x4_pitch", "flexiq_quantize_lower", "flexiq_quantize_lower_dynamic_noalloc", "flexiq_mixed_gemm", "flexiq_mixed_conv",
     "flexiq_layer_export", "flexiq_force_tile", "flexiq_check_status", "flexiq_last_error",
 ]
 
@@ -53,6 +53,7 @@ def lib():
         L.flexiq_get_max_4bit_ch.argtypes = [vp, C.POINTER(i32)]
         L.flexiq_x4_pitch.argtypes = [vp, i32, C.POINTER(i64)]
         L.flexiq_quantize_lower.argtypes = [vp, vp, i32, i64, f32, i32, vp, vp, vp, vp, vp]
+        L.flexiq_quantize_lower_dynamic_noalloc.argtypes = [vp, vp, i32, i64, f32, vp, vp, vp, vp]
         L.flexiq_mixed_gemm.argtypes = [vp, vp, vp, vp, i64, f32, f32, i32, vp, vp]
         L.flexiq_mixed_conv.argtypes = [vp, vp, vp, vp, i32, i32, i32, f32, f32, i32, vp, vp]
         L.flexiq_layer_export.argtypes = [vp, vp, vp, vp]
@@ -126,6 +127,13 @@ def flexiq_quantize_lower(h, X_dev, x_dtype, M, x_scale, dynamic_pos, X4_dev, X8
                           scratch_dev=None):
     _check(lib().flexiq_quantize_lower(h, _ptr(X_dev), x_dtype, M, x_scale, int(dynamic_pos), _ptr(X4_dev), _ptr(X8_dev),
                                        _ptr(x_shift_out_dev), _ptr(scratch_dev), _stream()))
+
+
+def flexiq_quantize_lower_dynamic_noalloc(h, X_dev, x_dtype, M, x_scale, X4_dev, X8_dev, x_shift_out_dev):
+    """Dynamic-position prologue that allocates nothing: its scratch is a fixed array inside the
+    library (at most 4096 channel groups; calls on one device must not overlap)."""
+    _check(lib().flexiq_quantize_lower_dynamic_noalloc(h, _ptr(X_dev), x_dtype, M, x_scale, _ptr(X4_dev), _ptr(X8_dev),
+                                                       _ptr(x_shift_out_dev), _stream()))
 
 
 def flexiq_mixed_gemm(h, X4_dev, X8_dev, x_shift_dev, M, x_scale, y_scale, out_mode, Y_dev):

@@ -216,6 +216,31 @@ __global__ void quantize_lower_kernel(const void *__restrict__ X, long long M, i
     }
 }
 
+// Scratch of the allocation-free dynamic prologue: one OR word per channel group.  The array
+// lives in the library image, so every GPU that loads the library holds these 16 KB until the
+// process exits.  All calls on a device share it.
+constexpr int kStaticScratchGroups = 4096;
+static __device__ __align__(256) unsigned g_static_group_or[kStaticScratchGroups];
+
+// Device address of the array above on the current device.  In host code the array's name is
+// only a handle for the runtime, not a device pointer, so the address is looked up with
+// cudaGetSymbolAddress -- once per device, with that device current -- and cached.
+static int static_scratch_address(unsigned **out)
+{
+    static unsigned *cached[64] = {};
+    int dev = 0;
+    FLEXIQ_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return set_error(FLEXIQ_ERR_UNSUPPORTED, "device ordinal %d is beyond the 64 this entry point tracks", dev);
+    if (cached[dev] == nullptr) {
+        void *p = nullptr;
+        FLEXIQ_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_group_or));
+        if (p == nullptr) return set_error(FLEXIQ_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
+        cached[dev] = static_cast<unsigned *>(p);
+    }
+    *out = cached[dev];
+    return FLEXIQ_OK;
+}
+
 template <int DTYPE>
 static int launch_prologue(const Layer *L, const void *X, long long M, float S, int dynamic, uint8_t *X4,
                            long long pitch, int8_t *X8, uint8_t *sx_out, unsigned *scratch, cudaStream_t st)
@@ -280,4 +305,20 @@ extern "C" int flexiq_quantize_lower(flexiq_layer_t layer, const void *X_dev, in
         case FLEXIQ_DTYPE_BF16: return launch_prologue<FLEXIQ_DTYPE_BF16>(L, X_dev, M, x_scale, dynamic_pos, X4_dev, pitch, X8_dev, x_shift_out_dev, scratch_dev, st);
         default: return launch_prologue<FLEXIQ_DTYPE_I8>(L, X_dev, M, x_scale, dynamic_pos, X4_dev, pitch, X8_dev, x_shift_out_dev, scratch_dev, st);
     }
+}
+
+extern "C" int flexiq_quantize_lower_dynamic_noalloc(flexiq_layer_t layer, const void *X_dev, int x_dtype, int64_t M,
+                                                     float x_scale, uint8_t *X4_dev, int8_t *X8_dev,
+                                                     uint8_t *x_shift_out_dev, void *stream)
+{
+    Layer *L = as_layer(layer);
+    if (!L) return set_error(FLEXIQ_ERR_INVALID_ARG, "not a live flexiq layer handle");
+    if (L->n_g > kStaticScratchGroups)
+        return set_error(FLEXIQ_ERR_INVALID_ARG,
+                         "layer has %d channel groups; the built-in scratch of this entry point holds at most %d "
+                         "(use flexiq_quantize_lower with caller-provided scratch instead)", L->n_g, kStaticScratchGroups);
+    unsigned *scratch = nullptr;
+    const int rc = static_scratch_address(&scratch);
+    if (rc) return rc;
+    return flexiq_quantize_lower(layer, X_dev, x_dtype, M, x_scale, 1, X4_dev, X8_dev, x_shift_out_dev, scratch, stream);
 }
