@@ -14,6 +14,8 @@
 #include "flexiq_internal.h"
 #include "sm100_ptx.cuh"
 
+#include <stdlib.h>
+
 namespace flexiq {
 
 __device__ unsigned int g_status_word = 0;
@@ -309,6 +311,11 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
     else __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_ptr_s;
+    // Everything above touched only this CTA's shared and tensor memory, so it may overlap the tail
+    // of the previous kernel of the stream (programmatic dependent launch); wait for that kernel
+    // (the prologue that writes the slabs) before reading or writing global memory.  This kernel
+    // does not release its own successor early: a successor parked on the SMs slows the mainloop.
+    ptx::pdl_wait();
 
     if (warp == 0) {
         // ------------------------------------------------------------- TMA producer
@@ -577,13 +584,15 @@ static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const
     cfg.blockDim = dim3(kThreads, 1, 1);
     cfg.dynamicSmemBytes = kSmemBytes;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = CG;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // overlap this launch's preamble with the predecessor's tail
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     FLEXIQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, mixed_gemm_kernel<CG>, a_lo, a_hi, b_lo, b_hi, p));
     return FLEXIQ_OK;
 }

@@ -7,6 +7,10 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include "sm100_ptx.cuh"
+
+#include <stdlib.h>
+
 namespace flexiq {
 
 // Eq. 1 divides by the scale.  The scale is the same for every element, so its correctly
@@ -133,6 +137,8 @@ __global__ void group_or_kernel(const void *__restrict__ X, long long M, int K, 
     extern __shared__ unsigned or_s[];
     const int n_c16 = K / 16, c_per_g = G / 16, n_g = K / G;
     for (int i = threadIdx.x; i < n_g; i += blockDim.x) or_s[i] = 0;
+    ptx::pdl_launch_dependents();
+    ptx::pdl_wait();  // the kernel before this one in the stream may still be producing X
     __syncthreads();
     // grid-wide thread count is a multiple of n_c16, so each thread keeps its chunk column
     const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -180,6 +186,8 @@ __global__ void quantize_lower_kernel(const void *__restrict__ X, long long M, i
     const int K_hi = K - K_lo;
     const long long total = M * n_c16;
     const Divider div = make_divider(S);
+    ptx::pdl_launch_dependents();
+    ptx::pdl_wait();  // the previous kernel may still read the slabs this one overwrites, or write X
     if (sx_out != nullptr && blockIdx.x == 0)
         for (int j = threadIdx.x; j < K / G; j += blockDim.x) sx_out[j] = (uint8_t)position_from_or(or_words[j]);
     for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
@@ -241,6 +249,23 @@ static int static_scratch_address(unsigned **out)
     return FLEXIQ_OK;
 }
 
+// Launch with programmatic stream serialization allowed (see pdl_wait in the kernels).
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned blocks, unsigned threads, size_t smem, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(blocks, 1, 1);
+    cfg.blockDim = dim3(threads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 template <int DTYPE>
 static int launch_prologue(const Layer *L, const void *X, long long M, float S, int dynamic, uint8_t *X4,
                            long long pitch, int8_t *X8, uint8_t *sx_out, unsigned *scratch, cudaStream_t st)
@@ -256,17 +281,15 @@ static int launch_prologue(const Layer *L, const void *X, long long M, float S, 
         long long blocks = want < (long long)sms * 8 ? want : (long long)sms * 8;
         // thread count must cover at least one full row of chunks
         while (blocks * threads < n_c16) ++blocks;
-        group_or_kernel<DTYPE><<<(unsigned)blocks, threads, sizeof(unsigned) * L->n_g, st>>>(X, M, K, G, S, L->perm, scratch);
-        FLEXIQ_CUDA_TRY(cudaGetLastError());
+        FLEXIQ_CUDA_TRY(launch_pdl(group_or_kernel<DTYPE>, (unsigned)blocks, threads, sizeof(unsigned) * L->n_g, st, X, M, K, G, S, L->perm, scratch));
     }
     long long want = (M * n_c16 + threads - 1) / threads;
     long long blocks = want < (long long)sms * 16 ? want : (long long)sms * 16;
     const uint8_t *sx = dynamic ? nullptr : L->sx;
     if (L->lowbit_path == FLEXIQ_LOWBIT_PACKED_U4)
-        quantize_lower_kernel<DTYPE, 1><<<(unsigned)blocks, threads, 0, st>>>(X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, dynamic ? sx_out : nullptr);
+        FLEXIQ_CUDA_TRY(launch_pdl(quantize_lower_kernel<DTYPE, 1>, (unsigned)blocks, threads, 0, st, X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, dynamic ? sx_out : nullptr));
     else
-        quantize_lower_kernel<DTYPE, 0><<<(unsigned)blocks, threads, 0, st>>>(X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, dynamic ? sx_out : nullptr);
-    FLEXIQ_CUDA_TRY(cudaGetLastError());
+        FLEXIQ_CUDA_TRY(launch_pdl(quantize_lower_kernel<DTYPE, 0>, (unsigned)blocks, threads, 0, st, X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, dynamic ? sx_out : nullptr));
     return FLEXIQ_OK;
 }
 

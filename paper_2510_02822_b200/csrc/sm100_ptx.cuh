@@ -12,6 +12,20 @@ __device__ __forceinline__ uint32_t smem_u32(const void *p)
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization
+// attribute may start while its predecessor in the stream still runs; it must not touch
+// memory the predecessor writes (or reads, if it overwrites it) before pdl_wait() returns.
+// pdl_launch_dependents() lets the successor start its own preamble.  Both are no-ops for
+// a plain launch.
+__device__ __forceinline__ void pdl_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // One lane of a converged warp (the same one every time while the warp stays converged).
 // Issuing TMA / MMA instructions under this predicate, with the whole warp walking the loop,
 // lets the compiler keep their operands in uniform registers.
