@@ -35,14 +35,15 @@ __device__ long long g_prof[16];
 #endif
 
 constexpr int BM = 128;
-constexpr int kNumEpiWarps = 16;                      // four per TMEM lane quadrant
-constexpr int kThreads = 32 * (2 + kNumEpiWarps);
+constexpr int kNumWorkWarps = 16;                     // epilogue warps (+ expander warps on the packed path)
+constexpr int kThreads = 32 * (2 + kNumWorkWarps);
+constexpr int kRawStages = 2;                         // packed path: ring of raw 4-bit tiles in front of the operand ring
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr int kABytes = BM * 128;                     // A stage (BK <= 128 bytes per row)
 constexpr int kStageRegion = 196608;                  // shared memory given to the operand ring
 constexpr int kFactorsPerWarp = 512;                  // alpha[64] | beta[64] of the warp's columns in the current tile
 constexpr int kMaxStages = 8;
-constexpr int kSmemBytes = kStageRegion + kNumEpiWarps * kFactorsPerWarp + 256;
+constexpr int kSmemBytes = kStageRegion + kNumWorkWarps * kFactorsPerWarp + 256;
 
 struct GemmParams {
     long long M;         // rows of the implicit GEMM (tokens or output pixels)
@@ -61,6 +62,10 @@ struct GemmParams {
     const float *beta;   // [N] per-output-channel addend of this call
     void *Y;
     int m_tiles, n_tiles;
+    // packed low-bit path only: positions the expander warps shift the 4-bit values back to
+    const uint8_t *sx;   // [n_g] activation positions, slab order
+    const uint8_t *sw;   // [n_g][N] weight positions
+    int G;               // channel-group size
 };
 
 // Bounded wait.  Returns false after the limit or when another role already gave up;
@@ -158,16 +163,37 @@ __device__ __forceinline__ void st_global_256(void *p, const uint32_t *w)
                  ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
 }
 
+// Eight packed bytes (16 two's-complement nibbles, channel 2t in bits 0-3 of byte t) -> 16 int8
+// values (nibble << s), as four little-endian words.  Nibbles are spread to bytes with two
+// byte permutes per word; the sign extension ORs in bits s+4..7 where bit 3 of the nibble is set.
+__device__ __forceinline__ void unpack16(uint32_t w0, uint32_t w1, int s, uint32_t out[4])
+{
+    const uint32_t k = (16u >> s) - 1u;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const uint32_t w = h == 0 ? w0 : w1;
+        const uint32_t e = w & 0x0f0f0f0fu, o = (w >> 4) & 0x0f0f0f0fu;  // even / odd nibbles, one per byte
+        const uint32_t x[2] = {__byte_perm(e, o, 0x5140), __byte_perm(e, o, 0x7362)};  // channel order
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const uint32_t fill = (((x[q] & 0x08080808u) << (s + 1)) & 0xf0f0f0f0u) * k;
+            out[2 * h + q] = (x[q] << s) | fill;
+        }
+    }
+}
+
 struct EpilogueCtx {
     uint32_t tmem_base, buf_stride, cta_rank;
     uint64_t *tmem_full, *tmem_empty;
     volatile int *abort_flag;
     float *fac;
     int first_tile, tile_step, num_tiles;
+    int parts, arrivals_on;  // column parts per tile (4 or 2); this warp arrives on the accumulator barrier
 };
 
 // One epilogue warp: TMEM lane quadrant `quad` (32 rows, lane = row), column quarter `part`
-// (BN/4 = 16..64 columns) of every tile of this CTA.  Per tile: fetch the columns' factors,
+// (BN/4 = 16..64 columns per pass; two passes when only eight warps drain the tile) of every
+// tile of this CTA.  Per pass: fetch the columns' factors,
 // read the whole slice of the accumulator into registers, hand the accumulator back, then
 // scale / round / clip and store each row's bytes straight to global memory.
 template <int CG, int MODE>
@@ -185,64 +211,74 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
     uint32_t buf_phase = 0;
     PROF_DECL(prof_wait);
     PROF_T0(prof_start);
+    const int passes = 4 / x.parts;              // 1 with sixteen epilogue warps, 2 with eight
     TileWalk tw;
     for (tw.init(x.first_tile, x.tile_step, x.num_tiles, p.n_tiles); tw.left > 0; tw.next()) {
-        const int nw = tw.n_blk * BN + part * cols;  // first output channel of this warp
         const long long row = ((long long)tw.m_blk * CG + x.cta_rank) * BM + quad * 32 + lane;
-        float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (kScaled && nw + 4 * (lane & 15) < p.N) f = __ldg(reinterpret_cast<const float4 *>(fsrc + nw));
-        PROF_T0(t0);
-        const bool ok = wait_bounded(&x.tmem_full[buf], buf_phase, x.abort_flag, 4);
-        PROF_ADD(prof_wait, t0);
-        if (!__all_sync(0xffffffffu, ok)) break;
-        ptx::tc_fence_after_sync();
-        const uint32_t taddr = x.tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)buf * x.buf_stride + (uint32_t)(part * cols);
-        uint32_t ra[32], rb[32];
-        if (cols >= 32) ptx::tmem_ld_32x32(taddr, ra); else ptx::tmem_ld_32x16(taddr, ra);
-        if (cols == 64) ptx::tmem_ld_32x32(taddr + 32, rb); else if (cols == 48) ptx::tmem_ld_32x16(taddr + 32, rb);
-        if (kScaled) {
-            __syncwarp();                                      // the previous tile's reads of the table are done
-            reinterpret_cast<float4 *>(x.fac)[lane] = f;
-            __syncwarp();
-        }
-        ptx::tmem_ld_wait();
-        // the accumulator slice is in registers: hand it back to the MMA warp before the math
-        ptx::tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) {
-            if (CG == 2) ptx::mbar_arrive_cluster_relaxed(ptx::mapa(ptx::smem_u32(&x.tmem_empty[buf]), 0));
-            else ptx::mbar_arrive_relaxed(&x.tmem_empty[buf]);
-        }
-        if (row < p.M) {
-            uint8_t *yrow = static_cast<uint8_t *>(p.Y) + (row * p.N + nw) * kElem;
+        bool waited = false;
+        for (int pass = 0; pass < passes; ++pass) {
+            const int col0 = (part * passes + pass) * cols;  // first tile column of this warp in this pass
+            const int nw = tw.n_blk * BN + col0;             // ... as an output channel
+            float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (kScaled && nw + 4 * (lane & 15) < p.N) f = __ldg(reinterpret_cast<const float4 *>(fsrc + nw));
+            if (!waited) {
+                PROF_T0(t0);
+                const bool ok = wait_bounded(&x.tmem_full[buf], buf_phase, x.abort_flag, 4);
+                PROF_ADD(prof_wait, t0);
+                if (!__all_sync(0xffffffffu, ok)) return;
+                ptx::tc_fence_after_sync();
+                waited = true;
+            }
+            const uint32_t taddr = x.tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)buf * x.buf_stride + (uint32_t)col0;
+            uint32_t ra[32], rb[32];
+            if (cols >= 32) ptx::tmem_ld_32x32(taddr, ra); else ptx::tmem_ld_32x16(taddr, ra);
+            if (cols == 64) ptx::tmem_ld_32x32(taddr + 32, rb); else if (cols == 48) ptx::tmem_ld_32x16(taddr + 32, rb);
+            if (kScaled) {
+                __syncwarp();                                      // the previous reads of the table are done
+                reinterpret_cast<float4 *>(x.fac)[lane] = f;
+                __syncwarp();
+            }
+            ptx::tmem_ld_wait();
+            if (pass + 1 == passes) {
+                // the accumulator slice is in registers: hand it back to the MMA warp before the math
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) {
+                    if (CG == 2) ptx::mbar_arrive_cluster_relaxed(ptx::mapa(ptx::smem_u32(&x.tmem_empty[buf]), 0));
+                    else ptx::mbar_arrive_relaxed(&x.tmem_empty[buf]);
+                }
+            }
+            if (row < p.M) {
+                uint8_t *yrow = static_cast<uint8_t *>(p.Y) + (row * p.N + nw) * kElem;
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {                       // two halves of 32 columns
-                const uint32_t *r = h == 0 ? ra : rb;
-                const int n = nw + 32 * h;
-                if (32 * h < cols && n < p.N) {
-                    const bool second = 32 * h + 16 < cols && n + 16 < p.N;  // columns 16..31 of this half are live
-                    if (MODE == FLEXIQ_OUT_REQUANT_I8) {
-                        uint32_t w[8];
-                        finish16<MODE>(r, x.fac + 32 * h, x.fac + 64 + 32 * h, w);
-                        if (second) finish16<MODE>(r + 16, x.fac + 32 * h + 16, x.fac + 64 + 32 * h + 16, w + 4);
-                        if (second && wide && ((nw & 31) == 0)) st_global_256(yrow + 32 * h, w);  // 32-byte aligned only then
-                        else {
-                            st_global_128(yrow + 32 * h, w[0], w[1], w[2], w[3]);
-                            if (second) st_global_128(yrow + 32 * h + 16, w[4], w[5], w[6], w[7]);
-                        }
-                    } else {
+                for (int h = 0; h < 2; ++h) {                       // two halves of 32 columns
+                    const uint32_t *r = h == 0 ? ra : rb;
+                    const int n = nw + 32 * h;
+                    if (32 * h < cols && n < p.N) {
+                        const bool second = 32 * h + 16 < cols && n + 16 < p.N;  // columns 16..31 of this half are live
+                        if (MODE == FLEXIQ_OUT_REQUANT_I8) {
+                            uint32_t w[8];
+                            finish16<MODE>(r, x.fac + 32 * h, x.fac + 64 + 32 * h, w);
+                            if (second) finish16<MODE>(r + 16, x.fac + 32 * h + 16, x.fac + 64 + 32 * h + 16, w + 4);
+                            if (second && wide && ((nw & 31) == 0)) st_global_256(yrow + 32 * h, w);  // 32-byte aligned only then
+                            else {
+                                st_global_128(yrow + 32 * h, w[0], w[1], w[2], w[3]);
+                                if (second) st_global_128(yrow + 32 * h + 16, w[4], w[5], w[6], w[7]);
+                            }
+                        } else {
 #pragma unroll
-                        for (int g = 0; g < 2; ++g) {
-                            if (g == 0 || second) {
-                                uint32_t w[16];
-                                finish16<MODE>(r + 16 * g, x.fac + 32 * h + 16 * g, x.fac + 64 + 32 * h + 16 * g, w);
-                                uint8_t *dst = yrow + (32 * h + 16 * g) * 4;
-                                if (y32) {                      // rows of 4-byte elements with N % 16 == 0 are 64-byte aligned
-                                    st_global_256(dst, w);
-                                    st_global_256(dst + 32, w + 8);
-                                } else {
+                            for (int g = 0; g < 2; ++g) {
+                                if (g == 0 || second) {
+                                    uint32_t w[16];
+                                    finish16<MODE>(r + 16 * g, x.fac + 32 * h + 16 * g, x.fac + 64 + 32 * h + 16 * g, w);
+                                    uint8_t *dst = yrow + (32 * h + 16 * g) * 4;
+                                    if (y32) {                      // rows of 4-byte elements with N % 16 == 0 are 64-byte aligned
+                                        st_global_256(dst, w);
+                                        st_global_256(dst + 32, w + 8);
+                                    } else {
 #pragma unroll
-                                    for (int q = 0; q < 4; ++q) st_global_128(dst + 16 * q, w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+                                        for (int q = 0; q < 4; ++q) st_global_128(dst + 16 * q, w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+                                    }
                                 }
                             }
                         }
@@ -259,7 +295,9 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
 // each CTA loads its own 128 rows of A and its own half of B (no multicast), the leader
 // CTA issues cta_group::2 MMAs that read both halves, and each CTA drains the 128
 // accumulator rows held in its own TMEM.  Operand traffic from L2 per MAC drops by a third.
-template <int CG>
+// PK = 1 (single CTA only): the low slab arrives as packed 4-bit tiles; eight expander warps
+// widen them into the operand ring (eight epilogue warps remain).
+template <int CG, int PK>
 __global__ void __launch_bounds__(kThreads, 1)
 mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_constant__ CUtensorMap mapA_hi,
                   const __grid_constant__ CUtensorMap mapB_lo, const __grid_constant__ CUtensorMap mapB_hi,
@@ -272,11 +310,15 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
     }
     uint8_t *stage_base = smem;
     uint8_t *factors = smem + kStageRegion;
-    uint64_t *full_bar = reinterpret_cast<uint64_t *>(factors + kNumEpiWarps * kFactorsPerWarp);
+    uint64_t *full_bar = reinterpret_cast<uint64_t *>(factors + kNumWorkWarps * kFactorsPerWarp);
     uint64_t *empty_bar = full_bar + kMaxStages;
     uint64_t *tmem_full = empty_bar + kMaxStages;
     uint64_t *tmem_empty = tmem_full + 2;
-    uint32_t *tmem_ptr_s = reinterpret_cast<uint32_t *>(tmem_empty + 2);
+    uint64_t *raw_full = tmem_empty + 2;
+    uint64_t *raw_empty = raw_full + kRawStages;
+    uint32_t *tmem_ptr_s = reinterpret_cast<uint32_t *>(raw_empty + kRawStages);
+    constexpr int kEpiWarps = PK ? 8 : 16;
+    constexpr int kExpWarps = PK ? 8 : 0;
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_ptr_s + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -292,12 +334,16 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            ptx::mbar_init(&full_bar[s], 1);
+            ptx::mbar_init(&full_bar[s], PK ? kExpWarps : 1);  // packed path: every fill counts eight arrivals
             ptx::mbar_init(&empty_bar[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(&tmem_full[b], 1);
-            ptx::mbar_init(&tmem_empty[b], CG * kNumEpiWarps);
+            ptx::mbar_init(&tmem_empty[b], CG * kEpiWarps);
+        }
+        for (int r = 0; r < kRawStages; ++r) {
+            ptx::mbar_init(&raw_full[r], 1);
+            ptx::mbar_init(&raw_empty[r], PK ? kExpWarps : 1);
         }
         *abort_flag = 0;
         ptx::fence_mbar_init();
@@ -333,6 +379,9 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
         const uint32_t full0 = ptx::smem_u32(full_bar);
         const uint32_t full0_lead = CG == 2 ? ptx::mapa(full0, 0) : full0;  // transaction bytes go to the leader's barrier
         uint32_t stage = 0, phase = 0;
+        uint32_t rstage = 0, rphase = 0;                       // packed path: ring of raw 4-bit tiles
+        const uint32_t raw0 = stage0 + (uint32_t)(p.stages * stage_bytes);
+        const uint32_t raw_bytes = (uint32_t)((BM + BN) * (p.BK / 2));
         long long issued = 0;
         bool ok = true;
         PROF_DECL(prof_wait);
@@ -361,12 +410,35 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                 for (int tap = 0; tap < p.T && ok; ++tap) {
                     int xa = 0, xb = xb_tap;
                     for (int cb = 0; cb < nb; ++cb) {
+                        if (PK && part == 0) {
+                            // packed low block: half-size raw tiles for the expander warps; the operand-ring
+                            // stage this block will occupy is only counted here
+                            if (!__all_sync(0xffffffffu, wait_bounded(&raw_empty[rstage], rphase ^ 1, abort_flag, 5))) { ok = false; break; }
+                            if (ptx::elect_one()) {
+                                const uint32_t ra = raw0 + rstage * raw_bytes;
+                                const uint32_t bar = ptx::smem_u32(&raw_full[rstage]);
+                                ptx::mbar_expect_tx_s(bar, raw_bytes);
+                                if (p.im2col)
+                                    ptx::tma_load_im2col_4d_s<1>(ra, ma, bar, xa >> 1, pix_w, pix_h, pix_n, (uint16_t)tap_s, (uint16_t)tap_r);
+                                else
+                                    ptx::tma_load_2d_s<1>(ra, ma, bar, xa >> 1, (int)m0);
+                                ptx::tma_load_2d_s<1>(ra + BM * (p.BK / 2), mb, bar, xb >> 1, n0);
+                            }
+                            __syncwarp();
+                            if (++rstage == kRawStages) { rstage = 0; rphase ^= 1; }
+                            xa += p.BK;
+                            xb += p.BK;
+                            ++issued;
+                            if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
+                            continue;
+                        }
                         PROF_T0(t0);
                         if (!__all_sync(0xffffffffu, wait_bounded(empty0 + 8 * stage, phase ^ 1, abort_flag, 1))) { ok = false; break; }
                         PROF_ADD(prof_wait, t0);
                         if (ptx::elect_one()) {
                             const uint32_t sa = stage0 + stage * stage_bytes;
                             if (leader) ptx::mbar_expect_tx_s(full0 + 8 * stage, tx_bytes);
+                            if (PK) ptx::mbar_arrive_count(&full_bar[stage], PK ? kExpWarps - 1 : 0);  // stand in for the expander warps
                             const uint32_t bar = full0_lead + 8 * stage;
                             if (p.im2col)
                                 ptx::tma_load_im2col_4d_s<CG>(sa, ma, bar, xa, pix_w, pix_h, pix_n, (uint16_t)tap_s, (uint16_t)tap_r);
@@ -472,18 +544,81 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             PROF_STORE(6, clock64() - prof_start);
         }
     } else {
-        // ------------------------------------------------------------- epilogue
-        // warp e owns TMEM lane quadrant (warp & 3) and one quarter of the tile's columns;
-        // the warps do not synchronise with one another.
-        const int e = warp - 2;
-        EpilogueCtx x;
-        x.tmem_base = tmem_base; x.buf_stride = buf_stride; x.cta_rank = cta_rank;
-        x.tmem_full = tmem_full; x.tmem_empty = tmem_empty; x.abort_flag = abort_flag;
-        x.fac = reinterpret_cast<float *>(factors + e * kFactorsPerWarp);  // alpha[64] | beta[64]
-        x.first_tile = first_tile; x.tile_step = tile_step; x.num_tiles = num_tiles;
-        if (p.out_mode == FLEXIQ_OUT_REQUANT_I8) epilogue_role<CG, FLEXIQ_OUT_REQUANT_I8>(p, x, warp & 3, e >> 2, lane);
-        else if (p.out_mode == FLEXIQ_OUT_DEQUANT_F32) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_F32>(p, x, warp & 3, e >> 2, lane);
-        else epilogue_role<CG, FLEXIQ_OUT_ACC_I32>(p, x, warp & 3, e >> 2, lane);
+        if (warp < 2 + kEpiWarps) {
+            // --------------------------------------------------------- epilogue
+            // warp e owns TMEM lane quadrant (warp & 3) and one column part of the tile;
+            // the warps do not synchronise with one another.
+            const int e = warp - 2;
+            EpilogueCtx x;
+            x.tmem_base = tmem_base; x.buf_stride = buf_stride; x.cta_rank = cta_rank;
+            x.tmem_full = tmem_full; x.tmem_empty = tmem_empty; x.abort_flag = abort_flag;
+            x.fac = reinterpret_cast<float *>(factors + e * kFactorsPerWarp);  // alpha[64] | beta[64]
+            x.first_tile = first_tile; x.tile_step = tile_step; x.num_tiles = num_tiles;
+            x.parts = kEpiWarps / 4; x.arrivals_on = 1;
+            if (p.out_mode == FLEXIQ_OUT_REQUANT_I8) epilogue_role<CG, FLEXIQ_OUT_REQUANT_I8>(p, x, warp & 3, e >> 2, lane);
+            else if (p.out_mode == FLEXIQ_OUT_DEQUANT_F32) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_F32>(p, x, warp & 3, e >> 2, lane);
+            else epilogue_role<CG, FLEXIQ_OUT_ACC_I32>(p, x, warp & 3, e >> 2, lane);
+        } else if (PK) {
+            // --------------------------------------------------------- expanders (packed path)
+            // Widen each raw 4-bit tile into the operand ring: 8 packed bytes -> one 16-byte unit
+            // (nibble << position) at its swizzled place, activations shifted by sx[group], weights
+            // by sw[group][n].  Walks the same K blocks as the producer and the MMA warp.
+            const int tid_e = (warp - 2 - kEpiWarps) * 32 + lane;
+            constexpr int kExpThreads = kExpWarps * 32;
+            const int upr = p.BK >> 4;                    // 16-byte units per operand row: 8 or 4
+            const int half = p.BK >> 1;                   // raw bytes per row
+            const int cpg = p.G >> 4;                     // 16-channel chunks per group
+            uint8_t *raw_base = stage_base + p.stages * stage_bytes;
+            const int raw_bytes = (BM + BN) * half;
+            uint32_t stage = 0, phase = 0, rstage = 0, rphase = 0;
+            bool ok = true;
+            TileWalk tw;
+            for (tw.init(first_tile, tile_step, num_tiles, p.n_tiles); tw.left > 0 && ok; tw.next()) {
+                const int n0 = tw.n_blk * BN;
+                for (int part = 0; part < 2 && ok; ++part) {
+                    const int nb = part ? p.nb_hi : p.nb_lo;
+                    for (int tap = 0; tap < p.T && ok; ++tap) {
+                        for (int cb = 0; cb < nb; ++cb) {
+                            if (part == 0) {
+                                bool w1 = wait_bounded(&raw_full[rstage], rphase, abort_flag, 6);
+                                w1 = w1 && wait_bounded(&empty_bar[stage], phase ^ 1, abort_flag, 7);
+                                if (!__all_sync(0xffffffffu, w1)) { ok = false; break; }
+                                const uint8_t *rawA = raw_base + rstage * raw_bytes;
+                                const uint8_t *rawB = rawA + BM * half;
+                                uint8_t *dstA = stage_base + stage * stage_bytes;
+                                uint8_t *dstB = dstA + kABytes;
+                                const int total = (BM + BN) * upr;
+                                for (int idx = tid_e; idx < total; idx += kExpThreads) {
+                                    const bool isB = idx >= BM * upr;
+                                    const int i2 = isB ? idx - BM * upr : idx;
+                                    const int row = i2 / upr, u = i2 - row * upr;
+                                    const int chunk = cb * upr + u;          // 16-channel chunk of the low slab
+                                    int sh = 0;
+                                    if (chunk * 16 < p.C_lo) {
+                                        const int j = chunk / cpg;
+                                        if (!isB) sh = p.sx[j];
+                                        else if (n0 + row < p.N) sh = p.sw[(size_t)j * p.N + n0 + row];
+                                    }
+                                    const uint2 v = *reinterpret_cast<const uint2 *>((isB ? rawB : rawA) + row * half + u * 8);
+                                    uint32_t o[4];
+                                    unpack16(v.x, v.y, sh, o);
+                                    const int us = upr == 8 ? (u ^ (row & 7)) : (u ^ ((row >> 1) & 3));  // 128- / 64-byte swizzle
+                                    *reinterpret_cast<uint4 *>((isB ? dstB : dstA) + row * p.BK + us * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+                                }
+                                ptx::fence_proxy_async_smem();  // generic-proxy writes become visible to the MMA's reads
+                                __syncwarp();
+                                if (lane == 0) {
+                                    ptx::mbar_arrive(&full_bar[stage]);
+                                    ptx::mbar_arrive(&raw_empty[rstage]);
+                                }
+                                if (++rstage == kRawStages) { rstage = 0; rphase ^= 1; }
+                            }
+                            if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
+                        }
+                    }
+                }
+            }
+        }
     }
 
     ptx::tc_fence_before_sync();
@@ -545,7 +680,7 @@ static TileChoice choose_tile(long long M, int N, int k_blocks, int sms)
 }
 
 static int make_map_im2col(CUtensorMap *map, const void *base, int Cpart, long long pitch, int Nb, int H, int W,
-                           int R, int S, int stride, int pad, int bk)
+                           int R, int S, int stride, int pad, int bk, int swizzle_bytes)
 {
     EncodeIm2colFn enc = get_encode_im2col();
     if (!enc) return set_error(FLEXIQ_ERR_CUDA, "cuTensorMapEncodeIm2col is not available from the driver");
@@ -558,14 +693,14 @@ static int make_map_im2col(CUtensorMap *map, const void *base, int Cpart, long l
     cuuint32_t estr[4] = {1, (cuuint32_t)stride, (cuuint32_t)stride, 1};
     CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(base), dims, strides, lower, upper,
                      (cuuint32_t)bk, (cuuint32_t)BM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                     bk == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                     swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE),
                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS)
         return set_error(FLEXIQ_ERR_CUDA, "cuTensorMapEncodeIm2col failed with CUresult %d", (int)r);
     return FLEXIQ_OK;
 }
 
-template <int CG>
+template <int CG, int PK>
 static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const CUtensorMap &b_lo, const CUtensorMap &b_hi,
                          const GemmParams &p, int sms, cudaStream_t st)
 {
@@ -573,7 +708,7 @@ static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 64 && !attr_set[dev]) {
-        FLEXIQ_CUDA_TRY(cudaFuncSetAttribute(mixed_gemm_kernel<CG>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        FLEXIQ_CUDA_TRY(cudaFuncSetAttribute(mixed_gemm_kernel<CG, PK>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
         attr_set[dev] = true;
     }
     const long long tiles = (long long)p.m_tiles * p.n_tiles;
@@ -593,14 +728,13 @@ static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    FLEXIQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, mixed_gemm_kernel<CG>, a_lo, a_hi, b_lo, b_hi, p));
+    FLEXIQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, mixed_gemm_kernel<CG, PK>, a_lo, a_hi, b_lo, b_hi, p));
     return FLEXIQ_OK;
 }
 
 static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_t *x_shift, long long M, int Nb, int H,
                      int W, float x_scale, float y_scale, int out_mode, void *Y, cudaStream_t st)
 {
-    (void)x_shift;
     if (out_mode < FLEXIQ_OUT_ACC_I32 || out_mode > FLEXIQ_OUT_DEQUANT_F32)
         return set_error(FLEXIQ_ERR_INVALID_ARG, "unknown out_mode %d", out_mode);
     if (out_mode == FLEXIQ_OUT_REQUANT_I8 && !(y_scale > 0.0f))
@@ -612,8 +746,9 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     if (C_hi > 0 && !X8) return set_error(FLEXIQ_ERR_INVALID_ARG, "X8_dev is NULL but K_hi = %d", C_hi);
     if ((reinterpret_cast<uintptr_t>(Y) | reinterpret_cast<uintptr_t>(X4) | reinterpret_cast<uintptr_t>(X8)) & 15)
         return set_error(FLEXIQ_ERR_INVALID_ARG, "X4_dev, X8_dev and Y_dev must be 16-byte aligned");
-    if (L->lowbit_path != FLEXIQ_LOWBIT_MASKED_I8)
-        return set_error(FLEXIQ_ERR_UNSUPPORTED, "packed low-bit mainloop is not available in this build");
+    const bool packed = L->lowbit_path == FLEXIQ_LOWBIT_PACKED_U4 && C_lo > 0;
+    if (packed && L->is_conv && (L->C % 32) != 0)
+        return set_error(FLEXIQ_ERR_UNSUPPORTED, "packed low-bit convolution needs Cin %% 32 == 0 (TMA start alignment of the 4-bit weight taps)");
     int rc = check_device_sm100();
     if (rc) return rc;
     int sms = 148;
@@ -633,13 +768,35 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     }
     p.out_mode = out_mode; p.Y = Y;
     p.alpha = L->alpha; p.beta = L->beta;
-    const TileChoice tc = g_forced_tile.cg ? g_forced_tile : choose_tile(M, L->N, p.T * (p.nb_lo + p.nb_hi), sms);
+    TileChoice tc = g_forced_tile.cg ? g_forced_tile : choose_tile(M, L->N, p.T * (p.nb_lo + p.nb_hi), sms);
+    if (packed && tc.cg == 2) {  // the packed path runs single CTAs: re-choose among those
+        tc.cg = 1;
+        if (!g_forced_tile.cg) {
+            const long long mt = (M + BM - 1) / BM;
+            tc.bn = 256;
+            long long best = -1;
+            const int bns[4] = {256, 192, 128, 64};
+            for (int i = 0; i < 4; ++i) {
+                const long long tiles = mt * ((L->N + bns[i] - 1) / bns[i]);
+                const long long cost = ((tiles + sms - 1) / sms) * bns[i];
+                if (best < 0 || cost < best) { best = cost; tc.bn = bns[i]; }
+            }
+        }
+    }
     const int bn = tc.bn, cg = tc.cg;
+    p.sx = x_shift ? x_shift : L->sx;
+    p.sw = L->sw;
+    p.G = L->G;
     p.m_tiles = (int)((M + (long long)BM * cg - 1) / ((long long)BM * cg));
     p.BN = bn;
     p.n_tiles = (L->N + bn - 1) / bn;
     p.stages = kStageRegion / (kABytes + (bn / cg) * 128);
     if (p.stages > kMaxStages) p.stages = kMaxStages;
+    if (packed) {  // room for the ring of raw 4-bit tiles behind the operand ring
+        const int raw = kRawStages * (BM + bn) * (p.BK / 2);
+        p.stages = (kStageRegion - raw) / (kABytes + bn * 128);
+        if (p.stages > kMaxStages) p.stages = kMaxStages;
+    }
     // the per-output-channel factors depend on the call's scales: recomputed (one tiny launch,
     // stream-ordered before the GEMM) only when they differ from the previous call's
     if (out_mode != FLEXIQ_OUT_ACC_I32 &&
@@ -653,20 +810,24 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     // activation maps (per call: they depend on the caller's buffers, M and the ratio);
     // an empty slab borrows the other one's map and is never addressed
     CUtensorMap a_lo, a_hi;
-    const long long pitch_lo = C_lo;  // masked path: one int8 per value
+    // masked path: one int8 per value; packed path: two values per byte, rows padded to 16 bytes,
+    // raw (unswizzled) tiles of BK/2 bytes per row
+    const long long pitch_lo = packed ? (long long)((C_lo / 2 + 15) / 16) * 16 : (long long)C_lo;
+    const int lo_bytes = packed ? C_lo / 2 : C_lo, lo_box = packed ? p.BK / 2 : p.BK, lo_swz = packed ? 0 : p.BK;
     if (p.im2col) {
-        if (C_lo > 0 && (rc = make_map_im2col(&a_lo, X4, C_lo, pitch_lo, Nb, H, W, L->R, L->S, L->stride, L->pad, p.BK))) return rc;
-        if (C_hi > 0 && (rc = make_map_im2col(&a_hi, X8, C_hi, C_hi, Nb, H, W, L->R, L->S, L->stride, L->pad, p.BK))) return rc;
+        if (C_lo > 0 && (rc = make_map_im2col(&a_lo, X4, lo_bytes, pitch_lo, Nb, H, W, L->R, L->S, L->stride, L->pad, lo_box, lo_swz))) return rc;
+        if (C_hi > 0 && (rc = make_map_im2col(&a_hi, X8, C_hi, C_hi, Nb, H, W, L->R, L->S, L->stride, L->pad, p.BK, p.BK))) return rc;
     } else {
         const long long rows = L->is_conv ? (long long)Nb * H * W : M;
-        if (C_lo > 0 && (rc = make_map_2d(&a_lo, X4, (uint64_t)C_lo, (uint64_t)rows, (uint64_t)pitch_lo, p.BK, BM, p.BK))) return rc;
+        if (C_lo > 0 && (rc = make_map_2d(&a_lo, X4, (uint64_t)lo_bytes, (uint64_t)rows, (uint64_t)pitch_lo, lo_box, BM, lo_swz))) return rc;
         if (C_hi > 0 && (rc = make_map_2d(&a_hi, X8, (uint64_t)C_hi, (uint64_t)rows, (uint64_t)C_hi, p.BK, BM, p.BK))) return rc;
     }
     if (C_lo == 0) a_lo = a_hi;
     if (C_hi == 0) a_hi = a_lo;
     const int bi = weight_map_index(bn / cg);  // box rows = the B rows one CTA loads
-    if (cg == 2) return launch_kernel<2>(a_lo, a_hi, L->map_w8m[bi], L->map_w8[bi], p, sms, st);
-    return launch_kernel<1>(a_lo, a_hi, L->map_w8m[bi], L->map_w8[bi], p, sms, st);
+    if (packed) return launch_kernel<1, 1>(a_lo, a_hi, L->map_w4[bi], L->map_w8[bi], p, sms, st);
+    if (cg == 2) return launch_kernel<2, 0>(a_lo, a_hi, L->map_w8m[bi], L->map_w8[bi], p, sms, st);
+    return launch_kernel<1, 0>(a_lo, a_hi, L->map_w8m[bi], L->map_w8[bi], p, sms, st);
 }
 
 }  // namespace flexiq

@@ -210,9 +210,9 @@ def test_every_tile_shape(dev, cg, bn):
 
 
 # ---------------------------------------------------------------- convolution
-def _run_conv(case, dev, ratios, shifts=None):
+def _run_conv(case, dev, ratios, shifts=None, path=fx.LOWBIT_MASKED_I8):
     perm, sxg, sxs, sw = helpers.prepare_conv(case, shifts)
-    L = _layer(case, dev, perm, sxg, conv=True)
+    L = _layer(case, dev, perm, sxg, conv=True, path=path)
     X = torch.from_numpy(case.X).to(dev)
     q = oracle.quantize(case.X, case.x_scale)
     for r in ratios:
@@ -237,6 +237,31 @@ def test_resnet50_conv_full_size_56(dev):
     # full-size 3x3 C=64 @56x56 at batch 4 (the bench runs batch 32; rows are independent)
     case = inputs.resnet_conv("c56", 4, 56, 64, 64, 3, seed=3000)
     _run_conv(case, dev, [0.0, 0.5, 1.0])
+
+
+# ---------------------------------------------------------------- packed 4-bit slabs
+@pytest.mark.parametrize("M,K,N,G", [(300, 384, 272, 16), (129, 256, 48, 32), (1000, 1024, 400, 16), (257, 64, 64, 16),
+                                     (700, 192, 512, 64)])
+def test_packed_path_linear(dev, M, K, N, G):
+    case = inputs.ranged_linear("pk", M, K, N, G, seed=M + N, group_structured=True)
+    rng = np.random.default_rng(M + K)
+    shifts = rng.integers(0, 5, K // G).astype(np.uint8)
+    _run_linear(case, dev, [0.0, 0.25, 0.5, 1.0, 1.0 / (K // G)], shifts=shifts, path=fx.LOWBIT_PACKED_U4)
+
+
+def test_packed_path_config1_and_dynamic_positions(dev):
+    _run_linear(inputs.config1(), dev, inputs.RATIOS, path=fx.LOWBIT_PACKED_U4)
+    case = inputs.ranged_linear("pkdyn", 333, 384, 96, 16, seed=23, group_structured=True)
+    _run_linear(case, dev, [0.5, 1.0], dynamic=True, path=fx.LOWBIT_PACKED_U4)
+
+
+@pytest.mark.parametrize("Nb,H,C,Cout,R,stride", [(2, 14, 128, 64, 3, 1), (3, 28, 64, 64, 3, 1), (2, 14, 128, 256, 1, 1),
+                                                  (2, 14, 256, 80, 3, 2)])
+def test_packed_path_conv(dev, Nb, H, C, Cout, R, stride):
+    case = inputs.resnet_conv("pkc", Nb, H, C, Cout, R, seed=H + C + 1, stride=stride)
+    rng = np.random.default_rng(H * C + 1)
+    shifts = rng.integers(0, 5, C // case.G).astype(np.uint8)
+    _run_conv(case, dev, [0.25, 0.5, 1.0], shifts=shifts, path=fx.LOWBIT_PACKED_U4)
 
 
 # ---------------------------------------------------------------- full-size, sampled rows
