@@ -38,7 +38,7 @@ constexpr int BM = 128;
 constexpr int kNumWorkWarps = 16;                     // epilogue warps (+ expander warps on the packed path)
 constexpr int kThreads = 32 * (2 + kNumWorkWarps);
 constexpr int kRawStages = 2;                         // packed path: ring of raw 4-bit tiles in front of the operand ring
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint32_t kSpinLimit = 1u << 21;              // parked waits of <= 1 us each: about two seconds at most
 constexpr int kABytes = BM * 128;                     // A stage (BK <= 128 bytes per row)
 constexpr int kStageRegion = 196608;                  // shared memory given to the operand ring
 constexpr int kFactorsPerWarp = 512;                  // alpha[64] | beta[64] of the warp's columns in the current tile
@@ -73,12 +73,13 @@ struct GemmParams {
 // so that the hot loops remain small.
 __device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int where)
 {
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    // a few quick polls for the common short wait, then hardware-parked waits of up to a
+    // microsecond each: they wake at once when the phase completes and issue nothing meanwhile
+    for (uint32_t it = 0; it < 8; ++it)
         if (ptx::mbar_try_wait_s(bar, parity)) return true;
-        if (it > 256) {
-            if (*abort_flag) return false;
-            __nanosleep(it > 8192 ? 256 : 20);
-        }
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (ptx::mbar_try_wait_hint_s(bar, parity, 1000u)) return true;
+        if (*abort_flag) return false;
     }
     *abort_flag = 1;
     atomicMax(&g_status_word, 0x100u + (unsigned)where);
@@ -168,6 +169,10 @@ __device__ __forceinline__ void st_global_256(void *p, const uint32_t *w)
 // byte permutes per word; the sign extension ORs in bits s+4..7 where bit 3 of the nibble is set.
 __device__ __forceinline__ void unpack16(uint32_t w0, uint32_t w1, int s, uint32_t out[4])
 {
+#ifdef EXP_NOUNPACK
+    out[0] = w0; out[1] = w1; out[2] = w0 ^ s; out[3] = w1;
+    return;
+#endif
     const uint32_t k = (16u >> s) - 1u;
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
@@ -562,51 +567,100 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             // --------------------------------------------------------- expanders (packed path)
             // Widen each raw 4-bit tile into the operand ring: 8 packed bytes -> one 16-byte unit
             // (nibble << position) at its swizzled place, activations shifted by sx[group], weights
-            // by sw[group][n].  Walks the same K blocks as the producer and the MMA warp.
+            // by sw[group][n].  Thread t owns weight row t of the tile and half of activation row
+            // t mod 128; its positions for the coming K block are fetched before it waits for the
+            // tile.  Walks the same K blocks as the producer and the MMA warp.
             const int tid_e = (warp - 2 - kEpiWarps) * 32 + lane;
-            constexpr int kExpThreads = kExpWarps * 32;
             const int upr = p.BK >> 4;                    // 16-byte units per operand row: 8 or 4
-            const int half = p.BK >> 1;                   // raw bytes per row
-            const int cpg = p.G >> 4;                     // 16-channel chunks per group
+            const int half = p.BK >> 1;                   // raw bytes per row: 64 or 32
+            const int cpg_log2 = p.G == 16 ? 0 : (p.G == 32 ? 1 : 2);  // 16-channel chunks per group
+            const bool raw_swz = half == 64;              // 64-byte raw rows are stored with the 64-byte swizzle
             uint8_t *raw_base = stage_base + p.stages * stage_bytes;
             const int raw_bytes = (BM + BN) * half;
+            const int rowB = tid_e;                       // BN <= 256 = number of expander threads
+            const bool hasB = rowB < BN;
+            const int rowA = tid_e & (BM - 1);
+            const int uA0 = (tid_e >> 7) * (upr >> 1);    // first activation unit of this thread
             uint32_t stage = 0, phase = 0, rstage = 0, rphase = 0;
             bool ok = true;
+            PROF_DECL(prof_x_raw); PROF_DECL(prof_x_empty); PROF_DECL(prof_x_work); PROF_DECL(prof_x_fence);
+            PROF_T0(prof_x_start);
             TileWalk tw;
             for (tw.init(first_tile, tile_step, num_tiles, p.n_tiles); tw.left > 0 && ok; tw.next()) {
                 const int n0 = tw.n_blk * BN;
+                const bool liveB = hasB && n0 + rowB < p.N;
                 for (int part = 0; part < 2 && ok; ++part) {
                     const int nb = part ? p.nb_hi : p.nb_lo;
                     for (int tap = 0; tap < p.T && ok; ++tap) {
                         for (int cb = 0; cb < nb; ++cb) {
                             if (part == 0) {
+                                int shB[8], shA[4];
+#pragma unroll
+                                for (int u = 0; u < 8; ++u) {
+                                    const int chunk = cb * upr + u;       // 16-channel chunk of the low slab
+#ifdef EXP_NOSHIFT
+                                    shB[u] = chunk & 3;
+#else
+                                    shB[u] = (u < upr && liveB && chunk * 16 < p.C_lo) ? __ldg(p.sw + (size_t)(chunk >> cpg_log2) * p.N + n0 + rowB) : 0;
+#endif
+                                }
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) {
+                                    const int chunk = cb * upr + uA0 + k;
+                                    shA[k] = (k < (upr >> 1) && chunk * 16 < p.C_lo) ? __ldg(p.sx + (chunk >> cpg_log2)) : 0;
+                                }
+                                PROF_T0(tx0);
                                 bool w1 = wait_bounded(&raw_full[rstage], rphase, abort_flag, 6);
+                                PROF_ADD(prof_x_raw, tx0);
+                                PROF_T0(tx1);
                                 w1 = w1 && wait_bounded(&empty_bar[stage], phase ^ 1, abort_flag, 7);
+                                PROF_ADD(prof_x_empty, tx1);
                                 if (!__all_sync(0xffffffffu, w1)) { ok = false; break; }
+                                PROF_T0(tx2);
                                 const uint8_t *rawA = raw_base + rstage * raw_bytes;
                                 const uint8_t *rawB = rawA + BM * half;
                                 uint8_t *dstA = stage_base + stage * stage_bytes;
                                 uint8_t *dstB = dstA + kABytes;
-                                const int total = (BM + BN) * upr;
-                                for (int idx = tid_e; idx < total; idx += kExpThreads) {
-                                    const bool isB = idx >= BM * upr;
-                                    const int i2 = isB ? idx - BM * upr : idx;
-                                    const int row = i2 / upr, u = i2 - row * upr;
-                                    const int chunk = cb * upr + u;          // 16-channel chunk of the low slab
-                                    int sh = 0;
-                                    if (chunk * 16 < p.C_lo) {
-                                        const int j = chunk / cpg;
-                                        if (!isB) sh = p.sx[j];
-                                        else if (n0 + row < p.N) sh = p.sw[(size_t)j * p.N + n0 + row];
+                                if (hasB) {
+                                    const uint8_t *src = rawB + rowB * half;
+                                    uint8_t *dst = dstB + rowB * p.BK;
+                                    const int xr = raw_swz ? ((rowB >> 1) & 3) : 0;
+                                    const int xd = upr == 8 ? (rowB & 7) : ((rowB >> 1) & 3);
+#pragma unroll
+                                    for (int v = 0; v < 4; ++v) {             // 16 raw bytes = two units
+                                        if (2 * v < upr) {
+                                            const uint4 q = *reinterpret_cast<const uint4 *>(src + ((v ^ xr) << 4));
+                                            uint32_t o[4];
+                                            unpack16(q.x, q.y, shB[2 * v], o);
+                                            *reinterpret_cast<uint4 *>(dst + (((2 * v) ^ xd) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                                            unpack16(q.z, q.w, shB[2 * v + 1], o);
+                                            *reinterpret_cast<uint4 *>(dst + (((2 * v + 1) ^ xd) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                                        }
                                     }
-                                    const uint2 v = *reinterpret_cast<const uint2 *>((isB ? rawB : rawA) + row * half + u * 8);
-                                    uint32_t o[4];
-                                    unpack16(v.x, v.y, sh, o);
-                                    const int us = upr == 8 ? (u ^ (row & 7)) : (u ^ ((row >> 1) & 3));  // 128- / 64-byte swizzle
-                                    *reinterpret_cast<uint4 *>((isB ? dstB : dstA) + row * p.BK + us * 16) = make_uint4(o[0], o[1], o[2], o[3]);
                                 }
+                                {
+                                    const uint8_t *src = rawA + rowA * half;
+                                    uint8_t *dst = dstA + rowA * p.BK;
+                                    const int xr = raw_swz ? ((rowA >> 1) & 3) : 0;
+                                    const int xd = upr == 8 ? (rowA & 7) : ((rowA >> 1) & 3);
+#pragma unroll
+                                    for (int k = 0; k < 2; ++k) {             // this thread's half of the row
+                                        if (2 * k < (upr >> 1)) {
+                                            const int v = (uA0 >> 1) + k;
+                                            const uint4 q = *reinterpret_cast<const uint4 *>(src + ((v ^ xr) << 4));
+                                            uint32_t o[4];
+                                            unpack16(q.x, q.y, shA[2 * k], o);
+                                            *reinterpret_cast<uint4 *>(dst + (((2 * v) ^ xd) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                                            unpack16(q.z, q.w, shA[2 * k + 1], o);
+                                            *reinterpret_cast<uint4 *>(dst + (((2 * v + 1) ^ xd) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                                        }
+                                    }
+                                }
+                                PROF_ADD(prof_x_work, tx2);
+                                PROF_T0(tx3);
                                 ptx::fence_proxy_async_smem();  // generic-proxy writes become visible to the MMA's reads
                                 __syncwarp();
+                                PROF_ADD(prof_x_fence, tx3);
                                 if (lane == 0) {
                                     ptx::mbar_arrive(&full_bar[stage]);
                                     ptx::mbar_arrive(&raw_empty[rstage]);
@@ -618,6 +672,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                     }
                 }
             }
+            if (tid_e == 0) { PROF_STORE(10, prof_x_raw); PROF_STORE(11, prof_x_empty); PROF_STORE(12, prof_x_work); PROF_STORE(13, prof_x_fence); PROF_STORE(14, clock64() - prof_x_start); }
         }
     }
 
@@ -813,7 +868,8 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     // masked path: one int8 per value; packed path: two values per byte, rows padded to 16 bytes,
     // raw (unswizzled) tiles of BK/2 bytes per row
     const long long pitch_lo = packed ? (long long)((C_lo / 2 + 15) / 16) * 16 : (long long)C_lo;
-    const int lo_bytes = packed ? C_lo / 2 : C_lo, lo_box = packed ? p.BK / 2 : p.BK, lo_swz = packed ? 0 : p.BK;
+    const int lo_bytes = packed ? C_lo / 2 : C_lo, lo_box = packed ? p.BK / 2 : p.BK;
+    const int lo_swz = packed ? (p.BK / 2 == 64 ? 64 : 0) : p.BK;
     if (p.im2col) {
         if (C_lo > 0 && (rc = make_map_im2col(&a_lo, X4, lo_bytes, pitch_lo, Nb, H, W, L->R, L->S, L->stride, L->pad, lo_box, lo_swz))) return rc;
         if (C_hi > 0 && (rc = make_map_im2col(&a_hi, X8, C_hi, C_hi, Nb, H, W, L->R, L->S, L->stride, L->pad, p.BK, p.BK))) return rc;

@@ -186,7 +186,8 @@ int encode_weight_maps(Layer *L)
         if (rc) return rc;
         rc = make_map_2d(&L->map_w8m[i], L->w8m, (uint64_t)L->Kw, (uint64_t)L->N, (uint64_t)L->Kw, bk, bns[i], bk);
         if (rc) return rc;
-        rc = make_map_2d(&L->map_w4[i], L->w4, (uint64_t)L->Kw / 2, (uint64_t)L->N, (uint64_t)L->w4_pitch, bk / 2, bns[i], 0);
+        rc = make_map_2d(&L->map_w4[i], L->w4, (uint64_t)L->Kw / 2, (uint64_t)L->N, (uint64_t)L->w4_pitch, bk / 2, bns[i],
+                         bk / 2 == 64 ? 64 : 0);  // raw 4-bit tiles: 64-byte rows are read row-per-thread, so they are swizzled
         if (rc) return rc;
     }
     return FLEXIQ_OK;

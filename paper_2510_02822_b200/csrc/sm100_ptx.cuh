@@ -193,6 +193,22 @@ __device__ __forceinline__ bool mbar_try_wait_s(uint32_t bar, uint32_t parity)
         : "memory");
     return ok != 0;
 }
+// try_wait that lets the hardware park the thread for up to `ns` nanoseconds; it resumes at
+// once when the phase completes, so a long wait costs no polling instructions.
+__device__ __forceinline__ bool mbar_try_wait_hint_s(uint32_t bar, uint32_t parity, uint32_t ns)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ void mbar_expect_tx_s(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
