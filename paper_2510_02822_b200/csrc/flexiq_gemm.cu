@@ -169,10 +169,6 @@ __device__ __forceinline__ void st_global_256(void *p, const uint32_t *w)
 // byte permutes per word; the sign extension ORs in bits s+4..7 where bit 3 of the nibble is set.
 __device__ __forceinline__ void unpack16(uint32_t w0, uint32_t w1, int s, uint32_t out[4])
 {
-#ifdef EXP_NOUNPACK
-    out[0] = w0; out[1] = w1; out[2] = w0 ^ s; out[3] = w1;
-    return;
-#endif
     const uint32_t k = (16u >> s) - 1u;
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
@@ -598,11 +594,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
 #pragma unroll
                                 for (int u = 0; u < 8; ++u) {
                                     const int chunk = cb * upr + u;       // 16-channel chunk of the low slab
-#ifdef EXP_NOSHIFT
-                                    shB[u] = chunk & 3;
-#else
                                     shB[u] = (u < upr && liveB && chunk * 16 < p.C_lo) ? __ldg(p.sw + (size_t)(chunk >> cpg_log2) * p.N + n0 + rowB) : 0;
-#endif
                                 }
 #pragma unroll
                                 for (int k = 0; k < 4; ++k) {
