@@ -55,7 +55,10 @@ extern "C" {
  * PACKED : two 4-bit values per byte (half the bytes); the mainloop widens them to the
  *          tensor cores' 8-bit integer operands in shared memory.
  * MASKED : one int8 per value holding the 4-bit value already shifted back to its
- *          extraction position (x4 << sx); the mainloop is a plain 8-bit integer GEMM.
+ *          extraction position (x4 << sx), in ONE slab [M][K] together with the 8-bit groups
+ *          (low groups first); the mainloop is a plain 8-bit integer GEMM over whole K blocks
+ *          against one weight operand that follows the ratio (only the channel groups that
+ *          changed sides are copied, on the stream of the next mixed_* call).
  * Both give bit-identical accumulators. */
 #define FLEXIQ_LOWBIT_MASKED_I8 0
 #define FLEXIQ_LOWBIT_PACKED_U4 1
@@ -103,8 +106,8 @@ int flexiq_layer_set_lowbit_path(flexiq_layer_t layer, int lowbit_path);
 int flexiq_set_lowbit_ratio(flexiq_layer_t layer, float ratio);
 int flexiq_get_max_4bit_ch(flexiq_layer_t layer, int *K_lo);
 
-/* Row pitch in bytes of the low-bit slab for a given K_lo under the layer's path:
- * PACKED: K_lo / 2 rounded up to a multiple of 16;  MASKED: K_lo. */
+/* Row pitch in bytes of the X4_dev slab for a given K_lo under the layer's path:
+ * PACKED: K_lo / 2 rounded up to a multiple of 16;  MASKED: K (the slab holds every group). */
 int flexiq_x4_pitch(flexiq_layer_t layer, int K_lo, int64_t *pitch_bytes);
 
 /* Activation prologue (Sec. 2.1 Eq. 1, Sec. 4.1 bit-lowering, Sec. 5 layout):
@@ -114,9 +117,10 @@ int flexiq_x4_pitch(flexiq_layer_t layer, int K_lo, int64_t *pitch_bytes);
  * with channels gathered into slab order.
  *   X_dev    [M][K] row-major (linear) or NHWC with M = Nb*H*W pixels (conv), x_dtype
  *   X4_dev   [M][pitch] bytes, pitch = flexiq_x4_pitch(K_lo).  PACKED: byte t of a row
- *            holds slab channel 2t in bits 0-3 and 2t+1 in bits 4-7 (two's complement).
- *            MASKED: int8 (x4 << sx[j]).  May be NULL when K_lo == 0.
- *   X8_dev   [M][K_hi] int8.  May be NULL when K_hi == 0.
+ *            holds slab channel 2t in bits 0-3 and 2t+1 in bits 4-7 (two's complement); may
+ *            be NULL when K_lo == 0.  MASKED: the whole slab, int8 [M][K]: (x4 << sx[j]) for
+ *            the low groups, then q for the 8-bit groups; never NULL.
+ *   X8_dev   PACKED: [M][K_hi] int8, may be NULL when K_hi == 0.  MASKED: ignored.
  *   dynamic_pos != 0: the run-time extraction positions of Sec. 4.1 -- a bitwise OR over
  *            all values of a channel group in this call (negatives folded by ~) finds
  *            the highest used bit -- replace the static ones; they are written to
@@ -169,8 +173,10 @@ int flexiq_mixed_gemm(flexiq_layer_t layer, const uint8_t *X4_dev, const int8_t 
 
 /* Mixed-precision convolution as an implicit GEMM (Fig. 4): m = (image, p, q),
  * k = (r, s, c), x[image][p*stride + r - pad][q*stride + s - pad][c], zero outside; the
- * slabs are NHWC with the channel dimension split as in flexiq_quantize_lower
- * (X4_dev [Nb][H][W][pitch], X8_dev [Nb][H][W][C_hi]); Y_dev [Nb][P][Q][Cout]. */
+ * slabs are NHWC with the channel dimension laid out as in flexiq_quantize_lower
+ * (X4_dev [Nb][H][W][pitch], and on the packed path X8_dev [Nb][H][W][C_hi]); Y_dev [Nb][P][Q][Cout].
+ * Calls on one layer handle must be ordered on one stream (the handle's weight operand and
+ * epilogue factors follow the ratio and the scales of the latest call). */
 int flexiq_mixed_conv(flexiq_layer_t layer, const uint8_t *X4_dev, const int8_t *X8_dev,
                       const uint8_t *x_shift_dev, int Nb, int H, int W, float x_scale,
                       float y_scale, int out_mode, void *Y_dev, void *stream);

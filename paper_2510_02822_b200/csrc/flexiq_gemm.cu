@@ -678,6 +678,23 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
     }
 }
 
+// Brings the masked path's weight operand up to date with max_4bit_ch: the channel range
+// [k_from, k_to) of every tap and output channel is copied from `src` (w8m when the range became
+// low-bit, w8 when it returned to 8 bits), 16 bytes per thread.
+__global__ void patch_weights_kernel(int8_t *__restrict__ wf, const int8_t *__restrict__ src, int N, int T, int C,
+                                     int k_from, int k_to)
+{
+    const int upt = (k_to - k_from) >> 4;  // 16-byte units per (n, tap)
+    const long long total = (long long)N * T * upt;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    ptx::pdl_wait();  // the previous kernel of the stream may still read wf
+    if (idx >= total) return;
+    const int u = (int)(idx % upt);
+    const long long nt = idx / upt;  // n * T + tap
+    const size_t off = (size_t)nt * C + k_from + 16 * u;
+    *reinterpret_cast<uint4 *>(wf + off) = *reinterpret_cast<const uint4 *>(src + off);
+}
+
 // Per-output-channel factors of a call: REQUANT alpha = (S_x * S_w[n]) / S_y, beta = bias[n] / S_y;
 // DEQUANT alpha = S_x * S_w[n], beta = bias[n].  Each operation rounds once, in fp32.
 __global__ void scale_vectors_kernel(int N, float x_scale, float y_scale, int requant, const float *__restrict__ w_scale,
@@ -789,9 +806,11 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     if (M == 0) return FLEXIQ_OK;
     const int C_lo = L->K_lo, C_hi = L->C - C_lo;
     if (!Y) return set_error(FLEXIQ_ERR_INVALID_ARG, "Y_dev is NULL");
-    if (C_lo > 0 && !X4) return set_error(FLEXIQ_ERR_INVALID_ARG, "X4_dev is NULL but K_lo = %d", C_lo);
-    if (C_hi > 0 && !X8) return set_error(FLEXIQ_ERR_INVALID_ARG, "X8_dev is NULL but K_hi = %d", C_hi);
-    if ((reinterpret_cast<uintptr_t>(Y) | reinterpret_cast<uintptr_t>(X4) | reinterpret_cast<uintptr_t>(X8)) & 15)
+    const bool packed_path = L->lowbit_path == FLEXIQ_LOWBIT_PACKED_U4;
+    if (!packed_path && !X4) return set_error(FLEXIQ_ERR_INVALID_ARG, "X4_dev is NULL: on the masked path it is the whole slab");
+    if (packed_path && C_lo > 0 && !X4) return set_error(FLEXIQ_ERR_INVALID_ARG, "X4_dev is NULL but K_lo = %d", C_lo);
+    if (packed_path && C_hi > 0 && !X8) return set_error(FLEXIQ_ERR_INVALID_ARG, "X8_dev is NULL but K_hi = %d", C_hi);
+    if ((reinterpret_cast<uintptr_t>(Y) | reinterpret_cast<uintptr_t>(X4) | (packed_path ? reinterpret_cast<uintptr_t>(X8) : 0)) & 15)
         return set_error(FLEXIQ_ERR_INVALID_ARG, "X4_dev, X8_dev and Y_dev must be 16-byte aligned");
     const bool packed = L->lowbit_path == FLEXIQ_LOWBIT_PACKED_U4 && C_lo > 0;
     if (packed && L->is_conv && (L->C % 32) != 0)
@@ -801,12 +820,25 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, L->device);
 
+    if (!packed) {
+        // Masked path: activations are one slab [rows][C] and the weights one operand wf, so the
+        // mainloop is a plain 8-bit GEMM over whole K blocks whatever the ratio.  wf follows the
+        // ratio lazily: only the channel groups that changed sides are copied, in stream order.
+        if (L->wf_K_lo != C_lo) {
+            const int k_from = C_lo < L->wf_K_lo ? C_lo : L->wf_K_lo, k_to = C_lo < L->wf_K_lo ? L->wf_K_lo : C_lo;
+            const long long total = (long long)L->N * L->R * L->S * ((k_to - k_from) >> 4);
+            patch_weights_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(L->wf, C_lo > L->wf_K_lo ? L->w8m : L->w8, L->N,
+                                                                                  L->R * L->S, L->C, k_from, k_to);
+            FLEXIQ_CUDA_TRY(cudaGetLastError());
+            L->wf_K_lo = C_lo;
+        }
+    }
     GemmParams p{};
-    p.M = M; p.N = L->N; p.C = L->C; p.C_lo = C_lo; p.C_hi = C_hi;
+    p.M = M; p.N = L->N; p.C = L->C; p.C_lo = packed ? C_lo : 0; p.C_hi = packed ? C_hi : L->C;
     p.T = L->R * L->S; p.S = L->S;
     p.BK = choose_bk(L);
-    p.nb_lo = (C_lo + p.BK - 1) / p.BK;
-    p.nb_hi = (C_hi + p.BK - 1) / p.BK;
+    p.nb_lo = (p.C_lo + p.BK - 1) / p.BK;
+    p.nb_hi = (p.C_hi + p.BK - 1) / p.BK;
     p.im2col = L->is_conv && (L->R != 1 || L->S != 1 || L->stride != 1 || L->pad != 0);
     p.stride = L->stride; p.pad = L->pad;
     if (L->is_conv) {
@@ -857,25 +889,35 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     // activation maps (per call: they depend on the caller's buffers, M and the ratio);
     // an empty slab borrows the other one's map and is never addressed
     CUtensorMap a_lo, a_hi;
-    // masked path: one int8 per value; packed path: two values per byte, rows padded to 16 bytes,
-    // raw (unswizzled) tiles of BK/2 bytes per row
-    const long long pitch_lo = packed ? (long long)((C_lo / 2 + 15) / 16) * 16 : (long long)C_lo;
-    const int lo_bytes = packed ? C_lo / 2 : C_lo, lo_box = packed ? p.BK / 2 : p.BK;
-    const int lo_swz = packed ? (p.BK / 2 == 64 ? 64 : 0) : p.BK;
-    if (p.im2col) {
-        if (C_lo > 0 && (rc = make_map_im2col(&a_lo, X4, lo_bytes, pitch_lo, Nb, H, W, L->R, L->S, L->stride, L->pad, lo_box, lo_swz))) return rc;
-        if (C_hi > 0 && (rc = make_map_im2col(&a_hi, X8, C_hi, C_hi, Nb, H, W, L->R, L->S, L->stride, L->pad, p.BK, p.BK))) return rc;
+    if (!packed) {
+        // one int8 slab [rows][C] (a packed-path layer at ratio 0 has it in X8_dev)
+        const void *slab = packed_path ? static_cast<const void *>(X8) : static_cast<const void *>(X4);
+        if (p.im2col) {
+            if ((rc = make_map_im2col(&a_hi, slab, L->C, L->C, Nb, H, W, L->R, L->S, L->stride, L->pad, p.BK, p.BK))) return rc;
+        } else {
+            const long long rows = L->is_conv ? (long long)Nb * H * W : M;
+            if ((rc = make_map_2d(&a_hi, slab, (uint64_t)L->C, (uint64_t)rows, (uint64_t)L->C, p.BK, BM, p.BK))) return rc;
+        }
+        a_lo = a_hi;
     } else {
-        const long long rows = L->is_conv ? (long long)Nb * H * W : M;
-        if (C_lo > 0 && (rc = make_map_2d(&a_lo, X4, (uint64_t)lo_bytes, (uint64_t)rows, (uint64_t)pitch_lo, lo_box, BM, lo_swz))) return rc;
-        if (C_hi > 0 && (rc = make_map_2d(&a_hi, X8, (uint64_t)C_hi, (uint64_t)rows, (uint64_t)C_hi, p.BK, BM, p.BK))) return rc;
+        // packed path: two values per byte, rows padded to 16 bytes, raw tiles of BK/2 bytes per row
+        // (64-byte raw rows carry the 64-byte swizzle), plus the int8 slab of the 8-bit groups
+        const long long pitch_lo = (long long)((C_lo / 2 + 15) / 16) * 16;
+        const int lo_box = p.BK / 2, lo_swz = p.BK / 2 == 64 ? 64 : 0;
+        if (p.im2col) {
+            if ((rc = make_map_im2col(&a_lo, X4, C_lo / 2, pitch_lo, Nb, H, W, L->R, L->S, L->stride, L->pad, lo_box, lo_swz))) return rc;
+            if (C_hi > 0 && (rc = make_map_im2col(&a_hi, X8, C_hi, C_hi, Nb, H, W, L->R, L->S, L->stride, L->pad, p.BK, p.BK))) return rc;
+        } else {
+            const long long rows = L->is_conv ? (long long)Nb * H * W : M;
+            if ((rc = make_map_2d(&a_lo, X4, (uint64_t)C_lo / 2, (uint64_t)rows, (uint64_t)pitch_lo, lo_box, BM, lo_swz))) return rc;
+            if (C_hi > 0 && (rc = make_map_2d(&a_hi, X8, (uint64_t)C_hi, (uint64_t)rows, (uint64_t)C_hi, p.BK, BM, p.BK))) return rc;
+        }
+        if (C_hi == 0) a_hi = a_lo;
     }
-    if (C_lo == 0) a_lo = a_hi;
-    if (C_hi == 0) a_hi = a_lo;
     const int bi = weight_map_index(bn / cg);  // box rows = the B rows one CTA loads
     if (packed) return launch_kernel<1, 1>(a_lo, a_hi, L->map_w4[bi], L->map_w8[bi], p, sms, st);
-    if (cg == 2) return launch_kernel<2, 0>(a_lo, a_hi, L->map_w8m[bi], L->map_w8[bi], p, sms, st);
-    return launch_kernel<1, 0>(a_lo, a_hi, L->map_w8m[bi], L->map_w8[bi], p, sms, st);
+    if (cg == 2) return launch_kernel<2, 0>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], p, sms, st);
+    return launch_kernel<1, 0>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], p, sms, st);
 }
 
 }  // namespace flexiq

@@ -38,6 +38,8 @@ struct Layer {
     int8_t *w8;      // [N][Kw] slab-order int8 weights
     int8_t *w8m;     // [N][Kw] (w >> sw) << sw : 4-bit weights at their extraction position
     uint8_t *w4;     // [N][Kw/2] packed 4-bit weights (w >> sw)
+    int8_t *wf;      // [N][Kw] masked path's operand: w8m for the groups below wf_K_lo, w8 for the rest
+    int wf_K_lo;     // the max_4bit_ch that wf currently reflects (patched lazily, in stream order)
     uint8_t *sw;     // [n_g][N] weight extraction positions
     uint8_t *sx;     // [n_g] static activation positions, slab order
     int32_t *perm;   // [n_g]
@@ -47,7 +49,7 @@ struct Layer {
     int32_t *perm_host;
     uint8_t *sx_host;
     // tensor maps over the weights (encoded once)
-    CUtensorMap map_w8[kNumWeightMaps], map_w8m[kNumWeightMaps], map_w4[kNumWeightMaps];  // one per box height
+    CUtensorMap map_w8[kNumWeightMaps], map_w4[kNumWeightMaps], map_wf[kNumWeightMaps];  // one per box height
     // per-output-channel epilogue factors of the most recent call and what they were computed for
     float *alpha, *beta;
     float cache_xs, cache_ys;

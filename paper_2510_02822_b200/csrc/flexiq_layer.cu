@@ -170,7 +170,7 @@ static int validate_common(flexiq_layer_t *out, int C, int N, int G, const int8_
 static void free_layer(Layer *L)
 {
     if (!L) return;
-    cudaFree(L->w8); cudaFree(L->w8m); cudaFree(L->w4); cudaFree(L->sw); cudaFree(L->sx);
+    cudaFree(L->w8); cudaFree(L->w8m); cudaFree(L->w4); cudaFree(L->wf); cudaFree(L->sw); cudaFree(L->sx);
     cudaFree(L->perm); cudaFree(L->w_scale); cudaFree(L->bias); cudaFree(L->alpha); cudaFree(L->beta);
     free(L->perm_host); free(L->sx_host);
     L->magic = 0;
@@ -184,7 +184,7 @@ int encode_weight_maps(Layer *L)
     for (int i = 0; i < kNumWeightMaps; ++i) {
         int rc = make_map_2d(&L->map_w8[i], L->w8, (uint64_t)L->Kw, (uint64_t)L->N, (uint64_t)L->Kw, bk, bns[i], bk);
         if (rc) return rc;
-        rc = make_map_2d(&L->map_w8m[i], L->w8m, (uint64_t)L->Kw, (uint64_t)L->N, (uint64_t)L->Kw, bk, bns[i], bk);
+        rc = make_map_2d(&L->map_wf[i], L->wf, (uint64_t)L->Kw, (uint64_t)L->N, (uint64_t)L->Kw, bk, bns[i], bk);
         if (rc) return rc;
         rc = make_map_2d(&L->map_w4[i], L->w4, (uint64_t)L->Kw / 2, (uint64_t)L->N, (uint64_t)L->w4_pitch, bk / 2, bns[i],
                          bk / 2 == 64 ? 64 : 0);  // raw 4-bit tiles: 64-byte rows are read row-per-thread, so they are swizzled
@@ -232,6 +232,7 @@ static int create_common(flexiq_layer_t *out, int is_conv, int C, int N, int R, 
     } while (0)
     TRY_OR_FREE(cudaMalloc(&L->w8, wbytes));
     TRY_OR_FREE(cudaMalloc(&L->w8m, wbytes));
+    TRY_OR_FREE(cudaMalloc(&L->wf, wbytes));
     TRY_OR_FREE(cudaMalloc(&L->w4, (size_t)N * L->w4_pitch));
     TRY_OR_FREE(cudaMemsetAsync(L->w4, 0, (size_t)N * L->w4_pitch, stream));
     TRY_OR_FREE(cudaMalloc(&L->sw, (size_t)n_g * N));
@@ -251,6 +252,8 @@ static int create_common(flexiq_layer_t *out, int is_conv, int C, int N, int R, 
     prep_weights_kernel<<<(unsigned)((total + threads - 1) / threads), threads, 0, stream>>>(
         Wq, is_conv, C, N, G, R * S, L->perm, L->w8, L->w8m, L->w4, L->w4_pitch, L->sw);
     TRY_OR_FREE(cudaGetLastError());
+    TRY_OR_FREE(cudaMemcpyAsync(L->wf, L->w8, wbytes, cudaMemcpyDeviceToDevice, stream));  // ratio 0: all groups at 8 bits
+    L->wf_K_lo = 0;
     TRY_OR_FREE(cudaStreamSynchronize(stream));
 #undef TRY_OR_FREE
     rc = encode_weight_maps(L);
@@ -329,7 +332,7 @@ int flexiq_x4_pitch(flexiq_layer_t layer, int K_lo, int64_t *pitch_bytes)
     if (!L || !pitch_bytes) return set_error(FLEXIQ_ERR_INVALID_ARG, "bad handle or NULL output");
     if (K_lo < 0 || K_lo > L->C || K_lo % L->G != 0)
         return set_error(FLEXIQ_ERR_INVALID_ARG, "K_lo %d is not a multiple of the group size within [0, %d]", K_lo, L->C);
-    *pitch_bytes = L->lowbit_path == FLEXIQ_LOWBIT_PACKED_U4 ? (int64_t)((K_lo / 2 + 15) / 16) * 16 : (int64_t)K_lo;
+    *pitch_bytes = L->lowbit_path == FLEXIQ_LOWBIT_PACKED_U4 ? (int64_t)((K_lo / 2 + 15) / 16) * 16 : (int64_t)L->C;
     return FLEXIQ_OK;
 }
 

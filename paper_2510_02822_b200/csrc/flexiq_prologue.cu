@@ -180,10 +180,9 @@ template <int DTYPE, int PACKED>
 __global__ void quantize_lower_kernel(const void *__restrict__ X, long long M, int K, int G, int K_lo, float S,
                                       const int32_t *__restrict__ perm, const uint8_t *__restrict__ sx,
                                       const unsigned *__restrict__ or_words, uint8_t *__restrict__ X4,
-                                      long long x4_pitch, int8_t *__restrict__ X8, uint8_t *__restrict__ sx_out)
+                                      long long x4_pitch, int8_t *__restrict__ X8, long long x8_pitch, uint8_t *__restrict__ sx_out)
 {
     const int n_c16 = K / 16, c_per_g = G / 16, lo_c16 = K_lo / 16;
-    const int K_hi = K - K_lo;
     const long long total = M * n_c16;
     const Divider div = make_divider(S);
     ptx::pdl_launch_dependents();
@@ -219,7 +218,7 @@ __global__ void quantize_lower_kernel(const void *__restrict__ X, long long M, i
             }
         } else {
             quantize16<DTYPE>(src, div, -128.f, 127.f, w);
-            *reinterpret_cast<uint4 *>(X8 + m * (long long)K_hi + (size_t)(c16 - lo_c16) * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4 *>(X8 + m * x8_pitch + (size_t)(c16 - lo_c16) * 16) = make_uint4(w[0], w[1], w[2], w[3]);
         }
     }
 }
@@ -268,7 +267,7 @@ static cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned blocks, unsigne
 
 template <int DTYPE>
 static int launch_prologue(const Layer *L, const void *X, long long M, float S, int dynamic, uint8_t *X4,
-                           long long pitch, int8_t *X8, uint8_t *sx_out, unsigned *scratch, cudaStream_t st)
+                           long long pitch, int8_t *X8, long long pitch8, uint8_t *sx_out, unsigned *scratch, cudaStream_t st)
 {
     const int K = L->C, G = L->G;
     const int n_c16 = K / 16;
@@ -287,9 +286,9 @@ static int launch_prologue(const Layer *L, const void *X, long long M, float S, 
     long long blocks = want < (long long)sms * 16 ? want : (long long)sms * 16;
     const uint8_t *sx = dynamic ? nullptr : L->sx;
     if (L->lowbit_path == FLEXIQ_LOWBIT_PACKED_U4)
-        FLEXIQ_CUDA_TRY(launch_pdl(quantize_lower_kernel<DTYPE, 1>, (unsigned)blocks, threads, 0, st, X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, dynamic ? sx_out : nullptr));
+        FLEXIQ_CUDA_TRY(launch_pdl(quantize_lower_kernel<DTYPE, 1>, (unsigned)blocks, threads, 0, st, X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, pitch8, dynamic ? sx_out : nullptr));
     else
-        FLEXIQ_CUDA_TRY(launch_pdl(quantize_lower_kernel<DTYPE, 0>, (unsigned)blocks, threads, 0, st, X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, dynamic ? sx_out : nullptr));
+        FLEXIQ_CUDA_TRY(launch_pdl(quantize_lower_kernel<DTYPE, 0>, (unsigned)blocks, threads, 0, st, X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, pitch8, dynamic ? sx_out : nullptr));
     return FLEXIQ_OK;
 }
 
@@ -311,8 +310,10 @@ extern "C" int flexiq_quantize_lower(flexiq_layer_t layer, const void *X_dev, in
     if (M == 0) return FLEXIQ_OK;
     const int K_lo = L->K_lo, K_hi = L->C - K_lo;
     if (!X_dev) return set_error(FLEXIQ_ERR_INVALID_ARG, "X_dev is NULL");
-    if (K_lo > 0 && !X4_dev) return set_error(FLEXIQ_ERR_INVALID_ARG, "X4_dev is NULL but K_lo = %d", K_lo);
-    if (K_hi > 0 && !X8_dev) return set_error(FLEXIQ_ERR_INVALID_ARG, "X8_dev is NULL but K_hi = %d", K_hi);
+    const bool packed = L->lowbit_path == FLEXIQ_LOWBIT_PACKED_U4;
+    if (!packed && !X4_dev) return set_error(FLEXIQ_ERR_INVALID_ARG, "X4_dev is NULL: on the masked path it is the whole slab [M][K]");
+    if (packed && K_lo > 0 && !X4_dev) return set_error(FLEXIQ_ERR_INVALID_ARG, "X4_dev is NULL but K_lo = %d", K_lo);
+    if (packed && K_hi > 0 && !X8_dev) return set_error(FLEXIQ_ERR_INVALID_ARG, "X8_dev is NULL but K_hi = %d", K_hi);
     if (dynamic_pos && (!x_shift_out_dev || !scratch_dev))
         return set_error(FLEXIQ_ERR_INVALID_ARG, "dynamic_pos needs x_shift_out_dev and scratch_dev");
     if ((reinterpret_cast<uintptr_t>(X_dev) | reinterpret_cast<uintptr_t>(X4_dev) | reinterpret_cast<uintptr_t>(X8_dev)) & 15)
@@ -321,12 +322,15 @@ extern "C" int flexiq_quantize_lower(flexiq_layer_t layer, const void *X_dev, in
     if (rc) return rc;
     int64_t pitch = 0;
     flexiq_x4_pitch(layer, K_lo, &pitch);
+    // masked path: one slab, low groups first, the 8-bit groups behind them in the same rows
+    long long pitch8 = K_hi;
+    if (!packed) { X8_dev = reinterpret_cast<int8_t *>(X4_dev) + K_lo; pitch8 = L->C; }
     cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
     switch (x_dtype) {
-        case FLEXIQ_DTYPE_F32: return launch_prologue<FLEXIQ_DTYPE_F32>(L, X_dev, M, x_scale, dynamic_pos, X4_dev, pitch, X8_dev, x_shift_out_dev, scratch_dev, st);
-        case FLEXIQ_DTYPE_F16: return launch_prologue<FLEXIQ_DTYPE_F16>(L, X_dev, M, x_scale, dynamic_pos, X4_dev, pitch, X8_dev, x_shift_out_dev, scratch_dev, st);
-        case FLEXIQ_DTYPE_BF16: return launch_prologue<FLEXIQ_DTYPE_BF16>(L, X_dev, M, x_scale, dynamic_pos, X4_dev, pitch, X8_dev, x_shift_out_dev, scratch_dev, st);
-        default: return launch_prologue<FLEXIQ_DTYPE_I8>(L, X_dev, M, x_scale, dynamic_pos, X4_dev, pitch, X8_dev, x_shift_out_dev, scratch_dev, st);
+        case FLEXIQ_DTYPE_F32: return launch_prologue<FLEXIQ_DTYPE_F32>(L, X_dev, M, x_scale, dynamic_pos, X4_dev, pitch, X8_dev, pitch8, x_shift_out_dev, scratch_dev, st);
+        case FLEXIQ_DTYPE_F16: return launch_prologue<FLEXIQ_DTYPE_F16>(L, X_dev, M, x_scale, dynamic_pos, X4_dev, pitch, X8_dev, pitch8, x_shift_out_dev, scratch_dev, st);
+        case FLEXIQ_DTYPE_BF16: return launch_prologue<FLEXIQ_DTYPE_BF16>(L, X_dev, M, x_scale, dynamic_pos, X4_dev, pitch, X8_dev, pitch8, x_shift_out_dev, scratch_dev, st);
+        default: return launch_prologue<FLEXIQ_DTYPE_I8>(L, X_dev, M, x_scale, dynamic_pos, X4_dev, pitch, X8_dev, pitch8, x_shift_out_dev, scratch_dev, st);
     }
 }
 

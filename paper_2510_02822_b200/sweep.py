@@ -1,0 +1,181 @@
+"""Ratio sweeps over the benchmark configurations (one GPU).
+
+    python -m paper_2510_02822_b200.sweep --config 2            # ViT-B linears, M = 12608
+    python -m paper_2510_02822_b200.sweep --config 3            # ResNet-50 convolutions, batch 32
+    python -m paper_2510_02822_b200.sweep --config 4 --cold     # DeiT-S small batch, L2 flushed between calls
+    python -m paper_2510_02822_b200.sweep --config 5            # ViT-L stack, ratio switched between passes
+
+Prints one JSON line per (layer, ratio): device time of the prologue and of the mixed kernel
+(CUDA events on the launching stream), TOPS = 2*M*N*K / t and algorithmic GB/s of the mixed kernel.
+Warm numbers come from back-to-back launches; --cold flushes L2 (writes a 256 MB buffer) before
+every timed launch and times each launch on its own.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import time
+
+import numpy as np
+import torch
+
+from . import binding as fx
+from . import calib, inputs
+
+RATIOS = [0.0, 0.25, 0.5, 0.75, 1.0]
+
+
+def _layer_for(case, dev, is_conv, path):
+    qcal = calib.quantize_reference(torch.from_numpy(case.Xcal), case.x_scale)
+    perm, x_shift = calib.static_preparation(qcal, torch.from_numpy(case.Wq), case.G, conv=is_conv)
+    L = fx.Layer(torch.from_numpy(case.Wq).to(dev), torch.from_numpy(case.w_scale).to(dev), torch.from_numpy(case.bias).to(dev),
+                 perm, x_shift, case.G, conv=(case.stride, case.pad) if is_conv else None)
+    L.set_lowbit_path(path)
+    return L
+
+
+def _alg_bytes(case, is_conv, ratio, Mout):
+    K = case.C if is_conv else case.K
+    N = case.Cout if is_conv else case.N
+    taps = case.R * case.S if is_conv else 1
+    n_low = round(ratio * (K // case.G))
+    rho = n_low * case.G / K
+    Min = case.Nb * case.H * case.W if is_conv else case.M
+    return Min * K * (1 - rho / 2) + taps * K * N * (1 - rho / 2) + n_low * N + 8 * N + Mout * N
+
+
+def time_case(case, is_conv, dev, path, iters, cold, flush):
+    L = _layer_for(case, dev, is_conv, path)
+    X = torch.from_numpy(case.X).to(dev)
+    stream = torch.cuda.current_stream()
+    rows = []
+    for r in RATIOS:
+        L.set_lowbit_ratio(r)
+        x4, x8, _ = L.quantize_lower(X, case.x_scale)
+
+        def mixed(Y=None):
+            if is_conv:
+                return L.mixed_conv(x4, x8, case.Nb, case.H, case.W, case.x_scale, case.y_scale, fx.OUT_REQUANT_I8, Y=Y)
+            return L.mixed_gemm(x4, x8, case.M, case.x_scale, case.y_scale, fx.OUT_REQUANT_I8, Y=Y)
+
+        Y = mixed()
+        Mout = Y.numel() // Y.shape[-1]
+        K = case.C if is_conv else case.K
+        ops = 2.0 * Y.numel() * (case.R * case.S * K if is_conv else K)
+        for _ in range(3):
+            L.quantize_lower(X, case.x_scale)
+            mixed(Y)
+        torch.cuda.synchronize()
+        if cold:
+            tp = tg = 0.0
+            for _ in range(iters):
+                e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+                flush.add_(1)
+                e[0].record(stream)
+                L.quantize_lower(X, case.x_scale)
+                e[1].record(stream)
+                flush.add_(1)
+                e[2].record(stream)
+                mixed(Y)
+                e[3].record(stream)
+                torch.cuda.synchronize()
+                tp += e[0].elapsed_time(e[1])
+                tg += e[2].elapsed_time(e[3])
+            tp, tg = tp / iters, tg / iters
+        else:
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            e[0].record(stream)
+            for _ in range(iters):
+                L.quantize_lower(X, case.x_scale)
+            e[1].record(stream)
+            for _ in range(iters):
+                mixed(Y)
+            e[2].record(stream)
+            torch.cuda.synchronize()
+            tp, tg = e[0].elapsed_time(e[1]) / iters, e[1].elapsed_time(e[2]) / iters
+        rows.append({"layer": case.name, "ratio": r, "path": "packed" if path else "masked", "cold": bool(cold),
+                     "prologue_us": round(tp * 1e3, 2), "mixed_us": round(tg * 1e3, 2),
+                     "mixed_tops": round(ops / tg / 1e9, 1), "mixed_alg_gbs": round(_alg_bytes(case, is_conv, r, Mout) / tg / 1e6, 1)})
+        print(json.dumps(rows[-1]), flush=True)
+    fx.flexiq_check_status()
+    L.close()
+    return rows
+
+
+def run_stack(dev, batch, iters):
+    """ViT-L/16 stack of linears: every layer's prologue + mixed GEMM in sequence, the ratio switched
+    between passes with flexiq_set_lowbit_ratio (no re-packing, no re-allocation)."""
+    M = batch * 197
+    layers, meta = [], []
+    t0 = time.time()
+    Xs = {}
+    for blk in range(24):
+        for i, (name, K, N) in enumerate(inputs.VIT_L_LAYERS):
+            c = inputs.vit_linear(f"vitl_b{blk}_{name}", 256, K, N, 16, seed=5000 + blk * 4 + i)  # 256 rows: weights + calibration only
+            perm, xs = calib.static_preparation(calib.quantize_reference(torch.from_numpy(c.Xcal), c.x_scale), torch.from_numpy(c.Wq), 16)
+            L = fx.Layer(torch.from_numpy(c.Wq).to(dev), torch.from_numpy(c.w_scale).to(dev), torch.from_numpy(c.bias).to(dev), perm, xs, 16)
+            layers.append(L)
+            meta.append((K, N, c.x_scale, c.y_scale))
+            if K not in Xs:
+                big = inputs.vit_linear("x", M, K, 16, 16, seed=5900 + K)
+                Xs[K] = torch.from_numpy(big.X).to(dev)
+    slabs = {K: (torch.empty(M * K + 16, dtype=torch.uint8, device=dev), torch.empty(M * K + 16, dtype=torch.int8, device=dev)) for K in Xs}
+    Ys = {N: torch.empty((M, N), dtype=torch.int8, device=dev) for N in {n for _, n, _, _ in meta}}
+    print(json.dumps({"setup_s": round(time.time() - t0, 1), "layers": len(layers), "M": M}), flush=True)
+    ops = sum(2.0 * M * K * N for K, N, _, _ in meta)
+    stream = torch.cuda.current_stream()
+
+    def one_pass():
+        for L, (K, N, xs, ys) in zip(layers, meta):
+            x4, x8 = slabs[K]
+            fx.flexiq_quantize_lower(L.h, Xs[K], fx.DTYPE_F32, M, xs, 0, x4, x8)
+            fx.flexiq_mixed_gemm(L.h, x4, x8, None, M, xs, ys, fx.OUT_REQUANT_I8, Ys[N])
+
+    one_pass()
+    torch.cuda.synchronize()
+    for ratio in (0.0, 0.5, 1.0):
+        t_sw = time.perf_counter()
+        for L in layers:
+            L.set_lowbit_ratio(ratio)
+        switch_us = (time.perf_counter() - t_sw) * 1e6
+        one_pass()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(iters):
+            one_pass()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / iters
+        print(json.dumps({"config": 5, "ratio": ratio, "pass_ms": round(ms, 3), "pass_tops_prologue_plus_gemm": round(ops / ms / 1e9, 1),
+                          "ratio_switch_us_all_96_layers": round(switch_us, 1)}), flush=True)
+    fx.flexiq_check_status()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", type=int, default=2)
+    ap.add_argument("--iters", type=int, default=30)
+    ap.add_argument("--cold", action="store_true")
+    ap.add_argument("--path", default="masked", choices=["masked", "packed"])
+    ap.add_argument("--batch", type=int, default=0)
+    args = ap.parse_args()
+    dev = torch.device("cuda:0")
+    path = fx.LOWBIT_PACKED_U4 if args.path == "packed" else fx.LOWBIT_MASKED_I8
+    flush = torch.zeros(64 * 1024 * 1024, dtype=torch.int32, device=dev) if args.cold else None
+    if args.config == 1:
+        time_case(inputs.config1(), False, dev, path, args.iters, args.cold, flush)
+    elif args.config == 2:
+        for c in inputs.config2(args.batch or 64):
+            time_case(c, False, dev, path, args.iters, args.cold, flush)
+    elif args.config == 3:
+        for c in inputs.config3(args.batch or 32):
+            time_case(c, True, dev, path, args.iters, args.cold, flush)
+    elif args.config == 4:
+        for c in inputs.config4(args.batch or 1):
+            time_case(c, False, dev, path, args.iters, args.cold, flush)
+    elif args.config == 5:
+        run_stack(dev, args.batch or 128, max(1, args.iters // 10))
+
+
+if __name__ == "__main__":
+    main()

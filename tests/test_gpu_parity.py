@@ -65,15 +65,20 @@ def _run_linear(case, dev, ratios, shifts=None, x_dtype=torch.float32, path=fx.L
             sx_use = oracle.dynamic_positions(q, case.G, perm)
             assert np.array_equal(shifts_dev.cpu().numpy(), sx_use)
         e4, e8 = oracle.make_slabs(q, case.G, perm, sx_use, nl)
-        if K_lo:
-            pitch = fx.flexiq_x4_pitch(L.h, K_lo)
-            g4 = x4[:case.M * pitch].view(case.M, pitch).cpu().numpy()
-            if path == fx.LOWBIT_MASKED_I8:
-                assert np.array_equal(g4.view(np.int8), helpers.masked_slab(e4, case.G, sx_use, nl))
-            else:
+        pitch = fx.flexiq_x4_pitch(L.h, K_lo)
+        if path == fx.LOWBIT_MASKED_I8:
+            # one slab [M][K]: the low groups as (x4 << sx), then the 8-bit groups
+            assert pitch == case.K
+            g = x4[:case.M * case.K].view(case.M, case.K).cpu().numpy().view(np.int8)
+            if K_lo:
+                assert np.array_equal(g[:, :K_lo], helpers.masked_slab(e4, case.G, sx_use, nl))
+            assert np.array_equal(g[:, K_lo:], e8)
+        else:
+            if K_lo:
+                g4 = x4[:case.M * pitch].view(case.M, pitch).cpu().numpy()
                 assert np.array_equal(g4[:, :K_lo // 2], e4[:, :K_lo // 2])
-        if case.K - K_lo:
-            assert np.array_equal(x8[:case.M * (case.K - K_lo)].view(case.M, -1).cpu().numpy(), e8)
+            if case.K - K_lo:
+                assert np.array_equal(x8[:case.M * (case.K - K_lo)].view(case.M, -1).cpu().numpy(), e8)
         acc_e = oracle.mixed_gemm_acc(q, case.Wq, case.G, perm, sx_use, sw, nl)
         _check_outputs(L, case, x4, x8, acc_e, dev, x_shift=shifts_dev)
     L.close()
@@ -147,7 +152,7 @@ def test_quantization_matches_ieee_division_near_ties(dev, S):
     L.set_lowbit_ratio(0.0)
     x4, x8, _ = L.quantize_lower(torch.from_numpy(X).to(dev), S)
     torch.cuda.synchronize()
-    got = x8[:M * K].view(M, K).cpu().numpy()
+    got = x4[:M * K].view(M, K).cpu().numpy().view(np.int8)  # masked path: the whole slab is in X4
     assert np.array_equal(got, oracle.quantize(X, S))
     L.close()
 
