@@ -170,6 +170,15 @@ __global__ void group_or_kernel(const void *__restrict__ X, long long M, int K, 
         if (or_s[i]) atomicOr(&or_words[i], or_s[i]);
 }
 
+// Piggy-backed update of the masked path's weight operand: blocks from first_block on copy the
+// channel range [k_from, k_to) of each of `rows` = N * taps weight rows (row length C) from src.
+struct WeightPatch {
+    int8_t *wf;
+    const int8_t *src;
+    int rows, C, k_from, k_to;
+    unsigned first_block;  // = number of quantizing blocks; the grid is larger only when there is work
+};
+
 // Quantize + lower + gather.  Thread <-> (row m, 16-channel slab chunk c16).
 //   sx != nullptr : static positions (slab order);  else positions from or_words.
 // Lowering works on the packed int8 words: q is first clipped to the range the 4-bit value
@@ -180,17 +189,29 @@ template <int DTYPE, int PACKED>
 __global__ void quantize_lower_kernel(const void *__restrict__ X, long long M, int K, int G, int K_lo, float S,
                                       const int32_t *__restrict__ perm, const uint8_t *__restrict__ sx,
                                       const unsigned *__restrict__ or_words, uint8_t *__restrict__ X4,
-                                      long long x4_pitch, int8_t *__restrict__ X8, long long x8_pitch, uint8_t *__restrict__ sx_out)
+                                      long long x4_pitch, int8_t *__restrict__ X8, long long x8_pitch, uint8_t *__restrict__ sx_out,
+                                      WeightPatch wp)
 {
     const int n_c16 = K / 16, c_per_g = G / 16, lo_c16 = K_lo / 16;
     const long long total = M * n_c16;
     const Divider div = make_divider(S);
     ptx::pdl_launch_dependents();
     ptx::pdl_wait();  // the previous kernel may still read the slabs this one overwrites, or write X
+    if (blockIdx.x >= wp.first_block) {
+        // Extra blocks behind the quantizing ones: bring the masked path's weight operand up to date
+        // with the ratio (only the channel groups that changed sides), 16 bytes per thread.
+        const int upt = (wp.k_to - wp.k_from) >> 4;
+        const long long idx = (long long)(blockIdx.x - wp.first_block) * blockDim.x + threadIdx.x;
+        if (idx < (long long)wp.rows * upt) {
+            const size_t off = (size_t)(idx / upt) * wp.C + wp.k_from + 16 * (int)(idx % upt);
+            *reinterpret_cast<uint4 *>(wp.wf + off) = *reinterpret_cast<const uint4 *>(wp.src + off);
+        }
+        return;
+    }
     if (sx_out != nullptr && blockIdx.x == 0)
         for (int j = threadIdx.x; j < K / G; j += blockDim.x) sx_out[j] = (uint8_t)position_from_or(or_words[j]);
     for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-         idx += (long long)gridDim.x * blockDim.x) {
+         idx += (long long)wp.first_block * blockDim.x) {
         const long long m = idx / n_c16;
         const int c16 = (int)(idx - m * n_c16);
         const int j = c16 / c_per_g;
@@ -266,7 +287,7 @@ static cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned blocks, unsigne
 }
 
 template <int DTYPE>
-static int launch_prologue(const Layer *L, const void *X, long long M, float S, int dynamic, uint8_t *X4,
+static int launch_prologue(Layer *L, const void *X, long long M, float S, int dynamic, uint8_t *X4,
                            long long pitch, int8_t *X8, long long pitch8, uint8_t *sx_out, unsigned *scratch, cudaStream_t st)
 {
     const int K = L->C, G = L->G;
@@ -285,10 +306,26 @@ static int launch_prologue(const Layer *L, const void *X, long long M, float S, 
     long long want = (M * n_c16 + threads - 1) / threads;
     long long blocks = want < (long long)sms * 16 ? want : (long long)sms * 16;
     const uint8_t *sx = dynamic ? nullptr : L->sx;
-    if (L->lowbit_path == FLEXIQ_LOWBIT_PACKED_U4)
-        FLEXIQ_CUDA_TRY(launch_pdl(quantize_lower_kernel<DTYPE, 1>, (unsigned)blocks, threads, 0, st, X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, pitch8, dynamic ? sx_out : nullptr));
+    WeightPatch wp{};
+    wp.first_block = (unsigned)blocks;
+    long long extra = 0;
+    const bool masked = L->lowbit_path == FLEXIQ_LOWBIT_MASKED_I8;
+    if (masked && L->wf_K_lo != L->K_lo) {
+        // the GEMM that consumes these slabs needs the weight operand at the same ratio
+        wp.wf = L->wf;
+        wp.src = L->K_lo > L->wf_K_lo ? L->w8m : L->w8;
+        wp.rows = L->N * L->R * L->S;
+        wp.C = L->C;
+        wp.k_from = L->K_lo < L->wf_K_lo ? L->K_lo : L->wf_K_lo;
+        wp.k_to = L->K_lo < L->wf_K_lo ? L->wf_K_lo : L->K_lo;
+        extra = ((long long)wp.rows * ((wp.k_to - wp.k_from) >> 4) + threads - 1) / threads;
+    }
+    const unsigned grid = (unsigned)(blocks + extra);
+    if (!masked)
+        FLEXIQ_CUDA_TRY(launch_pdl(quantize_lower_kernel<DTYPE, 1>, grid, threads, 0, st, X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, pitch8, dynamic ? sx_out : nullptr, wp));
     else
-        FLEXIQ_CUDA_TRY(launch_pdl(quantize_lower_kernel<DTYPE, 0>, (unsigned)blocks, threads, 0, st, X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, pitch8, dynamic ? sx_out : nullptr));
+        FLEXIQ_CUDA_TRY(launch_pdl(quantize_lower_kernel<DTYPE, 0>, grid, threads, 0, st, X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, pitch8, dynamic ? sx_out : nullptr, wp));
+    if (extra) L->wf_K_lo = L->K_lo;
     return FLEXIQ_OK;
 }
 
