@@ -211,6 +211,8 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
     int buf = 0;
     uint32_t buf_phase = 0;
     PROF_DECL(prof_wait);
+    PROF_DECL(prof_ld);
+    PROF_DECL(prof_math);
     PROF_T0(prof_start);
     const int passes = 4 / x.parts;              // 1 with sixteen epilogue warps, 2 with eight
     TileWalk tw;
@@ -231,6 +233,7 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                 waited = true;
             }
             const uint32_t taddr = x.tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)buf * x.buf_stride + (uint32_t)col0;
+            PROF_T0(te0);
             uint32_t ra[32], rb[32];
             if (cols >= 32) ptx::tmem_ld_32x32(taddr, ra); else ptx::tmem_ld_32x16(taddr, ra);
             if (cols == 64) ptx::tmem_ld_32x32(taddr + 32, rb); else if (cols == 48) ptx::tmem_ld_32x16(taddr + 32, rb);
@@ -240,6 +243,8 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                 __syncwarp();
             }
             ptx::tmem_ld_wait();
+            PROF_ADD(prof_ld, te0);
+            PROF_T0(te1);
             if (pass + 1 == passes) {
                 // the accumulator slice is in registers: hand it back to the MMA warp before the math
                 ptx::tc_fence_before_sync();
@@ -286,10 +291,11 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                     }
                 }
             }
+            PROF_ADD(prof_math, te1);
         }
         if ((buf ^= 1) == 0) buf_phase ^= 1;
     }
-    if (quad == 2 && part == 0 && lane == 0) { PROF_STORE(8, prof_wait); PROF_STORE(9, clock64() - prof_start); }
+    if (quad == 2 && part == 0 && lane == 0) { PROF_STORE(8, prof_wait); PROF_STORE(9, clock64() - prof_start); PROF_STORE(10, prof_ld); PROF_STORE(11, prof_math); }
 }
 
 // CG = 1: one CTA per 128 x BN tile.  CG = 2: a CTA pair (cluster of two) per 256 x BN tile;

@@ -7,7 +7,8 @@
 
 Prints one JSON line per (layer, ratio): device time of the prologue and of the mixed kernel
 (CUDA events on the launching stream), TOPS = 2*M*N*K / t and algorithmic GB/s of the mixed kernel.
-Warm numbers come from back-to-back launches; --cold flushes L2 (writes a 256 MB buffer) before
+Warm numbers come from back-to-back launches (--graph: captured in a CUDA graph and replayed, which
+removes the host time between launches that dominates small shapes); --cold flushes L2 (writes a 256 MB buffer) before
 every timed launch and times each launch on its own.
 """
 from __future__ import annotations
@@ -44,7 +45,7 @@ def _alg_bytes(case, is_conv, ratio, Mout):
     return Min * K * (1 - rho / 2) + taps * K * N * (1 - rho / 2) + n_low * N + 8 * N + Mout * N
 
 
-def time_case(case, is_conv, dev, path, iters, cold, flush):
+def time_case(case, is_conv, dev, path, iters, cold, flush, graph=False):
     L = _layer_for(case, dev, is_conv, path)
     X = torch.from_numpy(case.X).to(dev)
     stream = torch.cuda.current_stream()
@@ -82,6 +83,27 @@ def time_case(case, is_conv, dev, path, iters, cold, flush):
                 tp += e[0].elapsed_time(e[1])
                 tg += e[2].elapsed_time(e[3])
             tp, tg = tp / iters, tg / iters
+        elif graph:
+            # the launches are captured once and replayed: no host time between them
+            times = []
+            for body in (lambda: L.quantize_lower(X, case.x_scale), lambda: mixed(Y)):
+                g = torch.cuda.CUDAGraph()
+                side = torch.cuda.Stream()
+                side.wait_stream(stream)
+                with torch.cuda.stream(side):
+                    with torch.cuda.graph(g, stream=side):
+                        for _ in range(iters):
+                            body()
+                torch.cuda.synchronize()
+                g.replay()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for _ in range(5):
+                    g.replay()
+                e1.record(stream)
+                torch.cuda.synchronize()
+                times.append(e0.elapsed_time(e1) / (5 * iters))
+            tp, tg = times
         else:
             e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
             e[0].record(stream)
@@ -93,7 +115,7 @@ def time_case(case, is_conv, dev, path, iters, cold, flush):
             e[2].record(stream)
             torch.cuda.synchronize()
             tp, tg = e[0].elapsed_time(e[1]) / iters, e[1].elapsed_time(e[2]) / iters
-        rows.append({"layer": case.name, "ratio": r, "path": "packed" if path else "masked", "cold": bool(cold),
+        rows.append({"layer": case.name, "ratio": r, "path": "packed" if path else "masked", "cold": bool(cold), "graph": bool(graph),
                      "prologue_us": round(tp * 1e3, 2), "mixed_us": round(tg * 1e3, 2),
                      "mixed_tops": round(ops / tg / 1e9, 1), "mixed_alg_gbs": round(_alg_bytes(case, is_conv, r, Mout) / tg / 1e6, 1)})
         print(json.dumps(rows[-1]), flush=True)
@@ -156,6 +178,7 @@ def main():
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--iters", type=int, default=30)
     ap.add_argument("--cold", action="store_true")
+    ap.add_argument("--graph", action="store_true", help="capture the launches in a CUDA graph and time its replay")
     ap.add_argument("--path", default="masked", choices=["masked", "packed"])
     ap.add_argument("--batch", type=int, default=0)
     args = ap.parse_args()
@@ -163,16 +186,16 @@ def main():
     path = fx.LOWBIT_PACKED_U4 if args.path == "packed" else fx.LOWBIT_MASKED_I8
     flush = torch.zeros(64 * 1024 * 1024, dtype=torch.int32, device=dev) if args.cold else None
     if args.config == 1:
-        time_case(inputs.config1(), False, dev, path, args.iters, args.cold, flush)
+        time_case(inputs.config1(), False, dev, path, args.iters, args.cold, flush, args.graph)
     elif args.config == 2:
         for c in inputs.config2(args.batch or 64):
-            time_case(c, False, dev, path, args.iters, args.cold, flush)
+            time_case(c, False, dev, path, args.iters, args.cold, flush, args.graph)
     elif args.config == 3:
         for c in inputs.config3(args.batch or 32):
-            time_case(c, True, dev, path, args.iters, args.cold, flush)
+            time_case(c, True, dev, path, args.iters, args.cold, flush, args.graph)
     elif args.config == 4:
         for c in inputs.config4(args.batch or 1):
-            time_case(c, False, dev, path, args.iters, args.cold, flush)
+            time_case(c, False, dev, path, args.iters, args.cold, flush, args.graph)
     elif args.config == 5:
         run_stack(dev, args.batch or 128, max(1, args.iters // 10))
 
