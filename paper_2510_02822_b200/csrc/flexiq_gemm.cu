@@ -39,7 +39,6 @@ constexpr int kNumWorkWarps = 16;                     // epilogue warps (+ expan
 constexpr int kThreads = 32 * (2 + kNumWorkWarps);
 constexpr int kRawStages = 2;                         // packed path: ring of raw 4-bit tiles in front of the operand ring
 constexpr uint32_t kSpinLimit = 1u << 21;              // parked waits of <= 1 us each: about two seconds at most
-constexpr int kABytes = BM * 128;                     // A stage (BK <= 128 bytes per row)
 constexpr int kStageRegion = 196608;                  // shared memory given to the operand ring
 constexpr int kFactorsPerWarp = 512;                  // alpha[64] | beta[64] of the warp's columns in the current tile
 constexpr int kMaxStages = 8;
@@ -54,6 +53,7 @@ struct GemmParams {
     int BK;              // K bytes per stage: 128 or 64
     int BN;              // tile width: 64, 128, 192 or 256
     int stages;          // depth of the operand ring
+    int tps;             // filter taps per ring stage (> 1 only for masked convolutions whose C fits one K block)
     int nb_lo, nb_hi;    // k-blocks per tap in the low / high slab
     int im2col;          // A operand through im2col-mode TMA
     int P, Q, stride, pad;
@@ -331,7 +331,9 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int BN = p.BN;
     const int b_rows = BN / CG;                       // rows of the B tile this CTA loads
-    const int stage_bytes = kABytes + b_rows * 128;
+    // one stage = tps sub-tiles of A (BM x BK each) followed by tps sub-tiles of B (b_rows x BK each)
+    const int a_sub = BM * p.BK, b_sub = b_rows * p.BK, b_off = p.tps * a_sub;
+    const int stage_bytes = p.tps * (a_sub + b_sub);
     const int num_tiles = p.m_tiles * p.n_tiles;
     const uint32_t cta_rank = CG == 2 ? ptx::cluster_ctarank() : 0u;
     const bool leader = cta_rank == 0;
@@ -405,6 +407,28 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                 pix_h = (rem / p.Q) * p.stride - p.pad;
                 pix_w = (rem % p.Q) * p.stride - p.pad;
             }
+            if (p.tps > 1) {
+                // several filter taps per stage: one barrier round trip pays for all of them
+                for (int tap0 = 0; tap0 < p.T && ok; tap0 += p.tps) {
+                    const int nt = min(p.tps, p.T - tap0);
+                    if (!__all_sync(0xffffffffu, wait_bounded(empty0 + 8 * stage, phase ^ 1, abort_flag, 1))) { ok = false; break; }
+                    if (ptx::elect_one()) {
+                        const uint32_t sa = stage0 + stage * stage_bytes;
+                        if (leader) ptx::mbar_expect_tx_s(full0 + 8 * stage, (uint32_t)(CG * nt * (a_sub + b_sub)));
+                        const uint32_t bar = full0_lead + 8 * stage;
+                        for (int i = 0; i < nt; ++i) {
+                            const int tap = tap0 + i;
+                            ptx::tma_load_im2col_4d_s<CG>(sa + i * a_sub, &mapA_hi, bar, 0, pix_w, pix_h, pix_n,
+                                                          (uint16_t)(tap % p.S), (uint16_t)(tap / p.S));
+                            ptx::tma_load_2d_s<CG>(sa + b_off + i * b_sub, &mapB_hi, bar, tap * p.C, n0);
+                        }
+                    }
+                    __syncwarp();
+                    ++issued;
+                    if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
+                }
+                continue;
+            }
             for (int part = 0; part < 2 && ok; ++part) {
                 const int nb = part ? p.nb_hi : p.nb_lo;
                 if (nb == 0) continue;
@@ -451,7 +475,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                                 ptx::tma_load_im2col_4d_s<CG>(sa, ma, bar, xa, pix_w, pix_h, pix_n, (uint16_t)tap_s, (uint16_t)tap_r);
                             else
                                 ptx::tma_load_2d_s<CG>(sa, ma, bar, xa, (int)m0);
-                            ptx::tma_load_2d_s<CG>(sa + kABytes, mb, bar, xb, n0);
+                            ptx::tma_load_2d_s<CG>(sa + b_off, mb, bar, xb, n0);
                         }
                         __syncwarp();
                         xa += p.BK;
@@ -489,7 +513,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             const uint64_t adesc0 = ptx::smem_desc(ptx::smem_u32(stage_base), p.BK);
             const uint32_t desc_hi = (uint32_t)(adesc0 >> 32);
             const uint32_t a_lo0 = (uint32_t)adesc0;
-            const uint32_t b_lo0 = a_lo0 + (kABytes >> 4);
+            const uint32_t b_lo0 = a_lo0 + (uint32_t)(b_off >> 4);
             const uint32_t stage_step = (uint32_t)(stage_bytes >> 4);  // stays inside the 14-bit address field
             const uint32_t empty0 = ptx::smem_u32(empty_bar);
             const uint32_t full0 = ptx::smem_u32(full_bar);
@@ -509,7 +533,26 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)buf * buf_stride;
                 uint32_t acc = 0;
-                for (int part = 0; part < 2 && ok; ++part) {
+                if (p.tps > 1) {
+                    const int ks = (p.C + 31) >> 5;  // K steps of one tap (C <= BK)
+                    for (int tap0 = 0; tap0 < p.T && ok; tap0 += p.tps) {
+                        const int nt = min(p.tps, p.T - tap0);
+                        if (!__all_sync(0xffffffffu, wait_bounded(full0 + 8 * stage, phase, abort_flag, 3))) { ok = false; break; }
+                        const uint32_t a_lo = a_lo0 + stage * stage_step, b_lo = b_lo0 + stage * stage_step;
+                        if (ptx::elect_one()) {
+                            for (int i = 0; i < nt; ++i)
+                                for (int k = 0; k < ks; ++k) {
+                                    ptx::mma_i8_s<CG>(d_tmem, a_lo + i * (a_sub >> 4) + 2 * k, b_lo + i * (b_sub >> 4) + 2 * k, desc_hi, idesc, acc);
+                                    acc = 1;
+                                }
+                            ptx::mma_commit_s<CG>(empty0 + 8 * stage);
+                        }
+                        __syncwarp();
+                        acc = 1;
+                        if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
+                    }
+                }
+                for (int part = 0; part < 2 && ok && p.tps == 1; ++part) {
                     const int nb = part ? p.nb_hi : p.nb_lo;
                     if (nb == 0) continue;
                     const int ks_last = ((part ? p.C_hi : p.C_lo) - (nb - 1) * p.BK + 31) >> 5;
@@ -618,7 +661,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                                 const uint8_t *rawA = raw_base + rstage * raw_bytes;
                                 const uint8_t *rawB = rawA + BM * half;
                                 uint8_t *dstA = stage_base + stage * stage_bytes;
-                                uint8_t *dstB = dstA + kABytes;
+                                uint8_t *dstB = dstA + b_off;
                                 if (hasB) {
                                     const uint8_t *src = rawB + rowB * half;
                                     uint8_t *dst = dstB + rowB * p.BK;
@@ -875,11 +918,19 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     p.m_tiles = (int)((M + (long long)BM * cg - 1) / ((long long)BM * cg));
     p.BN = bn;
     p.n_tiles = (L->N + bn - 1) / bn;
-    p.stages = kStageRegion / (kABytes + (bn / cg) * 128);
+    p.tps = 1;
+    if (!packed && p.im2col && L->C <= p.BK && L->S > 1) {
+        // convolution whose channels fit one K block: a stage holds up to a filter row of taps
+        const int per_tap = (BM + bn / cg) * p.BK;
+        const int limit = 49152 / per_tap;
+        p.tps = L->S < limit ? L->S : limit;
+        if (p.tps < 1) p.tps = 1;
+    }
+    p.stages = kStageRegion / (p.tps * (BM + bn / cg) * p.BK);
     if (p.stages > kMaxStages) p.stages = kMaxStages;
     if (packed) {  // room for the ring of raw 4-bit tiles behind the operand ring
         const int raw = kRawStages * (BM + bn) * (p.BK / 2);
-        p.stages = (kStageRegion - raw) / (kABytes + bn * 128);
+        p.stages = (kStageRegion - raw) / ((BM + bn) * p.BK);
         if (p.stages > kMaxStages) p.stages = kMaxStages;
     }
     // the per-output-channel factors depend on the call's scales: recomputed (one tiny launch,
