@@ -181,6 +181,43 @@ int flexiq_mixed_conv(flexiq_layer_t layer, const uint8_t *X4_dev, const int8_t 
                       const uint8_t *x_shift_dev, int Nb, int H, int W, float x_scale,
                       float y_scale, int out_mode, void *Y_dev, void *stream);
 
+/* out_order of flexiq_mixed_gemm_to_slab / flexiq_mixed_conv_to_slab */
+#define FLEXIQ_ORDER_ORIGINAL 0  /* output channel n of this layer is input channel n of the next one */
+#define FLEXIQ_ORDER_NEXT_SLAB 1 /* this layer's output channels were permuted offline into the next layer's slab order */
+
+/* Fused layer boundary: the mixed GEMM / convolution of `layer` whose epilogue writes the
+ * activation slab of `next_layer` directly, so that no 8-bit tensor and no prologue pass lies
+ * between two quantized layers.  Per output element it computes what the two-call sequence
+ *   flexiq_mixed_*(..., y_scale = next_x_scale, REQUANT_I8)  [-> max(., 0) if relu]
+ *   flexiq_quantize_lower(next_layer, ., FLEXIQ_DTYPE_I8, static positions)
+ * computes, bit for bit: the value re-quantized by Eq. 1's rounding at the next layer's scale,
+ * moved to its channel's place in the next layer's slab order (layout post-processing, Sec. 5),
+ * and, when its group lies below the next layer's current max_4bit_ch, bit-lowered at the group's
+ * static extraction position with saturation (Sec. 4.1) and stored as x4 << sx.
+ *   next_layer     a layer on the MASKED path of the same device with K (or Cin) equal to this
+ *                  layer's N (or Cout); its ratio at the time of this call decides the lowering
+ *   next_x_scale   the next layer's activation scale (> 0)
+ *   relu           non-zero: max(., 0) between the two layers (ResNet-style blocks)
+ *   out_order      ORIGINAL: each 16-channel chunk of the result is scattered to its place in the
+ *                  next layer's slab order (16-byte stores).  NEXT_SLAB: the caller created this
+ *                  layer from weights, scales and biases whose output channels were already
+ *                  permuted into the next layer's slab order (Sec. 5: the reordering is moved
+ *                  offline into the producing layer), so channel n lands at slab channel n and
+ *                  rows are written with full 32-byte stores -- the faster form.
+ *   next_X4_dev    [M][N] (or [Nb][P][Q][Cout]) the next layer's slab, 16-byte aligned, caller-owned
+ * Dynamic positions for the next layer are not available here (they need all rows first).
+ * The paper runs the two steps as separate kernels; it has no counterpart of this fusion.
+ * Errors as for flexiq_mixed_gemm, plus UNSUPPORTED when next_layer is on the PACKED path and
+ * INVALID_ARG when the channel counts or devices differ. */
+int flexiq_mixed_gemm_to_slab(flexiq_layer_t layer, const uint8_t *X4_dev, const int8_t *X8_dev,
+                              const uint8_t *x_shift_dev, int64_t M, float x_scale,
+                              flexiq_layer_t next_layer, float next_x_scale, int relu,
+                              int out_order, uint8_t *next_X4_dev, void *stream);
+int flexiq_mixed_conv_to_slab(flexiq_layer_t layer, const uint8_t *X4_dev, const int8_t *X8_dev,
+                              const uint8_t *x_shift_dev, int Nb, int H, int W, float x_scale,
+                              flexiq_layer_t next_layer, float next_x_scale, int relu,
+                              int out_order, uint8_t *next_X4_dev, void *stream);
+
 /* Test hooks: copy the layer's derived tables to host buffers (any may be NULL).
  *   sw_host [K/G][N] uint8 weight extraction positions (slab order),
  *   w8_host [N][Kw] int8 slab-order weights, w4_host [N][Kw/2] packed 4-bit weights,

@@ -17,11 +17,13 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4
 DTYPE_F32, DTYPE_F16, DTYPE_BF16, DTYPE_I8 = 0, 1, 2, 3
 OUT_ACC_I32, OUT_REQUANT_I8, OUT_DEQUANT_F32 = 0, 1, 2
 LOWBIT_MASKED_I8, LOWBIT_PACKED_U4 = 0, 1
+ORDER_ORIGINAL, ORDER_NEXT_SLAB = 0, 1
 
 EXPORTS = [
     "flexiq_layer_create_linear", "flexiq_layer_create_conv", "flexiq_layer_destroy",
     "flexiq_layer_set_lowbit_path", "flexiq_set_lowbit_ratio", "flexiq_get_max_4bit_ch",
     "flexiq_x4_pitch", "flexiq_quantize_lower", "flexiq_quantize_lower_dynamic_noalloc", "flexiq_mixed_gemm", "flexiq_mixed_conv",
+    "flexiq_mixed_gemm_to_slab", "flexiq_mixed_conv_to_slab",
     "flexiq_layer_export", "flexiq_force_tile", "flexiq_check_status", "flexiq_last_error",
 ]
 
@@ -56,6 +58,8 @@ def lib():
         L.flexiq_quantize_lower_dynamic_noalloc.argtypes = [vp, vp, i32, i64, f32, vp, vp, vp, vp]
         L.flexiq_mixed_gemm.argtypes = [vp, vp, vp, vp, i64, f32, f32, i32, vp, vp]
         L.flexiq_mixed_conv.argtypes = [vp, vp, vp, vp, i32, i32, i32, f32, f32, i32, vp, vp]
+        L.flexiq_mixed_gemm_to_slab.argtypes = [vp, vp, vp, vp, i64, f32, vp, f32, i32, i32, vp, vp]
+        L.flexiq_mixed_conv_to_slab.argtypes = [vp, vp, vp, vp, i32, i32, i32, f32, vp, f32, i32, i32, vp, vp]
         L.flexiq_layer_export.argtypes = [vp, vp, vp, vp]
         L.flexiq_check_status.argtypes = [vp]
         _lib = L
@@ -144,6 +148,16 @@ def flexiq_mixed_gemm(h, X4_dev, X8_dev, x_shift_dev, M, x_scale, y_scale, out_m
 def flexiq_mixed_conv(h, X4_dev, X8_dev, x_shift_dev, Nb, H, W, x_scale, y_scale, out_mode, Y_dev):
     _check(lib().flexiq_mixed_conv(h, _ptr(X4_dev), _ptr(X8_dev), _ptr(x_shift_dev), Nb, H, W, x_scale, y_scale,
                                    out_mode, _ptr(Y_dev), _stream()))
+
+
+def flexiq_mixed_gemm_to_slab(h, X4_dev, X8_dev, x_shift_dev, M, x_scale, next_h, next_x_scale, relu, out_order, next_X4_dev):
+    _check(lib().flexiq_mixed_gemm_to_slab(h, _ptr(X4_dev), _ptr(X8_dev), _ptr(x_shift_dev), M, x_scale, next_h,
+                                           next_x_scale, int(relu), out_order, _ptr(next_X4_dev), _stream()))
+
+
+def flexiq_mixed_conv_to_slab(h, X4_dev, X8_dev, x_shift_dev, Nb, H, W, x_scale, next_h, next_x_scale, relu, out_order, next_X4_dev):
+    _check(lib().flexiq_mixed_conv_to_slab(h, _ptr(X4_dev), _ptr(X8_dev), _ptr(x_shift_dev), Nb, H, W, x_scale, next_h,
+                                           next_x_scale, int(relu), out_order, _ptr(next_X4_dev), _stream()))
 
 
 def flexiq_layer_export(h, sw_host=None, w8_host=None, w4_host=None):
@@ -239,6 +253,22 @@ class Layer:
             Y = torch.empty((M, self.N), dtype=dt, device=self.device)
         flexiq_mixed_gemm(self.h, x4, x8, x_shift, M, x_scale, y_scale, out_mode, Y)
         return Y
+
+    def mixed_gemm_to_slab(self, x4, x8, M, x_scale, nxt, next_x_scale, relu=False, slab=None, x_shift=None, out_order=ORDER_ORIGINAL):
+        """Mixed GEMM whose epilogue writes the masked slab of the layer `nxt` (fused layer boundary)."""
+        if slab is None:
+            slab = nxt.alloc_slabs(M)[0]
+        flexiq_mixed_gemm_to_slab(self.h, x4, x8, x_shift, M, x_scale, nxt.h, next_x_scale, relu, out_order, slab)
+        return slab
+
+    def mixed_conv_to_slab(self, x4, x8, Nb, H, W, x_scale, nxt, next_x_scale, relu=False, slab=None, x_shift=None, out_order=ORDER_ORIGINAL):
+        stride, pad = self.conv
+        P = (H + 2 * pad - self.R) // stride + 1
+        Q = (W + 2 * pad - self.S) // stride + 1
+        if slab is None:
+            slab = nxt.alloc_slabs(Nb * P * Q)[0]
+        flexiq_mixed_conv_to_slab(self.h, x4, x8, x_shift, Nb, H, W, x_scale, nxt.h, next_x_scale, relu, out_order, slab)
+        return slab
 
     def mixed_conv(self, x4, x8, Nb, H, W, x_scale, y_scale, out_mode, Y=None, x_shift=None):
         import torch

@@ -43,3 +43,14 @@ def static_preparation(Xcal_q: torch.Tensor, Wq: torch.Tensor, G: int, conv: boo
     score = (torch.maximum(hi, -lo).to(torch.int64) * wmax.to(torch.int64)).reshape(-1, G).max(1).values
     perm = torch.sort(score, stable=True).indices.to(torch.int32)
     return np.ascontiguousarray(perm.numpy()), np.ascontiguousarray(x_shift.numpy())
+
+
+def permute_outputs_for_next(Wq: torch.Tensor, w_scale: torch.Tensor, bias, next_perm, next_G: int, conv: bool = False):
+    """Moves the next layer's channel reordering offline into this layer (Sec. 5): returns this
+    layer's weights, scales and bias with the output channels in the next layer's slab order, so
+    that output channel n of the permuted layer is slab channel n of the next one.
+
+    Wq: int8 [K, N] (linear) or [Cout, R, S, Cin] (conv); next_perm: the next layer's group order."""
+    cols = torch.cat([torch.arange(int(g) * next_G, (int(g) + 1) * next_G) for g in next_perm]).to(Wq.device)
+    Wp = Wq.index_select(0 if conv else 1, cols).contiguous()
+    return Wp, w_scale.index_select(0, cols).contiguous(), None if bias is None else bias.index_select(0, cols).contiguous()

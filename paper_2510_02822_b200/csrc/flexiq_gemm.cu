@@ -44,6 +44,10 @@ constexpr int kFactorsPerWarp = 512;                  // alpha[64] | beta[64] of
 constexpr int kMaxStages = 8;
 constexpr int kSmemBytes = kStageRegion + kNumWorkWarps * kFactorsPerWarp + 256;
 
+// Internal epilogue mode of the fused layer boundary: the int8 result goes straight into the
+// next layer's masked slab (its channel order, its low groups lowered).
+constexpr int kOutNextSlab = 3;
+
 struct GemmParams {
     long long M;         // rows of the implicit GEMM (tokens or output pixels)
     int N;               // output channels
@@ -62,6 +66,10 @@ struct GemmParams {
     const float *beta;   // [N] per-output-channel addend of this call
     void *Y;
     int m_tiles, n_tiles;
+    // fused layer boundary only: where each 16-channel chunk of the output lands in the next layer's slab
+    const int32_t *next_ent;   // [N/16] slab position (in chunks) of original chunk c | its group's position << 24
+    int next_K_lo;             // the next layer's max_4bit_ch
+    int relu;                  // clamp at zero before the re-quantization
     // packed low-bit path only: positions the expander warps shift the 4-bit values back to
     const uint8_t *sx;   // [n_g] activation positions, slab order
     const uint8_t *sw;   // [n_g][N] weight positions
@@ -154,6 +162,23 @@ __device__ __forceinline__ void finish16(const uint32_t *r, const float *alpha16
         }
     }
 }
+// Fused layer boundary: 16 outputs re-quantized with the next layer's activation scale, clipped
+// to [lo, hi] before the rounding (the range the next layer's 4-bit value can hold at its
+// position, or the int8 range), low bits cleared by `mask`: the next layer's masked slab bytes.
+__device__ __forceinline__ void finish16_next(const uint32_t *r, const float *alpha16, const float *beta16, float lo, float hi,
+                                              uint32_t mask, uint32_t *out)
+{
+    const float4 *fa = reinterpret_cast<const float4 *>(alpha16), *fb = reinterpret_cast<const float4 *>(beta16);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float4 a = fa[i], b = fb[i];
+        const float y0 = fminf(fmaxf(fmaf((float)(int)r[4 * i + 0], a.x, b.x), lo), hi);
+        const float y1 = fminf(fmaxf(fmaf((float)(int)r[4 * i + 1], a.y, b.y), lo), hi);
+        const float y2 = fminf(fmaxf(fmaf((float)(int)r[4 * i + 2], a.z, b.z), lo), hi);
+        const float y3 = fminf(fmaxf(fmaf((float)(int)r[4 * i + 3], a.w, b.w), lo), hi);
+        out[i] = requant4(y0, y1, y2, y3) & mask;
+    }
+}
 __device__ __forceinline__ void st_global_128(void *p, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
 {
     asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
@@ -201,7 +226,7 @@ template <int CG, int MODE>
 __device__ __forceinline__ void epilogue_role(const GemmParams &p, const EpilogueCtx &x, int quad, int part, int lane)
 {
     constexpr bool kScaled = MODE != FLEXIQ_OUT_ACC_I32;
-    constexpr int kElem = MODE == FLEXIQ_OUT_REQUANT_I8 ? 1 : 4;  // output bytes per element
+    constexpr int kElem = (MODE == FLEXIQ_OUT_REQUANT_I8 || MODE == kOutNextSlab) ? 1 : 4;  // output bytes per element
     const int BN = p.BN;
     const int cols = BN >> 2;                    // 16, 32, 48 or 64 columns for this warp
     const bool y32 = (reinterpret_cast<uintptr_t>(p.Y) & 31) == 0;
@@ -224,6 +249,8 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
             const int nw = tw.n_blk * BN + col0;             // ... as an output channel
             float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
             if (kScaled && nw + 4 * (lane & 15) < p.N) f = __ldg(reinterpret_cast<const float4 *>(fsrc + nw));
+            int ent = 0;                                     // fused boundary: lane g fetches chunk g's slab entry
+            if (MODE == kOutNextSlab && lane < 4 && nw + 16 * lane < p.N) ent = __ldg(p.next_ent + (nw >> 4) + lane);
             if (!waited) {
                 PROF_T0(t0);
                 const bool ok = wait_bounded(&x.tmem_full[buf], buf_phase, x.abort_flag, 4);
@@ -254,6 +281,11 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                     else ptx::mbar_arrive_relaxed(&x.tmem_empty[buf]);
                 }
             }
+            int ents[4] = {0, 0, 0, 0};
+            if (MODE == kOutNextSlab) {
+#pragma unroll
+                for (int g = 0; g < 4; ++g) ents[g] = __shfl_sync(0xffffffffu, ent, g);
+            }
             if (row < p.M) {
                 uint8_t *yrow = static_cast<uint8_t *>(p.Y) + (row * p.N + nw) * kElem;
 #pragma unroll
@@ -262,7 +294,41 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                     const int n = nw + 32 * h;
                     if (32 * h < cols && n < p.N) {
                         const bool second = 32 * h + 16 < cols && n + 16 < p.N;  // columns 16..31 of this half are live
-                        if (MODE == FLEXIQ_OUT_REQUANT_I8) {
+                        if (MODE == kOutNextSlab) {
+                            // each 16-channel chunk goes to its place in the next layer's slab row
+                            uint32_t w[8];
+                            int pos[2] = {0, 0};
+#pragma unroll
+                            for (int g = 0; g < 2; ++g) {
+                                if (g == 0 || second) {
+                                    const int e = ents[2 * h + g];
+                                    pos[g] = e & 0xffffff;
+                                    float lo = -128.f, hi = 127.f;
+                                    uint32_t mask = 0xffffffffu;
+                                    if (pos[g] * 16 < p.next_K_lo) {
+                                        const int sft = e >> 24;
+                                        hi = (float)(8 << sft) - 1.f;
+                                        lo = -(float)(8 << sft);
+                                        mask = ((0xffu << sft) & 0xffu) * 0x01010101u;
+                                    }
+                                    if (p.relu) lo = fmaxf(lo, 0.f);
+                                    // the pack saturates to [-128, 127] by itself: clamp only when the range is narrower (warp-uniform)
+                                    if (lo > -128.f || hi < 127.f)
+                                        finish16_next(r + 16 * g, x.fac + 32 * h + 16 * g, x.fac + 64 + 32 * h + 16 * g, lo, hi, mask, w + 4 * g);
+                                    else {
+                                        finish16<FLEXIQ_OUT_REQUANT_I8>(r + 16 * g, x.fac + 32 * h + 16 * g, x.fac + 64 + 32 * h + 16 * g, w + 4 * g);
+#pragma unroll
+                                        for (int q = 0; q < 4; ++q) w[4 * g + q] &= mask;
+                                    }
+                                }
+                            }
+                            uint8_t *srow = static_cast<uint8_t *>(p.Y) + row * p.N;
+                            if (second && wide && pos[1] == pos[0] + 1 && (pos[0] & 1) == 0) st_global_256(srow + pos[0] * 16, w);
+                            else {
+                                st_global_128(srow + pos[0] * 16, w[0], w[1], w[2], w[3]);
+                                if (second) st_global_128(srow + pos[1] * 16, w[4], w[5], w[6], w[7]);
+                            }
+                        } else if (MODE == FLEXIQ_OUT_REQUANT_I8) {
                             uint32_t w[8];
                             finish16<MODE>(r, x.fac + 32 * h, x.fac + 64 + 32 * h, w);
                             if (second) finish16<MODE>(r + 16, x.fac + 32 * h + 16, x.fac + 64 + 32 * h + 16, w + 4);
@@ -607,6 +673,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             x.parts = kEpiWarps / 4; x.arrivals_on = 1;
             if (p.out_mode == FLEXIQ_OUT_REQUANT_I8) epilogue_role<CG, FLEXIQ_OUT_REQUANT_I8>(p, x, warp & 3, e >> 2, lane);
             else if (p.out_mode == FLEXIQ_OUT_DEQUANT_F32) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_F32>(p, x, warp & 3, e >> 2, lane);
+            else if (p.out_mode == kOutNextSlab) epilogue_role<CG, kOutNextSlab>(p, x, warp & 3, e >> 2, lane);
             else epilogue_role<CG, FLEXIQ_OUT_ACC_I32>(p, x, warp & 3, e >> 2, lane);
         } else if (PK) {
             // --------------------------------------------------------- expanders (packed path)
@@ -846,11 +913,22 @@ static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const
 }
 
 static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_t *x_shift, long long M, int Nb, int H,
-                     int W, float x_scale, float y_scale, int out_mode, void *Y, cudaStream_t st)
+                     int W, float x_scale, float y_scale, int out_mode, void *Y, cudaStream_t st,
+                     const Layer *next = nullptr, int relu = 0, int out_order = 0)
 {
-    if (out_mode < FLEXIQ_OUT_ACC_I32 || out_mode > FLEXIQ_OUT_DEQUANT_F32)
+    if (next) {
+        // fused layer boundary: Y is the next layer's masked slab, y_scale its activation scale
+        if (next->lowbit_path != FLEXIQ_LOWBIT_MASKED_I8)
+            return set_error(FLEXIQ_ERR_UNSUPPORTED, "the next layer must use the masked low-bit path");
+        if (next->C != L->N)
+            return set_error(FLEXIQ_ERR_INVALID_ARG, "next layer has %d input channels, this layer %d output channels", next->C, L->N);
+        if (next->device != L->device) return set_error(FLEXIQ_ERR_INVALID_ARG, "the two layers live on different devices");
+        if (out_order != FLEXIQ_ORDER_ORIGINAL && out_order != FLEXIQ_ORDER_NEXT_SLAB)
+            return set_error(FLEXIQ_ERR_INVALID_ARG, "unknown out_order %d", out_order);
+        out_mode = kOutNextSlab;
+    } else if (out_mode < FLEXIQ_OUT_ACC_I32 || out_mode > FLEXIQ_OUT_DEQUANT_F32)
         return set_error(FLEXIQ_ERR_INVALID_ARG, "unknown out_mode %d", out_mode);
-    if (out_mode == FLEXIQ_OUT_REQUANT_I8 && !(y_scale > 0.0f))
+    if ((out_mode == FLEXIQ_OUT_REQUANT_I8 || next) && !(y_scale > 0.0f))
         return set_error(FLEXIQ_ERR_INVALID_ARG, "y_scale %g must be positive", (double)y_scale);
     if (M == 0) return FLEXIQ_OK;
     const int C_lo = L->K_lo, C_hi = L->C - C_lo;
@@ -895,6 +973,7 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
         p.Q = (W + 2 * L->pad - L->S) / L->stride + 1;
     }
     p.out_mode = out_mode; p.Y = Y;
+    if (next) { p.next_ent = out_order == FLEXIQ_ORDER_NEXT_SLAB ? next->chunk_ent_slab : next->chunk_ent; p.next_K_lo = next->K_lo; p.relu = relu != 0; }
     p.alpha = L->alpha; p.beta = L->beta;
     TileChoice tc = g_forced_tile.cg ? g_forced_tile : choose_tile(M, L->N, p.T * (p.nb_lo + p.nb_hi), sms);
     if (packed && tc.cg == 2) {  // the packed path runs single CTAs: re-choose among those
@@ -935,12 +1014,13 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     }
     // the per-output-channel factors depend on the call's scales: recomputed (one tiny launch,
     // stream-ordered before the GEMM) only when they differ from the previous call's
-    if (out_mode != FLEXIQ_OUT_ACC_I32 &&
-        !(L->cache_mode == out_mode && L->cache_xs == x_scale && (out_mode == FLEXIQ_OUT_DEQUANT_F32 || L->cache_ys == y_scale))) {
-        scale_vectors_kernel<<<(L->N + 255) / 256, 256, 0, st>>>(L->N, x_scale, y_scale, out_mode == FLEXIQ_OUT_REQUANT_I8,
+    const int fmode = next ? FLEXIQ_OUT_REQUANT_I8 : out_mode;  // the fused boundary re-quantizes with the same factors
+    if (fmode != FLEXIQ_OUT_ACC_I32 &&
+        !(L->cache_mode == fmode && L->cache_xs == x_scale && (fmode == FLEXIQ_OUT_DEQUANT_F32 || L->cache_ys == y_scale))) {
+        scale_vectors_kernel<<<(L->N + 255) / 256, 256, 0, st>>>(L->N, x_scale, y_scale, fmode == FLEXIQ_OUT_REQUANT_I8,
                                                                  L->w_scale, L->bias, L->alpha, L->beta);
         FLEXIQ_CUDA_TRY(cudaGetLastError());
-        L->cache_mode = out_mode; L->cache_xs = x_scale; L->cache_ys = y_scale;
+        L->cache_mode = fmode; L->cache_xs = x_scale; L->cache_ys = y_scale;
     }
 
     // activation maps (per call: they depend on the caller's buffers, M and the ratio);
@@ -1006,6 +1086,34 @@ extern "C" int flexiq_mixed_conv(flexiq_layer_t layer, const uint8_t *X4_dev, co
     if (P <= 0 || Q <= 0) return set_error(FLEXIQ_ERR_INVALID_ARG, "filter does not fit the padded input");
     return run_mixed(L, X4_dev, X8_dev, x_shift_dev, (long long)Nb * P * Q, Nb, H, W, x_scale, y_scale, out_mode, Y_dev,
                      reinterpret_cast<cudaStream_t>(stream));
+}
+
+extern "C" int flexiq_mixed_gemm_to_slab(flexiq_layer_t layer, const uint8_t *X4_dev, const int8_t *X8_dev,
+                                         const uint8_t *x_shift_dev, int64_t M, float x_scale, flexiq_layer_t next_layer,
+                                         float next_x_scale, int relu, int out_order, uint8_t *next_X4_dev, void *stream)
+{
+    Layer *L = as_layer(layer), *Nx = as_layer(next_layer);
+    if (!L || !Nx) return set_error(FLEXIQ_ERR_INVALID_ARG, "not a live flexiq layer handle");
+    if (L->is_conv) return set_error(FLEXIQ_ERR_INVALID_ARG, "layer is a convolution: use flexiq_mixed_conv_to_slab");
+    if (M < 0) return set_error(FLEXIQ_ERR_INVALID_ARG, "M = %lld is negative", (long long)M);
+    return run_mixed(L, X4_dev, X8_dev, x_shift_dev, M, 0, 0, 0, x_scale, next_x_scale, 0, next_X4_dev,
+                     reinterpret_cast<cudaStream_t>(stream), Nx, relu, out_order);
+}
+
+extern "C" int flexiq_mixed_conv_to_slab(flexiq_layer_t layer, const uint8_t *X4_dev, const int8_t *X8_dev,
+                                         const uint8_t *x_shift_dev, int Nb, int H, int W, float x_scale,
+                                         flexiq_layer_t next_layer, float next_x_scale, int relu, int out_order,
+                                         uint8_t *next_X4_dev, void *stream)
+{
+    Layer *L = as_layer(layer), *Nx = as_layer(next_layer);
+    if (!L || !Nx) return set_error(FLEXIQ_ERR_INVALID_ARG, "not a live flexiq layer handle");
+    if (!L->is_conv) return set_error(FLEXIQ_ERR_INVALID_ARG, "layer is linear: use flexiq_mixed_gemm_to_slab");
+    if (Nb < 0 || H <= 0 || W <= 0) return set_error(FLEXIQ_ERR_INVALID_ARG, "bad activation shape Nb=%d H=%d W=%d", Nb, H, W);
+    const int P = (H + 2 * L->pad - L->R) / L->stride + 1;
+    const int Q = (W + 2 * L->pad - L->S) / L->stride + 1;
+    if (P <= 0 || Q <= 0) return set_error(FLEXIQ_ERR_INVALID_ARG, "filter does not fit the padded input");
+    return run_mixed(L, X4_dev, X8_dev, x_shift_dev, (long long)Nb * P * Q, Nb, H, W, x_scale, next_x_scale, 0, next_X4_dev,
+                     reinterpret_cast<cudaStream_t>(stream), Nx, relu, out_order);
 }
 
 #ifdef FLEXIQ_PROFILE

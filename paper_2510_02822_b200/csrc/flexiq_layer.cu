@@ -171,7 +171,7 @@ static void free_layer(Layer *L)
 {
     if (!L) return;
     cudaFree(L->w8); cudaFree(L->w8m); cudaFree(L->w4); cudaFree(L->wf); cudaFree(L->sw); cudaFree(L->sx);
-    cudaFree(L->perm); cudaFree(L->w_scale); cudaFree(L->bias); cudaFree(L->alpha); cudaFree(L->beta);
+    cudaFree(L->perm); cudaFree(L->chunk_ent); cudaFree(L->chunk_ent_slab); cudaFree(L->w_scale); cudaFree(L->bias); cudaFree(L->alpha); cudaFree(L->beta);
     free(L->perm_host); free(L->sx_host);
     L->magic = 0;
     free(L);
@@ -245,6 +245,22 @@ static int create_common(flexiq_layer_t *out, int is_conv, int C, int N, int R, 
     L->cache_mode = -1;
     TRY_OR_FREE(cudaMemcpyAsync(L->perm, L->perm_host, sizeof(int32_t) * n_g, cudaMemcpyHostToDevice, stream));
     TRY_OR_FREE(cudaMemcpyAsync(L->sx, L->sx_host, n_g, cudaMemcpyHostToDevice, stream));
+    {
+        // chunk table: original chunk c lies in original group c*16/G, which is slab group j with perm[j] = that group
+        const int n_c = C / 16, cpg = G / 16;
+        int32_t *ent = (int32_t *)malloc(sizeof(int32_t) * n_c * 2);
+        for (int j = 0; j < n_g; ++j)
+            for (int i = 0; i < cpg; ++i) {
+                ent[perm[j] * cpg + i] = (j * cpg + i) | ((int32_t)L->sx_host[j] << 24);
+                ent[n_c + j * cpg + i] = (j * cpg + i) | ((int32_t)L->sx_host[j] << 24);
+            }
+        cudaError_t e1 = cudaMalloc(&L->chunk_ent, sizeof(int32_t) * n_c);
+        if (e1 == cudaSuccess) e1 = cudaMalloc(&L->chunk_ent_slab, sizeof(int32_t) * n_c);
+        if (e1 == cudaSuccess) e1 = cudaMemcpy(L->chunk_ent, ent, sizeof(int32_t) * n_c, cudaMemcpyHostToDevice);
+        if (e1 == cudaSuccess) e1 = cudaMemcpy(L->chunk_ent_slab, ent + n_c, sizeof(int32_t) * n_c, cudaMemcpyHostToDevice);
+        free(ent);
+        TRY_OR_FREE(e1);
+    }
     TRY_OR_FREE(cudaMemcpyAsync(L->w_scale, w_scale, sizeof(float) * N, cudaMemcpyDeviceToDevice, stream));
     if (bias) TRY_OR_FREE(cudaMemcpyAsync(L->bias, bias, sizeof(float) * N, cudaMemcpyDeviceToDevice, stream));
     const long long total = (long long)n_g * N;
