@@ -218,6 +218,22 @@ int flexiq_mixed_conv_to_slab(flexiq_layer_t layer, const uint8_t *X4_dev, const
                               flexiq_layer_t next_layer, float next_x_scale, int relu,
                               int out_order, uint8_t *next_X4_dev, void *stream);
 
+/* direction of flexiq_reorder_channels */
+#define FLEXIQ_REORDER_TO_SLAB 0   /* original channel order -> the layer's slab order */
+#define FLEXIQ_REORDER_FROM_SLAB 1 /* the layer's slab order -> original channel order  */
+
+/* Residual-branch reorder operator (Sec. 5, layout post-processing step 3): copies a tensor
+ * while moving whole channel groups between the original channel order and the slab order of
+ * `layer` (its K / Cin channels, groups of G), for tensors that travel on a residual connection
+ * around layers whose outputs were permuted offline.
+ *   TO_SLAB  : Y[m][j*G + i] = X[m][group_perm[j]*G + i]
+ *   FROM_SLAB: Y[m][group_perm[j]*G + i] = X[m][j*G + i]
+ *   X_dev, Y_dev  [M][K] elements of elem_bytes in {1, 2, 4} (int8, fp16/bf16, fp32/int32),
+ *                 row-major, 16-byte aligned, distinct buffers (not in place)
+ * The values are not interpreted.  M == 0 is a successful no-op. */
+int flexiq_reorder_channels(flexiq_layer_t layer, const void *X_dev, int elem_bytes, int64_t M,
+                            int direction, void *Y_dev, void *stream);
+
 /* Test hooks: copy the layer's derived tables to host buffers (any may be NULL).
  *   sw_host [K/G][N] uint8 weight extraction positions (slab order),
  *   w8_host [N][Kw] int8 slab-order weights, w4_host [N][Kw/2] packed 4-bit weights,

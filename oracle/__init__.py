@@ -235,3 +235,12 @@ def epilogue_f32(acc, x_scale, w_scale, bias) -> np.ndarray:
     lib().fqo_epilogue_f32(_p(a2), C.c_int64(a2.shape[0]), N, C.c_float(x_scale), _p(w_scale),
                            _p(b) if b is not None else None, _p(out))
     return out.reshape(acc.shape)
+
+
+def reorder_channels(x, G: int, perm, to_slab: bool = True) -> np.ndarray:
+    x = np.ascontiguousarray(x)
+    K = x.shape[-1]
+    perm = _c(perm, np.int32)
+    y = np.empty_like(x)
+    lib().fqo_reorder_channels(_p(x), C.c_int64(x.size // K), K, G, x.itemsize, _p(perm), int(bool(to_slab)), _p(y))
+    return y

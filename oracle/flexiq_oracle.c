@@ -433,6 +433,22 @@ void fqo_epilogue_f32(const int32_t *acc, int64_t M, int N, float x_scale, const
         }
 }
 
+/* Residual-branch reorder (Sec. 5, layout post-processing step 3): the channels of a tensor are
+ * moved group by group between the original order and a layer's slab order, values untouched.
+ * to_slab != 0:  y[m][j*G + i] = x[m][perm[j]*G + i];  else  y[m][perm[j]*G + i] = x[m][j*G + i].
+ * Elements are elem_bytes wide and copied byte by byte. */
+void fqo_reorder_channels(const uint8_t *x, int64_t M, int K, int G, int elem_bytes, const int32_t *perm,
+                          int to_slab, uint8_t *y)
+{
+    for (int64_t m = 0; m < M; ++m)
+        for (int j = 0; j < K / G; ++j)
+            for (int i = 0; i < G; ++i) {
+                const int64_t slab = m * K + (int64_t)j * G + i, orig = m * K + (int64_t)perm[j] * G + i;
+                const int64_t dst = to_slab ? slab : orig, src = to_slab ? orig : slab;
+                for (int b = 0; b < elem_bytes; ++b) y[dst * elem_bytes + b] = x[src * elem_bytes + b];
+            }
+}
+
 int fqo_max_threads(void)
 {
 #ifdef _OPENMP

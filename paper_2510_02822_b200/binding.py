@@ -18,12 +18,13 @@ DTYPE_F32, DTYPE_F16, DTYPE_BF16, DTYPE_I8 = 0, 1, 2, 3
 OUT_ACC_I32, OUT_REQUANT_I8, OUT_DEQUANT_F32 = 0, 1, 2
 LOWBIT_MASKED_I8, LOWBIT_PACKED_U4 = 0, 1
 ORDER_ORIGINAL, ORDER_NEXT_SLAB = 0, 1
+REORDER_TO_SLAB, REORDER_FROM_SLAB = 0, 1
 
 EXPORTS = [
     "flexiq_layer_create_linear", "flexiq_layer_create_conv", "flexiq_layer_destroy",
     "flexiq_layer_set_lowbit_path", "flexiq_set_lowbit_ratio", "flexiq_get_max_4bit_ch",
     "flexiq_x4_pitch", "flexiq_quantize_lower", "flexiq_quantize_lower_dynamic_noalloc", "flexiq_mixed_gemm", "flexiq_mixed_conv",
-    "flexiq_mixed_gemm_to_slab", "flexiq_mixed_conv_to_slab",
+    "flexiq_mixed_gemm_to_slab", "flexiq_mixed_conv_to_slab", "flexiq_reorder_channels",
     "flexiq_layer_export", "flexiq_force_tile", "flexiq_check_status", "flexiq_last_error",
 ]
 
@@ -60,6 +61,7 @@ def lib():
         L.flexiq_mixed_conv.argtypes = [vp, vp, vp, vp, i32, i32, i32, f32, f32, i32, vp, vp]
         L.flexiq_mixed_gemm_to_slab.argtypes = [vp, vp, vp, vp, i64, f32, vp, f32, i32, i32, vp, vp]
         L.flexiq_mixed_conv_to_slab.argtypes = [vp, vp, vp, vp, i32, i32, i32, f32, vp, f32, i32, i32, vp, vp]
+        L.flexiq_reorder_channels.argtypes = [vp, vp, i32, i64, i32, vp, vp]
         L.flexiq_layer_export.argtypes = [vp, vp, vp, vp]
         L.flexiq_check_status.argtypes = [vp]
         _lib = L
@@ -160,6 +162,10 @@ def flexiq_mixed_conv_to_slab(h, X4_dev, X8_dev, x_shift_dev, Nb, H, W, x_scale,
                                            next_x_scale, int(relu), out_order, _ptr(next_X4_dev), _stream()))
 
 
+def flexiq_reorder_channels(h, X_dev, elem_bytes, M, direction, Y_dev):
+    _check(lib().flexiq_reorder_channels(h, _ptr(X_dev), elem_bytes, M, direction, _ptr(Y_dev), _stream()))
+
+
 def flexiq_layer_export(h, sw_host=None, w8_host=None, w4_host=None):
     def hp(a):
         return None if a is None else a.ctypes.data_as(C.c_void_p)
@@ -252,6 +258,14 @@ class Layer:
             dt = {OUT_ACC_I32: torch.int32, OUT_REQUANT_I8: torch.int8, OUT_DEQUANT_F32: torch.float32}[out_mode]
             Y = torch.empty((M, self.N), dtype=dt, device=self.device)
         flexiq_mixed_gemm(self.h, x4, x8, x_shift, M, x_scale, y_scale, out_mode, Y)
+        return Y
+
+    def reorder_channels(self, X, direction=REORDER_TO_SLAB, Y=None):
+        """Residual-branch reorder of a [..., K] tensor between original and slab channel order."""
+        import torch
+        if Y is None:
+            Y = torch.empty_like(X)
+        flexiq_reorder_channels(self.h, X, X.element_size(), X.numel() // self.K, direction, Y)
         return Y
 
     def mixed_gemm_to_slab(self, x4, x8, M, x_scale, nxt, next_x_scale, relu=False, slab=None, x_shift=None, out_order=ORDER_ORIGINAL):

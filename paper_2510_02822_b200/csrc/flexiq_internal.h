@@ -43,6 +43,7 @@ struct Layer {
     uint8_t *sw;     // [n_g][N] weight extraction positions
     uint8_t *sx;     // [n_g] static activation positions, slab order
     int32_t *perm;   // [n_g]
+    int32_t *inv_perm;  // [n_g] slab position of each original group
     // where a producer that writes this layer's masked slab directly puts each 16-channel chunk of
     // the original channel order, and the static position of the chunk's group
     int32_t *chunk_ent;       // [C/16] by original chunk: slab position in chunks | position of the group << 24

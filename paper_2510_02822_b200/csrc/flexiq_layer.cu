@@ -171,7 +171,7 @@ static void free_layer(Layer *L)
 {
     if (!L) return;
     cudaFree(L->w8); cudaFree(L->w8m); cudaFree(L->w4); cudaFree(L->wf); cudaFree(L->sw); cudaFree(L->sx);
-    cudaFree(L->perm); cudaFree(L->chunk_ent); cudaFree(L->chunk_ent_slab); cudaFree(L->w_scale); cudaFree(L->bias); cudaFree(L->alpha); cudaFree(L->beta);
+    cudaFree(L->perm); cudaFree(L->inv_perm); cudaFree(L->chunk_ent); cudaFree(L->chunk_ent_slab); cudaFree(L->w_scale); cudaFree(L->bias); cudaFree(L->alpha); cudaFree(L->beta);
     free(L->perm_host); free(L->sx_host);
     L->magic = 0;
     free(L);
@@ -258,6 +258,9 @@ static int create_common(flexiq_layer_t *out, int is_conv, int C, int N, int R, 
         if (e1 == cudaSuccess) e1 = cudaMalloc(&L->chunk_ent_slab, sizeof(int32_t) * n_c);
         if (e1 == cudaSuccess) e1 = cudaMemcpy(L->chunk_ent, ent, sizeof(int32_t) * n_c, cudaMemcpyHostToDevice);
         if (e1 == cudaSuccess) e1 = cudaMemcpy(L->chunk_ent_slab, ent + n_c, sizeof(int32_t) * n_c, cudaMemcpyHostToDevice);
+        if (e1 == cudaSuccess) e1 = cudaMalloc(&L->inv_perm, sizeof(int32_t) * n_g);
+        for (int j = 0; j < n_g; ++j) ent[perm[j]] = j;
+        if (e1 == cudaSuccess) e1 = cudaMemcpy(L->inv_perm, ent, sizeof(int32_t) * n_g, cudaMemcpyHostToDevice);
         free(ent);
         TRY_OR_FREE(e1);
     }

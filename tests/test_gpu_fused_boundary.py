@@ -156,3 +156,27 @@ def test_argument_errors(dev):
     assert e.value.code == fx.ERR_UNSUPPORTED
     for L in (A, B, A2):
         L.close()
+
+
+@pytest.mark.parametrize("M,K,G,dt", [(300, 256, 16, torch.int8), (129, 192, 32, torch.float16), (1000, 768, 16, torch.float32),
+                                      (1, 64, 64, torch.int8), (12608, 768, 16, torch.int8)])
+def test_residual_reorder(dev, M, K, G, dt):
+    rng = np.random.default_rng(M + K)
+    perm = rng.permutation(K // G).astype(np.int32)
+    Wq = torch.zeros((K, 16), dtype=torch.int8, device=dev)
+    L = fx.Layer(Wq, torch.ones(16, device=dev), torch.zeros(16, device=dev), perm, np.zeros(K // G, np.uint8), G)
+    X = torch.from_numpy(rng.integers(-120, 120, (M, K)).astype(np.int32)).to(dt).to(dev)
+    xn = X.cpu().numpy()
+    Y, guard_ok = helpers.with_guard(torch, (M, K), dt, dev)
+    L.reorder_channels(X, fx.REORDER_TO_SLAB, Y=Y)
+    torch.cuda.synchronize()
+    guard_ok()
+    assert np.array_equal(Y.cpu().numpy(), oracle.reorder_channels(xn, G, perm, True))
+    Z = L.reorder_channels(X, fx.REORDER_FROM_SLAB)
+    assert np.array_equal(Z.cpu().numpy(), oracle.reorder_channels(xn, G, perm, False))
+    assert torch.equal(L.reorder_channels(Y, fx.REORDER_FROM_SLAB), X)
+    with pytest.raises(fx.FlexiqError):
+        fx.flexiq_reorder_channels(L.h, X, X.element_size(), M, fx.REORDER_TO_SLAB, X)  # in place
+    with pytest.raises(fx.FlexiqError):
+        fx.flexiq_reorder_channels(L.h, X, 3, M, fx.REORDER_TO_SLAB, Y)
+    L.close()

@@ -287,6 +287,27 @@ def test_slab_format():
     assert oracle.x4_pitch(16) == 16 and oracle.x4_pitch(96) == 48 and oracle.x4_pitch(48) == 32
 
 
+def test_residual_reorder_moves_whole_groups():
+    # hand case (Sec. 5 step 3): three groups of 2 channels, slab group j holds original group perm[j]
+    x = np.array([[10, 11, 20, 21, 30, 31]], np.int8)
+    perm = np.array([2, 0, 1], np.int32)
+    assert oracle.reorder_channels(x, 2, perm, True).tolist() == [[30, 31, 10, 11, 20, 21]]
+    assert oracle.reorder_channels(x, 2, perm, False).tolist() == [[20, 21, 30, 31, 10, 11]]
+    rng = np.random.default_rng(7)
+    for dt in (np.int8, np.float16, np.float32):
+        G, n_g, M = 16, 12, 9
+        X = rng.integers(-100, 100, (M, G * n_g)).astype(dt)
+        perm = rng.permutation(n_g).astype(np.int32)
+        cols = np.concatenate([np.arange(g * G, (g + 1) * G) for g in perm])
+        Y = oracle.reorder_channels(X, G, perm, True)
+        assert np.array_equal(Y, X[:, cols])                                     # a column gather
+        assert np.array_equal(oracle.reorder_channels(Y, G, perm, False), X)     # and its inverse
+    # the 8-bit slab of the prologue at ratio 0 is the same gather
+    q = rng.integers(-128, 128, (5, 64)).astype(np.int8)
+    perm = rng.permutation(4).astype(np.int32)
+    assert np.array_equal(oracle.make_slabs(q, 16, perm, np.zeros(4, np.uint8), 0)[1], oracle.reorder_channels(q, 16, perm, True))
+
+
 # ------------------------------------------------------------------ epilogue
 def test_epilogue_identity_scale_is_a_clip():
     acc = np.array([[-300, -128, -1, 0, 1, 127, 128, 100000] * 2], np.int32)
