@@ -42,7 +42,8 @@ constexpr uint32_t kSpinLimit = 1u << 21;              // parked waits of <= 1 u
 constexpr int kStageRegion = 196608;                  // shared memory given to the operand ring
 constexpr int kFactorsPerWarp = 512;                  // alpha[64] | beta[64] of the warp's columns in the current tile
 constexpr int kMaxStages = 8;
-constexpr int kSmemBytes = kStageRegion + kNumWorkWarps * kFactorsPerWarp + 256;
+constexpr int kStoreStagePerWarp = 1024;              // 32 rows x 32 int8 columns staged for a tiled bulk store
+constexpr int kSmemBytes = kStageRegion + kNumWorkWarps * (kFactorsPerWarp + kStoreStagePerWarp) + 256;
 
 // Internal epilogue mode of the fused layer boundary: the int8 result goes straight into the
 // next layer's masked slab (its channel order, its low groups lowered).
@@ -70,6 +71,7 @@ struct GemmParams {
     const int32_t *next_ent;   // [N/16] slab position (in chunks) of original chunk c | its group's position << 24
     int next_K_lo;             // the next layer's max_4bit_ch
     int relu;                  // clamp at zero before the re-quantization
+    int tma_store;             // int8 output leaves through shared memory and tiled bulk stores (mapY)
     // packed low-bit path only: positions the expander warps shift the 4-bit values back to
     const uint8_t *sx;   // [n_g] activation positions, slab order
     const uint8_t *sw;   // [n_g][N] weight positions
@@ -213,6 +215,8 @@ struct EpilogueCtx {
     uint64_t *tmem_full, *tmem_empty;
     volatile int *abort_flag;
     float *fac;
+    uint32_t store_stage;         // this warp's 1 KB of shared memory for staged stores
+    const CUtensorMap *map_y, *map_y16;   // boxes of 32 rows x 32 columns (32-byte swizzle) and 32 x 16 (plain)
     int first_tile, tile_step, num_tiles;
     int parts, arrivals_on;  // column parts per tile (4 or 2); this warp arrives on the accumulator barrier
 };
@@ -286,6 +290,39 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
 #pragma unroll
                 for (int g = 0; g < 4; ++g) ents[g] = __shfl_sync(0xffffffffu, ent, g);
             }
+            if (MODE == FLEXIQ_OUT_REQUANT_I8 && p.tma_store) {
+                // Each warp stages 32 rows x 32 columns (1 KB, 32-byte swizzle: no bank conflicts) and one
+                // lane hands them to a tiled bulk store, which writes whole sectors asynchronously and
+                // drops the rows and columns that lie outside Y.
+                const long long row0 = row - lane;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t *r = h == 0 ? ra : rb;
+                    const int n = nw + 32 * h;
+                    if (32 * h < cols && n < p.N && row0 < p.M) {   // warp-uniform
+                        const bool both = 32 * h + 16 < cols && n + 16 < p.N;  // a 32-column box, else a 16-column one
+                        uint32_t w[8];
+                        finish16<MODE>(r, x.fac + 32 * h, x.fac + 64 + 32 * h, w);
+                        if (both) finish16<MODE>(r + 16, x.fac + 32 * h + 16, x.fac + 64 + 32 * h + 16, w + 4);
+                        if (lane == 0) ptx::bulk_wait_read_all();    // the previous store has read the buffer
+                        __syncwarp();
+                        if (both) {
+                            const uint32_t dst = x.store_stage + (uint32_t)lane * 32u;
+                            const uint32_t sw16 = ((uint32_t)lane >> 2 & 1u) << 4;
+                            ptx::st_shared_128(dst + sw16, w[0], w[1], w[2], w[3]);
+                            ptx::st_shared_128(dst + (sw16 ^ 16u), w[4], w[5], w[6], w[7]);
+                        } else {
+                            ptx::st_shared_128(x.store_stage + (uint32_t)lane * 16u, w[0], w[1], w[2], w[3]);
+                        }
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            ptx::tma_store_2d(both ? x.map_y : x.map_y16, x.store_stage, n, (int)row0);
+                            ptx::bulk_commit_group();
+                        }
+                    }
+                }
+            } else
             if (row < p.M) {
                 uint8_t *yrow = static_cast<uint8_t *>(p.Y) + (row * p.N + nw) * kElem;
 #pragma unroll
@@ -361,6 +398,7 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
         }
         if ((buf ^= 1) == 0) buf_phase ^= 1;
     }
+    if (MODE == FLEXIQ_OUT_REQUANT_I8 && p.tma_store && lane == 0) ptx::bulk_wait_all();  // the staged stores are performed
     if (quad == 2 && part == 0 && lane == 0) { PROF_STORE(8, prof_wait); PROF_STORE(9, clock64() - prof_start); PROF_STORE(10, prof_ld); PROF_STORE(11, prof_math); }
 }
 
@@ -374,6 +412,7 @@ template <int CG, int PK>
 __global__ void __launch_bounds__(kThreads, 1)
 mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_constant__ CUtensorMap mapA_hi,
                   const __grid_constant__ CUtensorMap mapB_lo, const __grid_constant__ CUtensorMap mapB_hi,
+                  const __grid_constant__ CUtensorMap mapY, const __grid_constant__ CUtensorMap mapY16,
                   const GemmParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -383,7 +422,8 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
     }
     uint8_t *stage_base = smem;
     uint8_t *factors = smem + kStageRegion;
-    uint64_t *full_bar = reinterpret_cast<uint64_t *>(factors + kNumWorkWarps * kFactorsPerWarp);
+    uint8_t *store_stage = factors + kNumWorkWarps * kFactorsPerWarp;  // 1024-byte aligned: the bulk stores' swizzle needs it
+    uint64_t *full_bar = reinterpret_cast<uint64_t *>(store_stage + kNumWorkWarps * kStoreStagePerWarp);
     uint64_t *empty_bar = full_bar + kMaxStages;
     uint64_t *tmem_full = empty_bar + kMaxStages;
     uint64_t *tmem_empty = tmem_full + 2;
@@ -669,6 +709,8 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             x.tmem_base = tmem_base; x.buf_stride = buf_stride; x.cta_rank = cta_rank;
             x.tmem_full = tmem_full; x.tmem_empty = tmem_empty; x.abort_flag = abort_flag;
             x.fac = reinterpret_cast<float *>(factors + e * kFactorsPerWarp);  // alpha[64] | beta[64]
+            x.store_stage = ptx::smem_u32(store_stage + e * kStoreStagePerWarp);
+            x.map_y = &mapY; x.map_y16 = &mapY16;
             x.first_tile = first_tile; x.tile_step = tile_step; x.num_tiles = num_tiles;
             x.parts = kEpiWarps / 4; x.arrivals_on = 1;
             if (p.out_mode == FLEXIQ_OUT_REQUANT_I8) epilogue_role<CG, FLEXIQ_OUT_REQUANT_I8>(p, x, warp & 3, e >> 2, lane);
@@ -834,6 +876,14 @@ __global__ void scale_vectors_kernel(int N, float x_scale, float y_scale, int re
 // configuration listed first).  cost = waves * tile time.
 struct TileChoice { int cg, bn; };
 static TileChoice g_forced_tile{0, 0};  // test hook: 0 = choose automatically
+static bool direct_stores_only()
+{
+#ifdef FLEXIQ_PROFILE
+    return getenv("FLEXIQ_DIRECT_STORES") != nullptr;  // A/B timing in the profiling build
+#else
+    return false;
+#endif
+}
 static TileChoice choose_tile(long long M, int N, int k_blocks, int sms)
 {
     const int bns[4] = {256, 192, 128, 64};
@@ -882,7 +932,7 @@ static int make_map_im2col(CUtensorMap *map, const void *base, int Cpart, long l
 
 template <int CG, int PK>
 static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const CUtensorMap &b_lo, const CUtensorMap &b_hi,
-                         const GemmParams &p, int sms, cudaStream_t st)
+                         const CUtensorMap &y_map, const CUtensorMap &y_map16, const GemmParams &p, int sms, cudaStream_t st)
 {
     static bool attr_set[64] = {};
     int dev = 0;
@@ -908,7 +958,7 @@ static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    FLEXIQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, mixed_gemm_kernel<CG, PK>, a_lo, a_hi, b_lo, b_hi, p));
+    FLEXIQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, mixed_gemm_kernel<CG, PK>, a_lo, a_hi, b_lo, b_hi, y_map, y_map16, p));
     return FLEXIQ_OK;
 }
 
@@ -1051,10 +1101,18 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
         }
         if (C_hi == 0) a_hi = a_lo;
     }
+    // int8 output leaves through staged tiled bulk stores
+    CUtensorMap y_map = a_hi, y_map16 = a_hi;
+    p.tma_store = 0;
+    if (out_mode == FLEXIQ_OUT_REQUANT_I8 && !direct_stores_only()) {
+        if (L->N >= 32 && (rc = make_map_2d(&y_map, Y, (uint64_t)L->N, (uint64_t)M, (uint64_t)L->N, 32, 32, 32))) return rc;
+        if ((rc = make_map_2d(&y_map16, Y, (uint64_t)L->N, (uint64_t)M, (uint64_t)L->N, 16, 32, 0))) return rc;
+        p.tma_store = 1;
+    }
     const int bi = weight_map_index(bn / cg);  // box rows = the B rows one CTA loads
-    if (packed) return launch_kernel<1, 1>(a_lo, a_hi, L->map_w4[bi], L->map_w8[bi], p, sms, st);
-    if (cg == 2) return launch_kernel<2, 0>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], p, sms, st);
-    return launch_kernel<1, 0>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], p, sms, st);
+    if (packed) return launch_kernel<1, 1>(a_lo, a_hi, L->map_w4[bi], L->map_w8[bi], y_map, y_map16, p, sms, st);
+    if (cg == 2) return launch_kernel<2, 0>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], y_map, y_map16, p, sms, st);
+    return launch_kernel<1, 0>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], y_map, y_map16, p, sms, st);
 }
 
 }  // namespace flexiq
