@@ -218,6 +218,43 @@ int flexiq_mixed_conv_to_slab(flexiq_layer_t layer, const uint8_t *X4_dev, const
                               flexiq_layer_t next_layer, float next_x_scale, int relu,
                               int out_order, uint8_t *next_X4_dev, void *stream);
 
+/* ---- Calibration on the device (off the hot path; produces what flexiq_layer_create_* takes) ----
+ *
+ * flexiq_calib_channel_ranges: per input channel the range [lo, hi] (lo <= 0 <= hi) of the
+ *   Eq. 1-quantized calibration activations X_dev [M][K] ("estimating the value ranges of the
+ *   activation channels using sampled calibration data", Sec. 4.2).  accumulate != 0 merges into
+ *   the ranges already in lo_dev / hi_dev (several calibration batches); 0 starts from [0, 0].
+ *   lo_dev, hi_dev: [K] int32.  K % 16 == 0.
+ * flexiq_calib_weight_absmax: wmax_dev[k] = max |w| over the output channels (and taps) of input
+ *   channel k ("the corresponding weight parameters' channels across the output channel dimension
+ *   to determine the maximum value range", Sec. 4.2).  Linear: Wq_dev [K][N], taps ignored;
+ *   convolution (is_conv != 0): Wq_dev [N][taps][K].
+ * flexiq_calib_prepare: from those three tables, per channel group of group_size channels
+ *     x_shift_dev[g]  static extraction position of ORIGINAL group g: that of its widest channel
+ *                     (Sec. 4.1; used magnitude bits L -> max(0, L - 3))
+ *     score_dev[g]    error-estimation score: max over the group's channels of
+ *                     max(hi, -lo) * wmax (Sec. 4.2), int64
+ *     perm_dev        groups by ascending score, ties by index: the greedy nested order whose
+ *                     prefixes are the low-bit sets (Sec. 4.2 / Sec. 5), int32 [K/group_size]
+ *     unused_hist_dev [5] number of channels with 0, 1, 2, 3, >= 4 unused magnitude bits (Sec. 8.4)
+ *   perm_dev and x_shift_dev, copied to the host, are the group_perm_host / x_shift_host of
+ *   flexiq_layer_create_*.
+ * flexiq_calib_absmax_ema: activation range across batches by exponential moving average
+ *   (Sec. 7: momentum 0.99).  state_dev: 4 floats, zeroed by the caller before the first batch;
+ *   after each call state_dev[0] = momentum * previous + (1 - momentum) * max|x| of this batch
+ *   (the first batch sets it to its max|x|), state_dev[1] = batches seen.  x_scale = state[0] / 127.
+ *   count = number of elements, a multiple of 16; floating-point x_dtype only.
+ * All enqueue on `stream`, allocate nothing and return the usual codes. */
+int flexiq_calib_channel_ranges(const void *X_dev, int x_dtype, int64_t M, int K, float x_scale,
+                                int accumulate, int32_t *lo_dev, int32_t *hi_dev, void *stream);
+int flexiq_calib_weight_absmax(const int8_t *Wq_dev, int is_conv, int K, int N, int taps,
+                               int32_t *wmax_dev, void *stream);
+int flexiq_calib_prepare(const int32_t *lo_dev, const int32_t *hi_dev, const int32_t *wmax_dev, int K,
+                         int group_size, int32_t *perm_dev, uint8_t *x_shift_dev, int64_t *score_dev,
+                         int32_t *unused_hist_dev, void *stream);
+int flexiq_calib_absmax_ema(const void *X_dev, int x_dtype, int64_t count, float momentum,
+                            float *state_dev, void *stream);
+
 /* direction of flexiq_reorder_channels */
 #define FLEXIQ_REORDER_TO_SLAB 0   /* original channel order -> the layer's slab order */
 #define FLEXIQ_REORDER_FROM_SLAB 1 /* the layer's slab order -> original channel order  */

@@ -244,3 +244,19 @@ def reorder_channels(x, G: int, perm, to_slab: bool = True) -> np.ndarray:
     y = np.empty_like(x)
     lib().fqo_reorder_channels(_p(x), C.c_int64(x.size // K), K, G, x.itemsize, _p(perm), int(bool(to_slab)), _p(y))
     return y
+
+
+def unused_bits_histogram(lo, hi) -> np.ndarray:
+    lo = _c(lo, np.int32)
+    hi = _c(hi, np.int32)
+    hist = np.zeros(5, np.int32)
+    lib().fqo_unused_bits_histogram(_p(lo), _p(hi), lo.size, _p(hist))
+    return hist
+
+
+def absmax_ema(x_batches, momentum: float) -> float:
+    x = _c(x_batches, np.float32)
+    b = x.shape[0]
+    f = lib().fqo_absmax_ema
+    f.restype = C.c_float
+    return float(f(_p(x), C.c_int64(b), C.c_int64(x.size // b), C.c_float(momentum)))

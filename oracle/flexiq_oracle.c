@@ -449,6 +449,41 @@ void fqo_reorder_channels(const uint8_t *x, int64_t M, int K, int G, int elem_by
             }
 }
 
+/* Unused-bit statistics (Sec. 8.4): an int8 value has 7 magnitude bits; a channel whose range needs
+ * L of them leaves 7 - L unused ("maximum is less than 32 => the highest two bits are not used",
+ * Sec. 4.1).  hist[u] counts the channels with u unused bits, u = 4 standing for four or more. */
+void fqo_unused_bits_histogram(const int32_t *lo, const int32_t *hi, int K, int32_t *hist /*[5]*/)
+{
+    for (int u = 0; u < 5; ++u) hist[u] = 0;
+    for (int c = 0; c < K; ++c) {
+        int u = 7 - fqo_used_bits_from_range(lo[c], hi[c]);
+        hist[u > 4 ? 4 : u] += 1;
+    }
+}
+
+/* Activation range across batches by exponential moving average (Sec. 7, momentum 0.99): the first
+ * batch sets the state to its max |x|; batch b > 0 gives state = m * state + (1 - m) * max|x_b|,
+ * every operation rounded to fp32. */
+float fqo_absmax_ema(const float *x, int64_t batches, int64_t per_batch, float momentum)
+{
+    volatile float state = 0.0f;
+    for (int64_t b = 0; b < batches; ++b) {
+        float a = 0.0f;
+        for (int64_t i = 0; i < per_batch; ++i) {
+            float v = fabsf(x[b * per_batch + i]);
+            if (v > a) a = v;
+        }
+        if (b == 0) state = a;
+        else {
+            volatile float t1 = momentum * state;
+            volatile float om = 1.0f - momentum;
+            volatile float t2 = om * a;
+            state = t1 + t2;
+        }
+    }
+    return state;
+}
+
 int fqo_max_threads(void)
 {
 #ifdef _OPENMP

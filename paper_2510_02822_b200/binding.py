@@ -25,6 +25,7 @@ EXPORTS = [
     "flexiq_layer_set_lowbit_path", "flexiq_set_lowbit_ratio", "flexiq_get_max_4bit_ch",
     "flexiq_x4_pitch", "flexiq_quantize_lower", "flexiq_quantize_lower_dynamic_noalloc", "flexiq_mixed_gemm", "flexiq_mixed_conv",
     "flexiq_mixed_gemm_to_slab", "flexiq_mixed_conv_to_slab", "flexiq_reorder_channels",
+    "flexiq_calib_channel_ranges", "flexiq_calib_weight_absmax", "flexiq_calib_prepare", "flexiq_calib_absmax_ema",
     "flexiq_layer_export", "flexiq_force_tile", "flexiq_check_status", "flexiq_last_error",
 ]
 
@@ -62,6 +63,10 @@ def lib():
         L.flexiq_mixed_gemm_to_slab.argtypes = [vp, vp, vp, vp, i64, f32, vp, f32, i32, i32, vp, vp]
         L.flexiq_mixed_conv_to_slab.argtypes = [vp, vp, vp, vp, i32, i32, i32, f32, vp, f32, i32, i32, vp, vp]
         L.flexiq_reorder_channels.argtypes = [vp, vp, i32, i64, i32, vp, vp]
+        L.flexiq_calib_channel_ranges.argtypes = [vp, i32, i64, i32, f32, i32, vp, vp, vp]
+        L.flexiq_calib_weight_absmax.argtypes = [vp, i32, i32, i32, i32, vp, vp]
+        L.flexiq_calib_prepare.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]
+        L.flexiq_calib_absmax_ema.argtypes = [vp, i32, i64, f32, vp, vp]
         L.flexiq_layer_export.argtypes = [vp, vp, vp, vp]
         L.flexiq_check_status.argtypes = [vp]
         _lib = L
@@ -164,6 +169,23 @@ def flexiq_mixed_conv_to_slab(h, X4_dev, X8_dev, x_shift_dev, Nb, H, W, x_scale,
 
 def flexiq_reorder_channels(h, X_dev, elem_bytes, M, direction, Y_dev):
     _check(lib().flexiq_reorder_channels(h, _ptr(X_dev), elem_bytes, M, direction, _ptr(Y_dev), _stream()))
+
+
+def flexiq_calib_channel_ranges(X_dev, x_dtype, M, K, x_scale, accumulate, lo_dev, hi_dev):
+    _check(lib().flexiq_calib_channel_ranges(_ptr(X_dev), x_dtype, M, K, x_scale, int(accumulate), _ptr(lo_dev), _ptr(hi_dev), _stream()))
+
+
+def flexiq_calib_weight_absmax(Wq_dev, is_conv, K, N, taps, wmax_dev):
+    _check(lib().flexiq_calib_weight_absmax(_ptr(Wq_dev), int(is_conv), K, N, taps, _ptr(wmax_dev), _stream()))
+
+
+def flexiq_calib_prepare(lo_dev, hi_dev, wmax_dev, K, G, perm_dev, x_shift_dev, score_dev, hist_dev):
+    _check(lib().flexiq_calib_prepare(_ptr(lo_dev), _ptr(hi_dev), _ptr(wmax_dev), K, G, _ptr(perm_dev), _ptr(x_shift_dev),
+                                      _ptr(score_dev), _ptr(hist_dev), _stream()))
+
+
+def flexiq_calib_absmax_ema(X_dev, x_dtype, count, momentum, state_dev):
+    _check(lib().flexiq_calib_absmax_ema(_ptr(X_dev), x_dtype, count, momentum, _ptr(state_dev), _stream()))
 
 
 def flexiq_layer_export(h, sw_host=None, w8_host=None, w4_host=None):

@@ -54,3 +54,35 @@ def permute_outputs_for_next(Wq: torch.Tensor, w_scale: torch.Tensor, bias, next
     cols = torch.cat([torch.arange(int(g) * next_G, (int(g) + 1) * next_G) for g in next_perm]).to(Wq.device)
     Wp = Wq.index_select(0 if conv else 1, cols).contiguous()
     return Wp, w_scale.index_select(0, cols).contiguous(), None if bias is None else bias.index_select(0, cols).contiguous()
+
+
+def static_preparation_device(Xcal: torch.Tensor, x_scale: float, Wq: torch.Tensor, G: int, conv: bool = False, batches: int = 1):
+    """The same preparation with the library's calibration kernels, on device tensors.
+
+    Xcal: calibration activations [..., C] (fp32 / fp16 / bf16 / int8) on the GPU; Wq as in
+    static_preparation, on the GPU.  The rows are fed in `batches` accumulating calls.
+    Returns (group_perm, x_shift, info) with info = {lo, hi, wmax, score, unused_hist} (torch tensors)."""
+    from . import binding as fx
+    dev = Xcal.device
+    C = Xcal.shape[-1]
+    X2 = Xcal.reshape(-1, C)
+    lo = torch.empty(C, dtype=torch.int32, device=dev)
+    hi = torch.empty(C, dtype=torch.int32, device=dev)
+    rows = X2.shape[0]
+    step = (rows + batches - 1) // batches
+    for b in range(batches):
+        part = X2[b * step:(b + 1) * step]
+        fx.flexiq_calib_channel_ranges(part, fx._dtype_code(part), part.shape[0], C, x_scale, b > 0, lo, hi)
+    wmax = torch.empty(C, dtype=torch.int32, device=dev)
+    if conv:
+        fx.flexiq_calib_weight_absmax(Wq, True, C, Wq.shape[0], Wq.shape[1] * Wq.shape[2], wmax)
+    else:
+        fx.flexiq_calib_weight_absmax(Wq, False, C, Wq.shape[1], 1, wmax)
+    n_g = C // G
+    perm = torch.empty(n_g, dtype=torch.int32, device=dev)
+    x_shift = torch.empty(n_g, dtype=torch.uint8, device=dev)
+    score = torch.empty(n_g, dtype=torch.int64, device=dev)
+    hist = torch.empty(5, dtype=torch.int32, device=dev)
+    fx.flexiq_calib_prepare(lo, hi, wmax, C, G, perm, x_shift, score, hist)
+    info = {"lo": lo, "hi": hi, "wmax": wmax, "score": score, "unused_hist": hist}
+    return np.ascontiguousarray(perm.cpu().numpy()), np.ascontiguousarray(x_shift.cpu().numpy()), info

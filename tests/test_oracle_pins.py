@@ -287,6 +287,25 @@ def test_slab_format():
     assert oracle.x4_pitch(16) == 16 and oracle.x4_pitch(96) == 48 and oracle.x4_pitch(48) == 32
 
 
+def test_unused_bit_histogram_and_ema():
+    # Sec. 4.1's two worked ranges: max < 32 leaves two magnitude bits unused, min > -16 three
+    lo = np.array([0, -15, -128, 0, -1, 0, -64, 0], np.int32)
+    hi = np.array([31, 0, 127, 0, 0, 7, 63, 64], np.int32)
+    #  used bits:   5    4    7   0   0   3    6   7   ->  unused 2, 3, 0, 7, 7, 4, 1, 0  (>= 4 counted together)
+    assert oracle.unused_bits_histogram(lo, hi).tolist() == [2, 1, 1, 1, 3]
+    # consistency with the extraction position: position = max(0, 4 - unused) for every int8 range
+    for l in range(-128, 1, 7):
+        for h in range(0, 128, 5):
+            u = int(np.argmax(oracle.unused_bits_histogram([l], [h])))
+            assert oracle.position_from_range(l, h) == max(0, 4 - u) or u == 4
+    # EMA: constant batches are a fixed point; momentum 0 follows the last batch; momentum 0.5 by hand
+    x = np.array([[1.0, -3.0], [2.0, 0.5], [-8.0, 1.0]], np.float32)
+    assert oracle.absmax_ema(np.tile(np.float32([[1.5, -2.5]]), (5, 1)), 0.99) == np.float32(2.5)
+    assert oracle.absmax_ema(x, 0.0) == 8.0
+    assert oracle.absmax_ema(x, 0.5) == 0.5 * (0.5 * 3.0 + 0.5 * 2.0) + 0.5 * 8.0
+    assert oracle.absmax_ema(x[:1], 0.99) == 3.0
+
+
 def test_residual_reorder_moves_whole_groups():
     # hand case (Sec. 5 step 3): three groups of 2 channels, slab group j holds original group perm[j]
     x = np.array([[10, 11, 20, 21, 30, 31]], np.int8)
