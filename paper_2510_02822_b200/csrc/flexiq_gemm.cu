@@ -994,8 +994,7 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
         return set_error(FLEXIQ_ERR_UNSUPPORTED, "packed low-bit convolution needs Cin %% 32 == 0 (TMA start alignment of the 4-bit weight taps)");
     int rc = check_device_sm100();
     if (rc) return rc;
-    int sms = 148;
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, L->device);
+    const int sms = device_sm_count(L->device);
 
     if (!packed) {
         // Masked path: activations are one slab [rows][C] and the weights one operand wf, so the
@@ -1076,9 +1075,15 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     // activation maps (per call: they depend on the caller's buffers, M and the ratio);
     // an empty slab borrows the other one's map and is never addressed
     CUtensorMap a_lo, a_hi;
-    if (!packed) {
+    const bool staged = out_mode == FLEXIQ_OUT_REQUANT_I8 && !direct_stores_only();
+    const void *slab = packed_path ? static_cast<const void *>(X8) : static_cast<const void *>(X4);
+    Layer::CallMaps &cm = L->call_maps;
+    const bool cached = !packed && cm.slab == slab && cm.M == M && cm.Nb == Nb && cm.H == H && cm.W == W && cm.bk == p.BK &&
+                        cm.im2col == (int)p.im2col && (!staged || (cm.staged && cm.Y == Y));
+    if (cached) {
+        a_lo = a_hi = cm.a;
+    } else if (!packed) {
         // one int8 slab [rows][C] (a packed-path layer at ratio 0 has it in X8_dev)
-        const void *slab = packed_path ? static_cast<const void *>(X8) : static_cast<const void *>(X4);
         if (p.im2col) {
             if ((rc = make_map_im2col(&a_hi, slab, L->C, L->C, Nb, H, W, L->R, L->S, L->stride, L->pad, p.BK, p.BK))) return rc;
         } else {
@@ -1103,11 +1108,17 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     }
     // int8 output leaves through staged tiled bulk stores
     CUtensorMap y_map = a_hi, y_map16 = a_hi;
-    p.tma_store = 0;
-    if (out_mode == FLEXIQ_OUT_REQUANT_I8 && !direct_stores_only()) {
+    p.tma_store = staged;
+    if (staged && cached) {
+        y_map = cm.y;
+        y_map16 = cm.y16;
+    } else if (staged) {
         if (L->N >= 32 && (rc = make_map_2d(&y_map, Y, (uint64_t)L->N, (uint64_t)M, (uint64_t)L->N, 32, 32, 32))) return rc;
         if ((rc = make_map_2d(&y_map16, Y, (uint64_t)L->N, (uint64_t)M, (uint64_t)L->N, 16, 32, 0))) return rc;
-        p.tma_store = 1;
+    }
+    if (!packed && !cached) {
+        cm.slab = slab; cm.Y = staged ? Y : nullptr; cm.M = M; cm.Nb = Nb; cm.H = H; cm.W = W; cm.bk = p.BK; cm.im2col = p.im2col;
+        cm.staged = staged; cm.a = a_hi; cm.y = y_map; cm.y16 = y_map16;
     }
     const int bi = weight_map_index(bn / cg);  // box rows = the B rows one CTA loads
     if (packed) return launch_kernel<1, 1>(a_lo, a_hi, L->map_w4[bi], L->map_w8[bi], y_map, y_map16, p, sms, st);

@@ -60,12 +60,21 @@ struct Layer {
     float cache_xs, cache_ys;
     int cache_mode;
     int w4_pitch;    // row pitch of w4 in bytes: Kw/2 rounded up to 16
+    // tensor maps of the most recent masked-path call, reused while the caller passes the same buffers
+    // and shapes (encoding three maps costs more host time than the rest of a small call)
+    struct CallMaps {
+        const void *slab, *Y;
+        long long M;
+        int Nb, H, W, bk, im2col, staged;
+        CUtensorMap a, y, y16;
+    } call_maps;
 };
 
 constexpr uint32_t kLayerMagic = 0x464c5851u;  // "FLXQ"
 
 int set_error(int code, const char *fmt, ...);
 int check_device_sm100();
+int device_sm_count(int device);  // cached per device
 Layer *as_layer(flexiq_layer_t h);
 
 // driver entry point for tensor-map encoding, resolved through the runtime

@@ -23,18 +23,32 @@ int set_error(int code, const char *fmt, ...)
 
 int check_device_sm100()
 {
+    static int major_of[64] = {};  // compute capability major per device ordinal, looked up once
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess)
         return set_error(FLEXIQ_ERR_CUDA, "cudaGetDevice failed: %s", cudaGetErrorString(e));
-    int major = 0;
-    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
-    if (e != cudaSuccess)
-        return set_error(FLEXIQ_ERR_CUDA, "cudaDeviceGetAttribute failed: %s", cudaGetErrorString(e));
+    int major = dev < 64 ? major_of[dev] : 0;
+    if (major == 0) {
+        e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        if (e != cudaSuccess)
+            return set_error(FLEXIQ_ERR_CUDA, "cudaDeviceGetAttribute failed: %s", cudaGetErrorString(e));
+        if (dev < 64) major_of[dev] = major;
+    }
     if (major != 10)
         return set_error(FLEXIQ_ERR_UNSUPPORTED,
                          "device compute capability %d.x is not sm_100; there is no fallback path", major);
     return FLEXIQ_OK;
+}
+
+int device_sm_count(int device)
+{
+    static int sms_of[64] = {};
+    if (device >= 0 && device < 64 && sms_of[device]) return sms_of[device];
+    int sms = 148;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device);
+    if (device >= 0 && device < 64) sms_of[device] = sms;
+    return sms;
 }
 
 Layer *as_layer(flexiq_layer_t h)

@@ -185,8 +185,7 @@ static int launch_prologue(Layer *L, const void *X, long long M, float S, int dy
 {
     const int K = L->C, G = L->G;
     const int n_c16 = K / 16;
-    int sms = 148;
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, L->device);
+    const int sms = device_sm_count(L->device);
     const int threads = 256;
     if (dynamic) {
         FLEXIQ_CUDA_TRY(cudaMemsetAsync(scratch, 0, sizeof(unsigned) * L->n_g, st));
