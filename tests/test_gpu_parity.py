@@ -294,3 +294,21 @@ def test_vit_b_full_size_sampled_rows(dev, layer):
         acc2 = L.mixed_gemm(x4, x8, case.M, case.x_scale, case.y_scale, fx.OUT_ACC_I32)
         assert torch.equal(acc, acc2)
     L.close()
+
+
+@pytest.mark.parametrize("K", [240, 256, 1024])
+def test_extreme_accumulators(dev, K):
+    """The largest accumulator magnitudes a layer can produce (all operands at -128 / 127) survive the
+    int32 -> fp32 -> int8 epilogue exactly, below and above 2^22 and 2^24."""
+    M, N, G = 200, 64, 16
+    case = inputs.ranged_linear("x", M, K, N, G, seed=K)
+    rng = np.random.default_rng(K)
+    case.Wq = np.where(rng.random((K, N)) < 0.5, -128, 127).astype(np.int8)
+    case.Wq[:, 0] = -128
+    case.Wq[:, 1] = 127
+    sgn = np.where(rng.random((M, K)) < 0.5, -1.0, 1.0).astype(np.float32)
+    sgn[0] = -1.0
+    sgn[1] = 1.0
+    case.X = (sgn * 200.0 * case.x_scale).astype(np.float32)  # quantizes to -128 / 127
+    case.y_scale = float(np.float32(K * 128.0))
+    _run_linear(case, dev, [0.0, 0.5, 1.0])
