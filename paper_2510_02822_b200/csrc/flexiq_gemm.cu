@@ -181,6 +181,27 @@ __device__ __forceinline__ void finish16_next(const uint32_t *r, const float *al
         out[i] = requant4(y0, y1, y2, y3) & mask;
     }
 }
+// One 16-channel chunk of the fused layer boundary.  `ent` = slab position (in chunks) | extraction position << 24.
+__device__ __forceinline__ void next_slab16(const GemmParams &p, int ent, const uint32_t *r, const float *alpha16, const float *beta16,
+                                            uint32_t *out)
+{
+    float lo = -128.f, hi = 127.f;
+    uint32_t mask = 0xffffffffu;
+    if ((ent & 0xffffff) * 16 < p.next_K_lo) {
+        const int sft = ent >> 24;
+        hi = (float)(8 << sft) - 1.f;
+        lo = -(float)(8 << sft);
+        mask = ((0xffu << sft) & 0xffu) * 0x01010101u;
+    }
+    if (p.relu) lo = fmaxf(lo, 0.f);
+    // the pack saturates to [-128, 127] by itself: clamp only when the range is narrower (warp-uniform)
+    if (lo > -128.f || hi < 127.f) finish16_next(r, alpha16, beta16, lo, hi, mask, out);
+    else {
+        finish16<FLEXIQ_OUT_REQUANT_I8>(r, alpha16, beta16, out);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) out[q] &= mask;
+    }
+}
 __device__ __forceinline__ void st_global_128(void *p, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
 {
     asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
@@ -290,7 +311,7 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
 #pragma unroll
                 for (int g = 0; g < 4; ++g) ents[g] = __shfl_sync(0xffffffffu, ent, g);
             }
-            if (MODE == FLEXIQ_OUT_REQUANT_I8 && p.tma_store) {
+            if ((MODE == FLEXIQ_OUT_REQUANT_I8 || MODE == kOutNextSlab) && p.tma_store) {
                 // Each warp stages 32 rows x 32 columns (1 KB, 32-byte swizzle: no bank conflicts) and one
                 // lane hands them to a tiled bulk store, which writes whole sectors asynchronously and
                 // drops the rows and columns that lie outside Y.
@@ -302,8 +323,16 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                     if (32 * h < cols && n < p.N && row0 < p.M) {   // warp-uniform
                         const bool both = 32 * h + 16 < cols && n + 16 < p.N;  // a 32-column box, else a 16-column one
                         uint32_t w[8];
-                        finish16<MODE>(r, x.fac + 32 * h, x.fac + 64 + 32 * h, w);
-                        if (both) finish16<MODE>(r + 16, x.fac + 32 * h + 16, x.fac + 64 + 32 * h + 16, w + 4);
+                        if (MODE == kOutNextSlab) {
+                            // the producer already emits the next layer's slab order: chunk c stays chunk c and
+                            // is lowered when it lies below the next layer's max_4bit_ch
+#pragma unroll
+                            for (int g = 0; g < 2; ++g)
+                                if (g == 0 || both) next_slab16(p, ents[2 * h + g], r + 16 * g, x.fac + 32 * h + 16 * g, x.fac + 64 + 32 * h + 16 * g, w + 4 * g);
+                        } else {
+                            finish16<FLEXIQ_OUT_REQUANT_I8>(r, x.fac + 32 * h, x.fac + 64 + 32 * h, w);
+                            if (both) finish16<FLEXIQ_OUT_REQUANT_I8>(r + 16, x.fac + 32 * h + 16, x.fac + 64 + 32 * h + 16, w + 4);
+                        }
                         if (lane == 0) ptx::bulk_wait_read_all();    // the previous store has read the buffer
                         __syncwarp();
                         if (both) {
@@ -338,25 +367,8 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
 #pragma unroll
                             for (int g = 0; g < 2; ++g) {
                                 if (g == 0 || second) {
-                                    const int e = ents[2 * h + g];
-                                    pos[g] = e & 0xffffff;
-                                    float lo = -128.f, hi = 127.f;
-                                    uint32_t mask = 0xffffffffu;
-                                    if (pos[g] * 16 < p.next_K_lo) {
-                                        const int sft = e >> 24;
-                                        hi = (float)(8 << sft) - 1.f;
-                                        lo = -(float)(8 << sft);
-                                        mask = ((0xffu << sft) & 0xffu) * 0x01010101u;
-                                    }
-                                    if (p.relu) lo = fmaxf(lo, 0.f);
-                                    // the pack saturates to [-128, 127] by itself: clamp only when the range is narrower (warp-uniform)
-                                    if (lo > -128.f || hi < 127.f)
-                                        finish16_next(r + 16 * g, x.fac + 32 * h + 16 * g, x.fac + 64 + 32 * h + 16 * g, lo, hi, mask, w + 4 * g);
-                                    else {
-                                        finish16<FLEXIQ_OUT_REQUANT_I8>(r + 16 * g, x.fac + 32 * h + 16 * g, x.fac + 64 + 32 * h + 16 * g, w + 4 * g);
-#pragma unroll
-                                        for (int q = 0; q < 4; ++q) w[4 * g + q] &= mask;
-                                    }
+                                    pos[g] = ents[2 * h + g] & 0xffffff;
+                                    next_slab16(p, ents[2 * h + g], r + 16 * g, x.fac + 32 * h + 16 * g, x.fac + 64 + 32 * h + 16 * g, w + 4 * g);
                                 }
                             }
                             uint8_t *srow = static_cast<uint8_t *>(p.Y) + row * p.N;
@@ -398,7 +410,7 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
         }
         if ((buf ^= 1) == 0) buf_phase ^= 1;
     }
-    if (MODE == FLEXIQ_OUT_REQUANT_I8 && p.tma_store && lane == 0) ptx::bulk_wait_all();  // the staged stores are performed
+    if ((MODE == FLEXIQ_OUT_REQUANT_I8 || MODE == kOutNextSlab) && p.tma_store && lane == 0) ptx::bulk_wait_all();  // the staged stores are performed
     if (quad == 2 && part == 0 && lane == 0) { PROF_STORE(8, prof_wait); PROF_STORE(9, clock64() - prof_start); PROF_STORE(10, prof_ld); PROF_STORE(11, prof_math); }
 }
 
@@ -1075,7 +1087,7 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     // activation maps (per call: they depend on the caller's buffers, M and the ratio);
     // an empty slab borrows the other one's map and is never addressed
     CUtensorMap a_lo, a_hi;
-    const bool staged = out_mode == FLEXIQ_OUT_REQUANT_I8 && !direct_stores_only();
+    const bool staged = (out_mode == FLEXIQ_OUT_REQUANT_I8 || (next && out_order == FLEXIQ_ORDER_NEXT_SLAB)) && !direct_stores_only();
     const void *slab = packed_path ? static_cast<const void *>(X8) : static_cast<const void *>(X4);
     Layer::CallMaps &cm = L->call_maps;
     const bool cached = !packed && cm.slab == slab && cm.M == M && cm.Nb == Nb && cm.H == H && cm.W == W && cm.bk == p.BK &&
