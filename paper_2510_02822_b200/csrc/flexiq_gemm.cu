@@ -253,7 +253,10 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
     constexpr bool kScaled = MODE != FLEXIQ_OUT_ACC_I32;
     constexpr int kElem = (MODE == FLEXIQ_OUT_REQUANT_I8 || MODE == kOutNextSlab) ? 1 : 4;  // output bytes per element
     const int BN = p.BN;
-    const int cols = BN >> 2;                    // 16, 32, 48 or 64 columns for this warp
+    // Columns per warp and pass: 64 (tiles of 192 or 256 columns) or 32 (128 or 64), so that every staged
+    // box is 32 columns = whole sectors; with 192 or 64 columns the last column slot of a lane quadrant has no
+    // columns and its warp only keeps step with the accumulator barriers.
+    const int cols = BN >= 192 ? 64 : 32;
     const bool y32 = (reinterpret_cast<uintptr_t>(p.Y) & 31) == 0;
     const bool wide = y32 && (p.N & 31) == 0;    // int8 rows are 32-byte aligned: 256-bit stores
     // lane l keeps factors 4l..4l+3 of the table alpha[64] | beta[64]
@@ -272,6 +275,21 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
         for (int pass = 0; pass < passes; ++pass) {
             const int col0 = (part * passes + pass) * cols;  // first tile column of this warp in this pass
             const int nw = tw.n_blk * BN + col0;             // ... as an output channel
+            if (col0 >= BN) {
+                // no columns for this warp in this pass: only keep step with the accumulator barriers
+                if (!waited) {
+                    if (!__all_sync(0xffffffffu, wait_bounded(&x.tmem_full[buf], buf_phase, x.abort_flag, 4))) return;
+                    waited = true;
+                }
+                if (pass + 1 == passes) {
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (CG == 2) ptx::mbar_arrive_cluster_relaxed(ptx::mapa(ptx::smem_u32(&x.tmem_empty[buf]), 0));
+                        else ptx::mbar_arrive_relaxed(&x.tmem_empty[buf]);
+                    }
+                }
+                continue;
+            }
             float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
             if (kScaled && nw + 4 * (lane & 15) < p.N) f = __ldg(reinterpret_cast<const float4 *>(fsrc + nw));
             int ent = 0;                                     // fused boundary: lane g fetches chunk g's slab entry
@@ -287,8 +305,8 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
             const uint32_t taddr = x.tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)buf * x.buf_stride + (uint32_t)col0;
             PROF_T0(te0);
             uint32_t ra[32], rb[32];
-            if (cols >= 32) ptx::tmem_ld_32x32(taddr, ra); else ptx::tmem_ld_32x16(taddr, ra);
-            if (cols == 64) ptx::tmem_ld_32x32(taddr + 32, rb); else if (cols == 48) ptx::tmem_ld_32x16(taddr + 32, rb);
+            ptx::tmem_ld_32x32(taddr, ra);
+            if (cols == 64) ptx::tmem_ld_32x32(taddr + 32, rb);
             if (kScaled) {
                 __syncwarp();                                      // the previous reads of the table are done
                 reinterpret_cast<float4 *>(x.fac)[lane] = f;
@@ -321,7 +339,7 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                     const uint32_t *r = h == 0 ? ra : rb;
                     const int n = nw + 32 * h;
                     if (32 * h < cols && n < p.N && row0 < p.M) {   // warp-uniform
-                        const bool both = 32 * h + 16 < cols && n + 16 < p.N;  // a 32-column box, else a 16-column one
+                        const bool both = n + 16 < p.N;  // a 32-column box, else (last 16 channels of N) a 16-column one
                         uint32_t w[8];
                         if (MODE == kOutNextSlab) {
                             // the producer already emits the next layer's slab order: chunk c stays chunk c and
@@ -359,7 +377,7 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                     const uint32_t *r = h == 0 ? ra : rb;
                     const int n = nw + 32 * h;
                     if (32 * h < cols && n < p.N) {
-                        const bool second = 32 * h + 16 < cols && n + 16 < p.N;  // columns 16..31 of this half are live
+                        const bool second = n + 16 < p.N;  // columns 16..31 of this half are live
                         if (MODE == kOutNextSlab) {
                             // each 16-channel chunk goes to its place in the next layer's slab row
                             uint32_t w[8];
