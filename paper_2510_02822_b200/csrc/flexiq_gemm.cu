@@ -899,11 +899,14 @@ __global__ void scale_vectors_kernel(int N, float x_scale, float y_scale, int re
 // ------------------------------------------------------------------------------------
 // host side
 
-// Tile shape, from a cost model with constants measured on B200 (cycles per 128-byte K block):
-// the MMA takes 2*BN cycles, the TMA fill of the operands about (128 + BN/cg) * 128 / 97, and no
-// K block goes faster than about 420 cycles of issue overhead; the epilogue of a tile takes about
-// 2400 + 8 * BN cycles and, being overlapped, only costs when it exceeds the mainloop (ties go to the
-// configuration listed first).  cost = waves * tile time.
+// Tile shape, from a cost model in SM cycles whose constants were fitted to measured times of every
+// tile shape on twenty layer shapes (ViT-B, DeiT-S at batch 1 and 8, ResNet-50 convolutions):
+//   per K block  max(MMA 2*BN cycles per 128 bytes of K;  TMA fill of (128 + BN/cg) rows at 90 bytes per
+//                cycle, 70 when (almost) every SM is loading, and at least 3.5 cycles per 64-byte row;
+//                a floor of 350 cycles, 500 with every SM busy)
+//   per tile     the K blocks + 800 cycles; its epilogue (800 + 4*BN cycles) overlaps the next tile
+//   in all       waves * tile + one epilogue that nothing overlaps + 1600 cycles for a CTA pair
+//                (cluster launch and barriers), which pays off once the machine is full.
 struct TileChoice { int cg, bn; };
 static TileChoice g_forced_tile{0, 0};  // test hook: 0 = choose automatically
 static bool direct_stores_only()
@@ -914,26 +917,31 @@ static bool direct_stores_only()
     return false;
 #endif
 }
-static TileChoice choose_tile(long long M, int N, int k_blocks, int sms)
+static TileChoice choose_tile(long long M, int N, int k_blocks, int bk, int sms)
 {
     const int bns[4] = {256, 192, 128, 64};
     TileChoice best{1, 256};
     double best_cost = 1e300;
-    for (int cg = 2; cg >= 1; --cg)  // pairs first: they halve the B traffic per SM
+    for (int cg = 2; cg >= 1; --cg)  // ties go to pairs: they halve the B traffic per SM
         for (int i = 0; i < 4; ++i) {
             const int bn = bns[i];
             if (cg == 2 && bn < 128) continue;
             const long long m_tiles = (M + (long long)BM * cg - 1) / ((long long)BM * cg);
             const long long n_tiles = (N + bn - 1) / bn;
             const long long slots = sms / cg;
-            const long long waves = (m_tiles * n_tiles + slots - 1) / slots;
-            double per_kb = 2.0 * bn;
-            const double tma = (128.0 + (double)bn / cg) * 128.0 / 97.0;
-            if (tma > per_kb) per_kb = tma;
-            if (per_kb < 420.0) per_kb = 420.0;
+            const long long tiles = m_tiles * n_tiles;
+            const long long waves = (tiles + slots - 1) / slots;
+            const bool busy = (tiles < slots ? tiles : slots) * cg >= 140;
+            const double rows = 128.0 + (double)bn / cg;
+            const double mma = 2.0 * bn * bk / 128.0;
+            double tma = rows * bk / (busy ? 70.0 : 90.0);
+            if (bk == 64 && tma < rows * 3.5) tma = rows * 3.5;
+            const double floor_kb = (busy ? 500.0 : 350.0) * (bk == 128 ? 1.0 : 0.6);
+            double per_kb = mma > tma ? mma : tma;
+            if (per_kb < floor_kb) per_kb = floor_kb;
             const double mainloop = k_blocks * per_kb + 800.0;
-            const double epi = 2400.0 + 8.0 * bn;
-            const double cost = (double)waves * (mainloop > epi ? mainloop : epi);
+            const double epi = 800.0 + 4.0 * bn;
+            const double cost = (double)waves * (mainloop > epi ? mainloop : epi) + epi + (cg == 2 ? 1600.0 : 0.0);
             if (cost < best_cost - 1e-9) { best_cost = cost; best = TileChoice{cg, bn}; }
         }
     return best;
@@ -1054,7 +1062,7 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     p.out_mode = out_mode; p.Y = Y;
     if (next) { p.next_ent = out_order == FLEXIQ_ORDER_NEXT_SLAB ? next->chunk_ent_slab : next->chunk_ent; p.next_K_lo = next->K_lo; p.relu = relu != 0; }
     p.alpha = L->alpha; p.beta = L->beta;
-    TileChoice tc = g_forced_tile.cg ? g_forced_tile : choose_tile(M, L->N, p.T * (p.nb_lo + p.nb_hi), sms);
+    TileChoice tc = g_forced_tile.cg ? g_forced_tile : choose_tile(M, L->N, p.T * (p.nb_lo + p.nb_hi), p.BK, sms);
     if (packed && tc.cg == 2) {  // the packed path runs single CTAs: re-choose among those
         tc.cg = 1;
         if (!g_forced_tile.cg) {
