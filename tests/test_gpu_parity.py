@@ -312,3 +312,65 @@ def test_extreme_accumulators(dev, K):
     case.X = (sgn * 200.0 * case.x_scale).astype(np.float32)  # quantizes to -128 / 127
     case.y_scale = float(np.float32(K * 128.0))
     _run_linear(case, dev, [0.0, 0.5, 1.0])
+
+
+# ---------------------------------------------------------------- streams and graphs
+def test_cuda_graph_replay_matches_oracle(dev):
+    """Prologue + GEMM captured in a CUDA graph (nothing allocates, the launches carry their
+    programmatic-dependency attributes) and replayed on new input values."""
+    case = inputs.ranged_linear("g", 300, 384, 272, 16, seed=21, group_structured=True)
+    perm, sxg, sxs, sw = helpers.prepare_linear(case)
+    L = _layer(case, dev, perm, sxg)
+    L.set_lowbit_ratio(0.5)
+    nl = oracle.n_low(0.5, case.K // case.G)
+    X = torch.from_numpy(case.X).to(dev)
+    x4, x8 = L.alloc_slabs(case.M)
+    Y = torch.empty((case.M, case.N), dtype=torch.int8, device=dev)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        fx.flexiq_quantize_lower(L.h, X, fx.DTYPE_F32, case.M, case.x_scale, 0, x4, x8)   # warm-up outside the capture
+        fx.flexiq_mixed_gemm(L.h, x4, x8, None, case.M, case.x_scale, case.y_scale, fx.OUT_REQUANT_I8, Y)
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            fx.flexiq_quantize_lower(L.h, X, fx.DTYPE_F32, case.M, case.x_scale, 0, x4, x8)
+            fx.flexiq_mixed_gemm(L.h, x4, x8, None, case.M, case.x_scale, case.y_scale, fx.OUT_REQUANT_I8, Y)
+    torch.cuda.synchronize()
+    for rep in range(2):
+        Xn = case.X * np.float32(1.0 - 0.37 * rep)
+        X.copy_(torch.from_numpy(Xn))
+        Y.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        q = oracle.quantize(Xn, case.x_scale)
+        acc = oracle.mixed_gemm_acc(q, case.Wq, case.G, perm, sxs, sw, nl)
+        assert np.array_equal(Y.cpu().numpy(), oracle.epilogue_i8(acc, case.x_scale, case.w_scale, case.bias, case.y_scale))
+    fx.flexiq_check_status()
+    L.close()
+
+
+def test_two_layers_on_two_streams(dev):
+    """Independent layer handles may run on different streams at the same time."""
+    cases = [inputs.ranged_linear("a", 700, 256, 320, 16, seed=31), inputs.ranged_linear("b", 500, 512, 144, 32, seed=32)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    prepared, outs = [], []
+    for c in cases:
+        perm, sxg, sxs, sw = helpers.prepare_linear(c)
+        L = _layer(c, dev, perm, sxg)
+        L.set_lowbit_ratio(0.5)
+        prepared.append((L, perm, sxs, sw, torch.from_numpy(c.X).to(dev)))
+    torch.cuda.synchronize()
+    for rep in range(5):
+        for (L, perm, sxs, sw, X), c, st in zip(prepared, cases, streams):
+            with torch.cuda.stream(st):
+                x4, x8, _ = L.quantize_lower(X, c.x_scale)
+                Y = L.mixed_gemm(x4, x8, c.M, c.x_scale, c.y_scale, fx.OUT_ACC_I32)
+                if rep == 4:
+                    outs.append(Y)
+    torch.cuda.synchronize()
+    for (L, perm, sxs, sw, X), c, Y in zip(prepared, cases, outs):
+        q = oracle.quantize(c.X, c.x_scale)
+        assert np.array_equal(Y.cpu().numpy(), oracle.mixed_gemm_acc(q, c.Wq, c.G, perm, sxs, sw, oracle.n_low(0.5, c.K // c.G)))
+        L.close()
+    fx.flexiq_check_status()
