@@ -5,10 +5,13 @@
 // Design for sm_100a.  The 4-bit values, shifted back to their extraction positions, are
 // 8-bit integers (|x4 << sx| <= 128), so low and high channel groups feed ONE chain of
 // tcgen05.mma.kind::i8 instructions accumulating in TMEM: no per-group round trip through
-// registers for the shift.  A persistent, warp-specialised CTA per SM:
-//   warp 0      TMA producer (tiled loads for linear layers, im2col loads for convs)
-//   warp 1      TMEM allocation + single-thread MMA issue
-//   warps 2..9  epilogue: tcgen05.ld, scale / bias / round / clip, staged coalesced stores
+// registers for the shift.  A persistent, warp-specialised CTA per SM, or a CTA pair (cluster of two,
+// cta_group::2) per 256-row tile:
+//   warp 0       TMA producer (tiled loads for linear layers, im2col loads for convs)
+//   warp 1       TMEM allocation + MMA issue (one elected lane)
+//   warps 2..17  epilogue, four per TMEM lane quadrant: tcgen05.ld, scale / bias / round / clip, int8
+//                tiles staged in shared memory and written by tiled bulk stores (fp32 / int32: direct
+//                256-bit stores); on the packed path eight of them widen 4-bit tiles instead
 // Two TMEM accumulators let the epilogue of tile i overlap the mainloop of tile i+1.
 // Every wait is bounded; an expired wait raises the status word and the CTA drains.
 #include "flexiq_internal.h"
