@@ -225,6 +225,13 @@ int flexiq_mixed_conv_to_slab(flexiq_layer_t layer, const uint8_t *X4_dev, const
  *   activation channels using sampled calibration data", Sec. 4.2).  accumulate != 0 merges into
  *   the ranges already in lo_dev / hi_dev (several calibration batches); 0 starts from [0, 0].
  *   lo_dev, hi_dev: [K] int32.  K % 16 == 0.
+ * flexiq_calib_channel_histogram / flexiq_calib_ranges_from_histogram: ranges that cover a given
+ *   share of each channel's values instead of all of them (Sec. 8.4 presumes ranges "to cover 99 %
+ *   of neuron values for each channel").  The first counts the Eq. 1-quantized values per channel,
+ *   hist_dev [K][256] uint32 with bin q + 128 (accumulate as above); the second drops at most `tail`
+ *   samples from each end of every channel's histogram -- the caller passes
+ *   tail = floor(n * (1 - coverage) / 2) for n samples per channel -- and widens the result to
+ *   contain zero.  tail = 0 gives the exact ranges of flexiq_calib_channel_ranges.
  * flexiq_calib_weight_absmax: wmax_dev[k] = max |w| over the output channels (and taps) of input
  *   channel k ("the corresponding weight parameters' channels across the output channel dimension
  *   to determine the maximum value range", Sec. 4.2).  Linear: Wq_dev [K][N], taps ignored;
@@ -247,6 +254,10 @@ int flexiq_mixed_conv_to_slab(flexiq_layer_t layer, const uint8_t *X4_dev, const
  * All enqueue on `stream`, allocate nothing and return the usual codes. */
 int flexiq_calib_channel_ranges(const void *X_dev, int x_dtype, int64_t M, int K, float x_scale,
                                 int accumulate, int32_t *lo_dev, int32_t *hi_dev, void *stream);
+int flexiq_calib_channel_histogram(const void *X_dev, int x_dtype, int64_t M, int K, float x_scale,
+                                   int accumulate, uint32_t *hist_dev, void *stream);
+int flexiq_calib_ranges_from_histogram(const uint32_t *hist_dev, int K, int64_t tail, int32_t *lo_dev,
+                                       int32_t *hi_dev, void *stream);
 int flexiq_calib_weight_absmax(const int8_t *Wq_dev, int is_conv, int K, int N, int taps,
                                int32_t *wmax_dev, void *stream);
 int flexiq_calib_prepare(const int32_t *lo_dev, const int32_t *hi_dev, const int32_t *wmax_dev, int K,

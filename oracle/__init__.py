@@ -260,3 +260,20 @@ def absmax_ema(x_batches, momentum: float) -> float:
     f = lib().fqo_absmax_ema
     f.restype = C.c_float
     return float(f(_p(x), C.c_int64(b), C.c_int64(x.size // b), C.c_float(momentum)))
+
+
+def channel_histogram(q) -> np.ndarray:
+    q = _c(q, np.int8)
+    M, K = q.shape
+    hist = np.empty((K, 256), np.uint32)
+    lib().fqo_channel_histogram(_p(q), C.c_int64(M), K, _p(hist))
+    return hist
+
+
+def ranges_from_histogram(hist, tail: int):
+    hist = _c(hist, np.uint32)
+    K = hist.shape[0]
+    lo = np.empty(K, np.int32)
+    hi = np.empty(K, np.int32)
+    lib().fqo_ranges_from_histogram(_p(hist), K, C.c_int64(tail), _p(lo), _p(hi))
+    return lo, hi

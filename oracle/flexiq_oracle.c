@@ -449,6 +449,30 @@ void fqo_reorder_channels(const uint8_t *x, int64_t M, int K, int G, int elem_by
             }
 }
 
+/* Coverage-based channel ranges (Sec. 8.4: ranges presumed "to cover 99 % of neuron values for each
+ * channel"): hist[c][q + 128] counts the quantized values of channel c; the range drops at most `tail`
+ * samples from each end (tail = floor(n * (1 - coverage) / 2) for n samples) and is widened to contain
+ * zero.  tail = 0 is the exact min / max of fqo_channel_ranges. */
+void fqo_channel_histogram(const int8_t *q, int64_t M, int K, uint32_t *hist /*[K][256]*/)
+{
+    for (int64_t i = 0; i < (int64_t)K * 256; ++i) hist[i] = 0;
+    for (int64_t m = 0; m < M; ++m)
+        for (int c = 0; c < K; ++c) hist[(int64_t)c * 256 + q[m * K + c] + 128] += 1;
+}
+void fqo_ranges_from_histogram(const uint32_t *hist, int K, int64_t tail, int32_t *lo, int32_t *hi)
+{
+    for (int c = 0; c < K; ++c) {
+        const uint32_t *h = hist + (int64_t)c * 256;
+        int64_t dropped = 0;
+        int l = -128, u = 127;
+        while (l < 0 && dropped + h[l + 128] <= tail) { dropped += h[l + 128]; ++l; }
+        dropped = 0;
+        while (u > 0 && dropped + h[u + 128] <= tail) { dropped += h[u + 128]; --u; }
+        lo[c] = l;
+        hi[c] = u;
+    }
+}
+
 /* Unused-bit statistics (Sec. 8.4): an int8 value has 7 magnitude bits; a channel whose range needs
  * L of them leaves 7 - L unused ("maximum is less than 32 => the highest two bits are not used",
  * Sec. 4.1).  hist[u] counts the channels with u unused bits, u = 4 standing for four or more. */

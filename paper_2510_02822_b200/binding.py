@@ -25,7 +25,8 @@ EXPORTS = [
     "flexiq_layer_set_lowbit_path", "flexiq_set_lowbit_ratio", "flexiq_get_max_4bit_ch",
     "flexiq_x4_pitch", "flexiq_quantize_lower", "flexiq_quantize_lower_dynamic_noalloc", "flexiq_mixed_gemm", "flexiq_mixed_conv",
     "flexiq_mixed_gemm_to_slab", "flexiq_mixed_conv_to_slab", "flexiq_reorder_channels",
-    "flexiq_calib_channel_ranges", "flexiq_calib_weight_absmax", "flexiq_calib_prepare", "flexiq_calib_absmax_ema",
+    "flexiq_calib_channel_ranges", "flexiq_calib_channel_histogram", "flexiq_calib_ranges_from_histogram",
+    "flexiq_calib_weight_absmax", "flexiq_calib_prepare", "flexiq_calib_absmax_ema",
     "flexiq_layer_export", "flexiq_force_tile", "flexiq_check_status", "flexiq_last_error",
 ]
 
@@ -64,6 +65,8 @@ def lib():
         L.flexiq_mixed_conv_to_slab.argtypes = [vp, vp, vp, vp, i32, i32, i32, f32, vp, f32, i32, i32, vp, vp]
         L.flexiq_reorder_channels.argtypes = [vp, vp, i32, i64, i32, vp, vp]
         L.flexiq_calib_channel_ranges.argtypes = [vp, i32, i64, i32, f32, i32, vp, vp, vp]
+        L.flexiq_calib_channel_histogram.argtypes = [vp, i32, i64, i32, f32, i32, vp, vp]
+        L.flexiq_calib_ranges_from_histogram.argtypes = [vp, i32, i64, vp, vp, vp]
         L.flexiq_calib_weight_absmax.argtypes = [vp, i32, i32, i32, i32, vp, vp]
         L.flexiq_calib_prepare.argtypes = [vp, vp, vp, i32, i32, vp, vp, vp, vp, vp]
         L.flexiq_calib_absmax_ema.argtypes = [vp, i32, i64, f32, vp, vp]
@@ -183,6 +186,14 @@ def flexiq_reorder_channels(h, X_dev, elem_bytes, M, direction, Y_dev):
 
 def flexiq_calib_channel_ranges(X_dev, x_dtype, M, K, x_scale, accumulate, lo_dev, hi_dev):
     _check(lib().flexiq_calib_channel_ranges(_ptr(X_dev), x_dtype, M, K, x_scale, int(accumulate), _ptr(lo_dev), _ptr(hi_dev), _stream()))
+
+
+def flexiq_calib_channel_histogram(X_dev, x_dtype, M, K, x_scale, accumulate, hist_dev):
+    _check(lib().flexiq_calib_channel_histogram(_ptr(X_dev), x_dtype, M, K, x_scale, int(accumulate), _ptr(hist_dev), _stream()))
+
+
+def flexiq_calib_ranges_from_histogram(hist_dev, K, tail, lo_dev, hi_dev):
+    _check(lib().flexiq_calib_ranges_from_histogram(_ptr(hist_dev), K, int(tail), _ptr(lo_dev), _ptr(hi_dev), _stream()))
 
 
 def flexiq_calib_weight_absmax(Wq_dev, is_conv, K, N, taps, wmax_dev):

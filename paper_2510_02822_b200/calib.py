@@ -56,11 +56,14 @@ def permute_outputs_for_next(Wq: torch.Tensor, w_scale: torch.Tensor, bias, next
     return Wp, w_scale.index_select(0, cols).contiguous(), None if bias is None else bias.index_select(0, cols).contiguous()
 
 
-def static_preparation_device(Xcal: torch.Tensor, x_scale: float, Wq: torch.Tensor, G: int, conv: bool = False, batches: int = 1):
+def static_preparation_device(Xcal: torch.Tensor, x_scale: float, Wq: torch.Tensor, G: int, conv: bool = False, batches: int = 1,
+                              coverage: float | None = None):
     """The same preparation with the library's calibration kernels, on device tensors.
 
     Xcal: calibration activations [..., C] (fp32 / fp16 / bf16 / int8) on the GPU; Wq as in
     static_preparation, on the GPU.  The rows are fed in `batches` accumulating calls.
+    coverage (e.g. 0.99): channel ranges that cover that share of each channel's calibration values
+    (per-channel histograms, equal tails dropped) instead of the exact min / max.
     Returns (group_perm, x_shift, info) with info = {lo, hi, wmax, score, unused_hist} (torch tensors)."""
     from . import binding as fx
     dev = Xcal.device
@@ -70,9 +73,15 @@ def static_preparation_device(Xcal: torch.Tensor, x_scale: float, Wq: torch.Tens
     hi = torch.empty(C, dtype=torch.int32, device=dev)
     rows = X2.shape[0]
     step = (rows + batches - 1) // batches
+    hist = torch.empty((C, 256), dtype=torch.int32, device=dev) if coverage is not None else None
     for b in range(batches):
         part = X2[b * step:(b + 1) * step]
-        fx.flexiq_calib_channel_ranges(part, fx._dtype_code(part), part.shape[0], C, x_scale, b > 0, lo, hi)
+        if coverage is None:
+            fx.flexiq_calib_channel_ranges(part, fx._dtype_code(part), part.shape[0], C, x_scale, b > 0, lo, hi)
+        else:
+            fx.flexiq_calib_channel_histogram(part, fx._dtype_code(part), part.shape[0], C, x_scale, b > 0, hist)
+    if coverage is not None:
+        fx.flexiq_calib_ranges_from_histogram(hist, C, int(rows * (1.0 - coverage) / 2.0), lo, hi)
     wmax = torch.empty(C, dtype=torch.int32, device=dev)
     if conv:
         fx.flexiq_calib_weight_absmax(Wq, True, C, Wq.shape[0], Wq.shape[1] * Wq.shape[2], wmax)

@@ -76,6 +76,57 @@ __global__ void calib_ranges_kernel(const void *__restrict__ X, long long M, int
     }
 }
 
+// Per-channel histogram of the Eq. 1-quantized activations (256 bins, bin = q + 128), the input of
+// coverage-based ranges (Sec. 8.4: ranges that cover 99 % of a channel's values).  A block owns 32
+// channels and a slice of the rows and counts in shared memory; one global atomic per non-empty bin.
+constexpr int kHistWindow = 32;
+template <int DTYPE>
+__global__ void calib_hist_kernel(const void *__restrict__ X, long long M, int K, float S, int slices, unsigned *__restrict__ hist)
+{
+    __shared__ unsigned h[kHistWindow * 256];
+    for (int i = threadIdx.x; i < kHistWindow * 256; i += blockDim.x) h[i] = 0;
+    __syncthreads();
+    const int win = blockIdx.x / slices, slice = blockIdx.x - win * slices;
+    const int chunk = threadIdx.x & 1, rlane = threadIdx.x >> 1;
+    const int rows_per_pass = blockDim.x >> 1;
+    const int c0 = win * kHistWindow + 16 * chunk;
+    const Divider div = make_divider(S);
+    if (c0 < K) {
+        for (long long m = (long long)slice * rows_per_pass + rlane; m < M; m += (long long)slices * rows_per_pass) {
+            unsigned w[4];
+            quantize16<DTYPE>(reinterpret_cast<const char *>(X) + ((size_t)m * K + c0) * elem_bytes<DTYPE>(), div, -128.f, 127.f, w);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    const int q = (int)(signed char)((w[k] >> (8 * b)) & 0xff);
+                    atomicAdd(&h[(16 * chunk + 4 * k + b) * 256 + q + 128], 1u);
+                }
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < kHistWindow * 256; i += blockDim.x) {
+        const int c = win * kHistWindow + (i >> 8);
+        if (h[i] && c < K) atomicAdd(&hist[(size_t)c * 256 + (i & 255)], h[i]);
+    }
+}
+
+// Range of a channel after dropping at most `tail` samples from each end of its histogram, widened to
+// contain zero (lo <= 0 <= hi).  tail = 0 gives the exact min / max.
+__global__ void ranges_from_hist_kernel(const unsigned *__restrict__ hist, int K, long long tail, int32_t *__restrict__ lo,
+                                        int32_t *__restrict__ hi)
+{
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= K) return;
+    const unsigned *h = hist + (size_t)c * 256;
+    long long below = 0, above = 0;
+    int l = -128, u = 127;
+    while (l < 0 && below + h[l + 128] <= tail) { below += h[l + 128]; ++l; }
+    while (u > 0 && above + h[u + 128] <= tail) { above += h[u + 128]; --u; }
+    lo[c] = l;
+    hi[c] = u;
+}
+
 // Largest |w| over the output channels (and taps) of every input channel.
 // Linear weights [K][N]: one warp per input channel (row).
 __global__ void weight_absmax_rows_kernel(const int8_t *__restrict__ W, int K, int N, int32_t *__restrict__ wmax)
@@ -212,6 +263,49 @@ extern "C" int flexiq_calib_channel_ranges(const void *X_dev, int x_dtype, int64
         case FLEXIQ_DTYPE_BF16: return launch_ranges<FLEXIQ_DTYPE_BF16>(X_dev, M, K, x_scale, lo_dev, hi_dev, sms, st);
         default: return launch_ranges<FLEXIQ_DTYPE_I8>(X_dev, M, K, x_scale, lo_dev, hi_dev, sms, st);
     }
+}
+
+extern "C" int flexiq_calib_channel_histogram(const void *X_dev, int x_dtype, int64_t M, int K, float x_scale, int accumulate,
+                                              uint32_t *hist_dev, void *stream)
+{
+    if (M < 0 || K <= 0 || K % 16 != 0) return set_error(FLEXIQ_ERR_INVALID_ARG, "bad shape M=%lld K=%d (K must be a positive multiple of 16)", (long long)M, K);
+    if (x_dtype < FLEXIQ_DTYPE_F32 || x_dtype > FLEXIQ_DTYPE_I8) return set_error(FLEXIQ_ERR_INVALID_ARG, "unknown x_dtype %d", x_dtype);
+    if (x_dtype != FLEXIQ_DTYPE_I8 && !(x_scale > 0.0f)) return set_error(FLEXIQ_ERR_INVALID_ARG, "x_scale %g must be positive", (double)x_scale);
+    if (!hist_dev) return set_error(FLEXIQ_ERR_INVALID_ARG, "hist_dev is NULL");
+    int rc = check_device_sm100();
+    if (rc) return rc;
+    cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+    if (!accumulate) FLEXIQ_CUDA_TRY(cudaMemsetAsync(hist_dev, 0, sizeof(uint32_t) * 256 * (size_t)K, st));
+    if (M == 0) return FLEXIQ_OK;
+    if (!X_dev || (reinterpret_cast<uintptr_t>(X_dev) & 15)) return set_error(FLEXIQ_ERR_INVALID_ARG, "X_dev is NULL or not 16-byte aligned");
+    int dev = 0;
+    cudaGetDevice(&dev);
+    const int sms = device_sm_count(dev);
+    const int windows = (K + kHistWindow - 1) / kHistWindow;
+    long long slices = ((long long)sms * 4 + windows - 1) / windows;
+    const long long max_slices = (M + 127) / 128;
+    if (slices > max_slices) slices = max_slices;
+    const unsigned grid = (unsigned)(windows * slices);
+    switch (x_dtype) {
+        case FLEXIQ_DTYPE_F32: calib_hist_kernel<FLEXIQ_DTYPE_F32><<<grid, 256, 0, st>>>(X_dev, M, K, x_scale, (int)slices, hist_dev); break;
+        case FLEXIQ_DTYPE_F16: calib_hist_kernel<FLEXIQ_DTYPE_F16><<<grid, 256, 0, st>>>(X_dev, M, K, x_scale, (int)slices, hist_dev); break;
+        case FLEXIQ_DTYPE_BF16: calib_hist_kernel<FLEXIQ_DTYPE_BF16><<<grid, 256, 0, st>>>(X_dev, M, K, x_scale, (int)slices, hist_dev); break;
+        default: calib_hist_kernel<FLEXIQ_DTYPE_I8><<<grid, 256, 0, st>>>(X_dev, M, K, x_scale, (int)slices, hist_dev); break;
+    }
+    FLEXIQ_CUDA_TRY(cudaGetLastError());
+    return FLEXIQ_OK;
+}
+
+extern "C" int flexiq_calib_ranges_from_histogram(const uint32_t *hist_dev, int K, int64_t tail, int32_t *lo_dev, int32_t *hi_dev,
+                                                  void *stream)
+{
+    if (K <= 0 || tail < 0) return set_error(FLEXIQ_ERR_INVALID_ARG, "bad K = %d or tail = %lld", K, (long long)tail);
+    if (!hist_dev || !lo_dev || !hi_dev) return set_error(FLEXIQ_ERR_INVALID_ARG, "a device pointer is NULL");
+    int rc = check_device_sm100();
+    if (rc) return rc;
+    ranges_from_hist_kernel<<<(K + 127) / 128, 128, 0, reinterpret_cast<cudaStream_t>(stream)>>>(hist_dev, K, (long long)tail, lo_dev, hi_dev);
+    FLEXIQ_CUDA_TRY(cudaGetLastError());
+    return FLEXIQ_OK;
 }
 
 extern "C" int flexiq_calib_weight_absmax(const int8_t *Wq_dev, int is_conv, int K, int N, int taps, int32_t *wmax_dev, void *stream)

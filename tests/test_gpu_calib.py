@@ -63,6 +63,31 @@ def test_wide_layer_and_ragged_window(dev):
     assert np.array_equal(lo.cpu().numpy(), elo) and np.array_equal(hi.cpu().numpy(), ehi)
 
 
+@pytest.mark.parametrize("M,K,dt", [(700, 96, torch.float32), (3000, 768, torch.float16), (129, 1040, torch.int8)])
+def test_histogram_and_coverage_ranges(dev, M, K, dt):
+    rng = np.random.default_rng(M + K)
+    xs = 0.05
+    x = (rng.normal(0, 1, (M, K)) * rng.uniform(0.2, 6, (1, K))).astype(np.float32)
+    if dt == torch.int8:
+        X = torch.from_numpy(oracle.quantize(x, xs)).to(dev)
+        q = X.cpu().numpy()
+    else:
+        X = torch.from_numpy(x).to(dt).to(dev)
+        q = oracle.quantize(X.float().cpu().numpy(), xs)
+    hist = torch.empty((K, 256), dtype=torch.int32, device=dev)
+    half = M // 2
+    fx.flexiq_calib_channel_histogram(X[:half], fx._dtype_code(X), half, K, xs, False, hist)
+    fx.flexiq_calib_channel_histogram(X[half:], fx._dtype_code(X), M - half, K, xs, True, hist)
+    eh = oracle.channel_histogram(q)
+    assert np.array_equal(hist.cpu().numpy().view(np.uint32), eh)
+    lo = torch.empty(K, dtype=torch.int32, device=dev)
+    hi = torch.empty(K, dtype=torch.int32, device=dev)
+    for tail in (0, int(M * 0.01 / 2), M):
+        fx.flexiq_calib_ranges_from_histogram(hist, K, tail, lo, hi)
+        elo, ehi = oracle.ranges_from_histogram(eh, tail)
+        assert np.array_equal(lo.cpu().numpy(), elo) and np.array_equal(hi.cpu().numpy(), ehi)
+
+
 def test_absmax_ema(dev):
     rng = np.random.default_rng(5)
     x = (rng.normal(0, 1, (7, 4096)) * rng.uniform(0.5, 4, (7, 1))).astype(np.float32)
@@ -87,3 +112,15 @@ def test_argument_errors(dev):
         fx.flexiq_calib_prepare(z, z, z, 64, 24, z, z, z, z)                           # group size
     with pytest.raises(fx.FlexiqError):
         fx.flexiq_calib_absmax_ema(x, fx.DTYPE_I8, 256, 0.99, x)                       # integer input has no range to track
+
+
+def test_front_end_with_coverage(dev):
+    case = inputs.vit_linear("v", 64, 768, 768, 16, seed=17)
+    Xc = torch.from_numpy(case.Xcal).to(dev)
+    perm, xs, info = calib.static_preparation_device(Xc, case.x_scale, torch.from_numpy(case.Wq).to(dev), case.G, batches=3, coverage=0.99)
+    q = oracle.quantize(case.Xcal, case.x_scale)
+    lo, hi = oracle.ranges_from_histogram(oracle.channel_histogram(q), int(q.shape[0] * (1.0 - 0.99) / 2.0))
+    assert np.array_equal(info["lo"].cpu().numpy(), lo) and np.array_equal(info["hi"].cpu().numpy(), hi)
+    assert np.array_equal(xs, oracle.static_positions(lo, hi, case.G))
+    perm_e, _ = oracle.greedy_order(lo, hi, oracle.weight_absmax_linear(case.Wq), case.G)
+    assert np.array_equal(perm, perm_e)

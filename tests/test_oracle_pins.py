@@ -306,6 +306,33 @@ def test_unused_bit_histogram_and_ema():
     assert oracle.absmax_ema(x[:1], 0.99) == 3.0
 
 
+def test_coverage_ranges_from_histogram():
+    rng = np.random.default_rng(11)
+    q = np.clip(np.rint(rng.normal(0, 20, (1000, 8)) * np.array([0.1, 0.5, 1, 2, 4, 0.2, 1, 3])), -128, 127).astype(np.int8)
+    q[:, 5] = np.abs(q[:, 5])          # a one-sided channel: its lower end stays at zero
+    hist = oracle.channel_histogram(q)
+    assert hist.sum(1).tolist() == [1000] * 8
+    assert np.array_equal(hist[2], np.bincount(q[:, 2].astype(np.int64) + 128, minlength=256))
+    # no tail dropped: the exact ranges
+    lo0, hi0 = oracle.ranges_from_histogram(hist, 0)
+    elo, ehi = oracle.channel_ranges(q)
+    assert np.array_equal(lo0, elo) and np.array_equal(hi0, ehi)
+    # 99 % coverage = 5 samples per tail: the 6th smallest / largest value (order statistics), never past zero
+    lo, hi = oracle.ranges_from_histogram(hist, 5)
+    for c in range(8):
+        srt = np.sort(q[:, c].astype(np.int64))
+        # dropping whole bins only: the bound is the value v with at most 5 samples strictly beyond it
+        assert lo[c] == min(0, max(v for v in range(-128, 1) if (srt < v).sum() <= 5))
+        assert hi[c] == max(0, min(v for v in range(0, 128) if (srt > v).sum() <= 5))
+        assert ((srt < lo[c]).sum() <= 5) and ((srt > hi[c]).sum() <= 5) and lo[c] <= 0 <= hi[c]
+    assert lo[5] == 0
+    # hand case: values -3 (x1), 0 (x7), 5 (x2); one sample per tail may go
+    h = np.zeros((1, 256), np.uint32)
+    h[0, 125], h[0, 128], h[0, 133] = 1, 7, 2
+    assert [x.tolist() for x in oracle.ranges_from_histogram(h, 1)] == [[0], [5]]
+    assert [x.tolist() for x in oracle.ranges_from_histogram(h, 2)] == [[0], [0]]
+
+
 def test_residual_reorder_moves_whole_groups():
     # hand case (Sec. 5 step 3): three groups of 2 channels, slab group j holds original group perm[j]
     x = np.array([[10, 11, 20, 21, 30, 31]], np.int8)
