@@ -3,6 +3,7 @@
     python -m paper_2510_02822_b200.sweep --config 2            # ViT-B linears, M = 12608
     python -m paper_2510_02822_b200.sweep --config 3            # ResNet-50 convolutions, batch 32
     python -m paper_2510_02822_b200.sweep --config 4 --cold     # DeiT-S small batch, L2 flushed between calls
+    python -m paper_2510_02822_b200.sweep --config 4 --stack    # DeiT-S 12-block stack, one CUDA graph per replica, cold and warm
     python -m paper_2510_02822_b200.sweep --config 5            # ViT-L stack, ratio switched between passes
 
 Prints one JSON line per (layer, ratio): device time of the prologue and of the mixed kernel
@@ -179,6 +180,76 @@ def run_stack(dev, batch, iters):
     fx.flexiq_check_status()
 
 
+def run_deit_stack(dev, batch, replicas, iters):
+    """DeiT-S stack of linears (12 blocks x 4 layers = 48 layer instances, each with its own weights,
+    input and output) captured in ONE CUDA graph per replica; `replicas` distinct copies of the whole
+    stack are replayed in turn so that nothing a replay touches is still in L2 from the previous time
+    (cold), then one replica is replayed alone (warm).  Reports time per pass and the algorithmic GB/s
+    (fp32 input + slab written and read + weights + int8 output) at ratios 0 / 0.5 / 1."""
+    M = batch * 197
+    stacks, total_bytes = [], 0
+    t0 = time.time()
+    base = {}
+    for i, (name, K, N) in enumerate(inputs.DEIT_S_LAYERS):
+        c = inputs.ranged_linear(f"deits_{name}", M, K, N, 16, seed=4000 + i)
+        perm, xs = calib.static_preparation(calib.quantize_reference(torch.from_numpy(c.Xcal), c.x_scale), torch.from_numpy(c.Wq), 16)
+        base[name] = (c, perm, xs)
+    for rep_i in range(replicas):
+        inst = []
+        for blk in range(12):
+            for name, K, N in inputs.DEIT_S_LAYERS:
+                c, perm, xs = base[name]
+                # distinct memory per instance (the values may repeat: only the addresses matter for the caches)
+                L = fx.Layer(torch.from_numpy(c.Wq).to(dev), torch.from_numpy(c.w_scale).to(dev), torch.from_numpy(c.bias).to(dev), perm, xs, 16)
+                X = torch.from_numpy(c.X).to(dev)
+                x4 = torch.empty(M * K + 16, dtype=torch.uint8, device=dev)
+                Y = torch.empty((M, N), dtype=torch.int8, device=dev)
+                inst.append((L, c, X, x4, Y))
+                total_bytes += 4 * K * N + M * K * 5 + M * N  # w8, w8m, wf, w4 ~ 3.5 K N; X fp32 + slab; Y
+        stacks.append(inst)
+    alg = sum(c.M * c.K * 4 + 2 * c.M * c.K + c.K * c.N + 8 * c.N + c.M * c.N for _, c, _, _, _ in stacks[0])
+    print(json.dumps({"setup_s": round(time.time() - t0, 1), "replicas": replicas, "instances": replicas * 48, "M": M,
+                      "resident_MB": round(total_bytes / 1e6, 1), "algorithmic_MB_per_pass": round(alg / 1e6, 2)}), flush=True)
+    stream = torch.cuda.current_stream()
+
+    def one_pass(inst):
+        for L, c, X, x4, Y in inst:
+            fx.flexiq_quantize_lower(L.h, X, fx.DTYPE_F32, c.M, c.x_scale, 0, x4, None)
+            fx.flexiq_mixed_gemm(L.h, x4, None, None, c.M, c.x_scale, c.y_scale, fx.OUT_REQUANT_I8, Y)
+
+    for ratio in (0.0, 0.5, 1.0):
+        graphs = []
+        for inst in stacks:
+            for L, *_ in inst:
+                L.set_lowbit_ratio(ratio)
+            one_pass(inst)  # weight operands move to this ratio outside the capture
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(g, stream=side):
+                    one_pass(inst)
+            graphs.append(g)
+        torch.cuda.synchronize()
+        res = {}
+        for label, order in (("cold", list(range(replicas))), ("warm", [0] * replicas)):
+            for gi in order:
+                graphs[gi].replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(iters):
+                for gi in order:
+                    graphs[gi].replay()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) / (iters * len(order)) * 1e3
+            res[label] = {"pass_us": round(us, 1), "us_per_layer": round(us / 48, 2), "alg_gbs": round(alg / us / 1e3, 1)}
+        print(json.dumps({"config": 4, "protocol": "48-layer graph per replica", "batch": batch, "ratio": ratio, **res}), flush=True)
+        del graphs
+    fx.flexiq_check_status()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", type=int, default=2)
@@ -187,6 +258,8 @@ def main():
     ap.add_argument("--graph", action="store_true", help="capture the launches in a CUDA graph and time its replay")
     ap.add_argument("--path", default="masked", choices=["masked", "packed"])
     ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--stack", action="store_true", help="config 4: 12-block DeiT-S stack in one CUDA graph, rotating replicas (cold) and one replica (warm)")
+    ap.add_argument("--replicas", type=int, default=0)
     args = ap.parse_args()
     dev = torch.device("cuda:0")
     path = fx.LOWBIT_PACKED_U4 if args.path == "packed" else fx.LOWBIT_MASKED_I8
@@ -199,6 +272,9 @@ def main():
     elif args.config == 3:
         for c in inputs.config3(args.batch or 32):
             time_case(c, True, dev, path, args.iters, args.cold, flush, args.graph)
+    elif args.config == 4 and args.stack:
+        b = args.batch or 1
+        run_deit_stack(dev, b, args.replicas or (10 if b == 1 else 4), max(2, args.iters // 10))
     elif args.config == 4:
         for c in inputs.config4(args.batch or 1):
             time_case(c, False, dev, path, args.iters, args.cold, flush, args.graph)
