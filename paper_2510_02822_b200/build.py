@@ -36,7 +36,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
             cmd.insert(1, "-Xptxas=-v")
         subprocess.run(cmd, check=True)
         objs.append(obj)
-    subprocess.run([nvcc, "-shared", "-o", LIB, *objs, "-cudart", "static"], check=True)
+    subprocess.run([nvcc, "-shared", "-Wno-deprecated-gpu-targets", "-o", LIB, *objs, "-cudart", "static"], check=True)
     return LIB
 
 
