@@ -102,6 +102,10 @@ int flexiq_layer_set_lowbit_path(flexiq_layer_t layer, int lowbit_path);
 /* Run-time ratio switch (Sec. 7, "Low-bitwidth Ratio Adjustment"): sets
  * max_4bit_ch = K_lo = ceil(ratio * n_g - 1e-4) * G, clamped to [0, K].  Host-only, one
  * integer, no data movement.  Takes effect for calls enqueued afterwards.
+ * The slabs a flexiq_quantize_lower call writes belong to the ratio in force when it was enqueued,
+ * and the mixed_* call that reads them must be enqueued at the same ratio: the library does not
+ * record which ratio a caller's buffer was written at (slabs of several ratios may be prepared ahead
+ * and used later), so a mismatch is not detected and gives wrong values, never an out-of-bounds access.
  * ratio outside [0, 1] or NaN: FLEXIQ_ERR_INVALID_ARG. */
 int flexiq_set_lowbit_ratio(flexiq_layer_t layer, float ratio);
 int flexiq_get_max_4bit_ch(flexiq_layer_t layer, int *K_lo);
