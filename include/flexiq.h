@@ -105,7 +105,10 @@ int flexiq_layer_set_lowbit_path(flexiq_layer_t layer, int lowbit_path);
  * The slabs a flexiq_quantize_lower call writes belong to the ratio in force when it was enqueued,
  * and the mixed_* call that reads them must be enqueued at the same ratio: the library does not
  * record which ratio a caller's buffer was written at (slabs of several ratios may be prepared ahead
- * and used later), so a mismatch is not detected and gives wrong values, never an out-of-bounds access.
+ * and used later), so a mismatch is not detected and gives wrong values.  On the PACKED path the
+ * mixed_* call addresses X4_dev / X8_dev with the row pitches of the ratio in force when IT is
+ * enqueued: buffers sized for a smaller low-bit slice would then be read past their end, so size
+ * them for the largest ratio used (the MASKED slab is [M][K] at every ratio).
  * ratio outside [0, 1] or NaN: FLEXIQ_ERR_INVALID_ARG. */
 int flexiq_set_lowbit_ratio(flexiq_layer_t layer, float ratio);
 int flexiq_get_max_4bit_ch(flexiq_layer_t layer, int *K_lo);
