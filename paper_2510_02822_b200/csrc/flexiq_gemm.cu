@@ -245,11 +245,11 @@ struct EpilogueCtx {
     int parts, arrivals_on;  // column parts per tile (4 or 2); this warp arrives on the accumulator barrier
 };
 
-// One epilogue warp: TMEM lane quadrant `quad` (32 rows, lane = row), column quarter `part`
-// (BN/4 = 16..64 columns per pass; two passes when only eight warps drain the tile) of every
-// tile of this CTA.  Per pass: fetch the columns' factors,
-// read the whole slice of the accumulator into registers, hand the accumulator back, then
-// scale / round / clip and store each row's bytes straight to global memory.
+// One epilogue warp: TMEM lane quadrant `quad` (32 rows, lane = row), column slot `part` (32 or 64
+// columns per pass; two passes when only eight warps drain the tile) of every tile of this CTA.
+// Per pass: fetch the columns' factors, read the whole slice of the accumulator into registers,
+// hand the accumulator back, then scale / round / clip; int8 results are staged in shared memory
+// and leave through tiled bulk stores, 4-byte results go straight to global memory row by row.
 template <int CG, int MODE>
 __device__ __forceinline__ void epilogue_role(const GemmParams &p, const EpilogueCtx &x, int quad, int part, int lane)
 {
