@@ -1,6 +1,7 @@
 """Runs one layer shape of the benchmark configurations a few times, for profilers.
 
     python -m paper_2510_02822_b200.profile_case --layer vitb_qkv --ratio 0.5 --iters 3
+    python -m paper_2510_02822_b200.profile_case --layer vitb_fc2 --aux reorder       # residual reorder of the layer's input
 
 Prints the average device time of the prologue and of the mixed GEMM (CUDA events on the
 launching stream).  Layers: vitb_{qkv,proj,fc1,fc2}, vitl_{...}, deits_{...} (append
@@ -45,6 +46,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=1)
     ap.add_argument("--path", default="masked", choices=["masked", "packed"])
     ap.add_argument("--out", default="i8", choices=["i8", "f32", "i32"])
+    ap.add_argument("--aux", default="", choices=["", "reorder", "calib"], help="run an auxiliary kernel on the layer's input instead: the residual reorder operator or the calibration range kernels")
     args = ap.parse_args()
     dev = torch.device("cuda:0")
     c, is_conv = make_case(args.layer)
@@ -58,6 +60,32 @@ def main():
     mode = {"i8": fx.OUT_REQUANT_I8, "f32": fx.OUT_DEQUANT_F32, "i32": fx.OUT_ACC_I32}[args.out]
     M = X.numel() // L.K
     stream = torch.cuda.current_stream()
+    if args.aux:
+        Xq = X.reshape(-1, L.K)
+        lo = torch.empty(L.K, dtype=torch.int32, device=dev)
+        hi = torch.empty(L.K, dtype=torch.int32, device=dev)
+        Yr = torch.empty_like(Xq)
+
+        def aux():
+            if args.aux == "reorder":
+                L.reorder_channels(Xq, fx.REORDER_TO_SLAB, Y=Yr)
+            else:
+                fx.flexiq_calib_channel_ranges(Xq, fx._dtype_code(Xq), Xq.shape[0], L.K, c.x_scale, False, lo, hi)
+
+        for _ in range(args.warmup):
+            aux()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(args.iters):
+            aux()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        t = e0.elapsed_time(e1) / args.iters
+        moved = Xq.numel() * Xq.element_size() * (2 if args.aux == "reorder" else 1)
+        print(f"{args.layer} {args.aux}: {t * 1e3:.1f} us, {moved / t / 1e6:.0f} GB/s")
+        L.close()
+        return
 
     def mixed(x4, x8):
         if is_conv:
