@@ -9,6 +9,13 @@
 
 namespace flexiq {
 
+// Loads 8 fp32 channels starting at p.
+__device__ __forceinline__ void load8(const void *p, float x[8])
+{
+    const float4 a = __ldg(reinterpret_cast<const float4 *>(p)), b = __ldg(reinterpret_cast<const float4 *>(p) + 1);
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+}
+
 // Per-channel range [lo, hi] (lo <= 0 <= hi) of the Eq. 1-quantized activations over all rows.
 // A block owns a window of 256 channels (16 chunks of 16) and a slice of the rows: thread
 // (chunk, row lane) walks its rows with byte-parallel min / max, the block merges in shared
@@ -46,9 +53,35 @@ __global__ void calib_ranges_kernel(const void *__restrict__ X, long long M, int
                 if (l < 0) atomicMin(&lo_s[c], l);
                 if (h > 0) atomicMax(&hi_s[c], h);
             }
-    } else if (c0 < K) {
+    } else if (DTYPE == FLEXIQ_DTYPE_F32) {
         // Eq. 1 is monotone in x (correctly rounded division by S > 0, rounding, clipping), so the range of
         // the quantized values is the quantized range of the inputs: min / max in floating point, quantize last.
+        // Eight channels per thread (32 half-chunks x 8 row lanes): sixteen running values keep the register
+        // count, and with it the number of loads in flight per SM, where a bandwidth-bound kernel needs it.
+        const int half = threadIdx.x & 31, rl = threadIdx.x >> 5;
+        const int c8 = win * kCalibWindow + 8 * half;
+        if (c8 < K) {
+            float lo_f[8], hi_f[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) { lo_f[k] = 0.f; hi_f[k] = 0.f; }
+            for (long long m = (long long)slice * 8 + rl; m < M; m += (long long)slices * 8) {
+                float x[8];
+                load8(reinterpret_cast<const char *>(X) + ((size_t)m * K + c8) * 4, x);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    lo_f[k] = fminf(lo_f[k], x[k]);
+                    hi_f[k] = fmaxf(hi_f[k], x[k]);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int l = __float2int_rn(fmaxf(div(lo_f[k]), -128.f)), h = __float2int_rn(fminf(div(hi_f[k]), 127.f));
+                if (l < 0) atomicMin(&lo_s[8 * half + k], l);
+                if (h > 0) atomicMax(&hi_s[8 * half + k], h);
+            }
+        }
+    } else if (c0 < K) {
+        // 16-bit inputs: sixteen channels (32 bytes) per thread
         float lo_f[16], hi_f[16];
 #pragma unroll
         for (int k = 0; k < 16; ++k) { lo_f[k] = 0.f; hi_f[k] = 0.f; }
@@ -226,7 +259,7 @@ static int launch_ranges(const void *X, long long M, int K, float S, int32_t *lo
 {
     const int windows = (K + kCalibWindow - 1) / kCalibWindow;
     long long slices = ((long long)sms * 3 + windows - 1) / windows;   // about three blocks per SM: few, long-lived blocks amortise the merge
-    const long long max_slices = (M + 15) / 16;
+    const long long max_slices = (M + 15) / 16;   // (fewer rows than lanes leave lanes idle, nothing more)
     if (slices > max_slices) slices = max_slices;
     calib_ranges_kernel<DTYPE><<<(unsigned)(windows * slices), kCalibWindow, 0, st>>>(X, M, K, S, (int)slices, lo, hi);
     FLEXIQ_CUDA_TRY(cudaGetLastError());
