@@ -68,7 +68,7 @@ class ClockSampler:
         time.sleep(0.12)
         self.proc.terminate()
         rows = [s for t, s in self.samples if t0 <= t <= t1 + 0.06] or [s for _, s in self.samples[-5:]]
-        sm, mx, reasons = [], None, set()
+        sm, mx, reasons, watts = [], None, set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in rows:
             f = [x.strip() for x in r.split(",")]
@@ -77,10 +77,15 @@ class ClockSampler:
                 mx = float(f[1])
             except Exception:
                 continue
+            try:
+                watts.append(float(f[2]))
+            except Exception:
+                pass
             for n, v in zip(names, f[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
-        out = {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(sm)}
+        out = {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons), "samples": len(sm),
+               "power_w": max(watts) if watts else None}
         if not sm:
             out["note"] = (self.samples[-1][1] if self.samples else "no output from nvidia-smi")[:160]
         return out
