@@ -176,3 +176,24 @@ def config3(batch=32):
 
 def config4(batch=1):
     return [ranged_linear(f"cfg4_deits_b{batch}_{n}", batch * 197, K, N, 16, seed=4000 + i) for i, (n, K, N) in enumerate(DEIT_S_LAYERS)]
+
+
+# ------------------------------------------------------------------ request traces (serving experiment)
+def poisson_arrivals(seed: int, rate: float, n: int) -> np.ndarray:
+    """Arrival times (seconds, ascending) of n requests of a Poisson process with `rate` requests per
+    second, the request pattern of the paper's serving experiment (100 to 3000 requests per second)."""
+    gaps = -np.log(1.0 - uniform(seed, 900, n)) / float(rate)
+    return np.cumsum(gaps)
+
+
+def fluctuating_arrivals(seed: int, rate_min: float, rate_max: float, period_s: float, duration_s: float) -> np.ndarray:
+    """Arrival times of a Poisson process whose rate swings between rate_min and rate_max (the paper
+    sets the peak to three times the minimum) along a raised cosine of the given period: stands in for
+    the public cloud traces the paper replays, which are not available here.  Drawn by thinning a
+    process of rate rate_max."""
+    n = int(rate_max * duration_s * 1.2) + 64
+    t = poisson_arrivals(seed, rate_max, n)
+    t = t[t < duration_s]
+    rate_t = rate_min + (rate_max - rate_min) * 0.5 * (1.0 - np.cos(2.0 * np.pi * t / period_s))
+    keep = uniform(seed, 901, t.size) * rate_max < rate_t
+    return t[keep]
