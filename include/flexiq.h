@@ -289,6 +289,46 @@ int flexiq_calib_absmax_ema(const void *X_dev, int x_dtype, int64_t count, float
 int flexiq_reorder_channels(flexiq_layer_t layer, const void *X_dev, int elem_bytes, int64_t M,
                             int direction, void *Y_dev, void *stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Run-time ratio controller and request queue (Sec. 8, "Adapting to Workload Fluctuation" and
+ * the Poisson serving experiment).  Host-only: no device work, no stream.
+ *
+ * Levels are the low-bit ratios a deployment switches between (0, 25, 50, 75, 100 % in the
+ * paper: n_levels = 5, level l = ratio l / (n_levels - 1)); the caller applies a level with
+ * flexiq_set_lowbit_ratio.  The controller holds the latency that was profiled per level over a
+ * grid of request rates and, given the request rate it is shown, moves the level one step up
+ * when the profiled latency of the current level at that rate is above the threshold; one step
+ * down when the next lower level's profiled latency at that rate is within the threshold (the
+ * paper states only the step up; its fluctuating-rate figure needs both).  Between two grid
+ * rates the profiled latency is interpolated linearly; outside the grid the end value holds.
+ *   rate_grid_host [n_rates]            requests per second, strictly ascending, n_rates >= 1
+ *   latency_host   [n_levels][n_rates]  profiled latency, seconds (any statistic: median, p90)
+ *   threshold      seconds;  window_s   seconds of arrivals the rate is measured over (> 0)
+ * All arrays are copied; the handle is freed by flexiq_controller_destroy. */
+typedef struct flexiq_controller *flexiq_controller_t;
+int flexiq_controller_create(flexiq_controller_t *out, int n_levels, int n_rates, const double *rate_grid_host,
+                             const double *latency_host, double threshold, double window_s, int initial_level);
+int flexiq_controller_destroy(flexiq_controller_t ctrl);
+int flexiq_controller_level(flexiq_controller_t ctrl, int *level);
+/* one decision from an observed request rate; *level receives the level after it */
+int flexiq_controller_update(flexiq_controller_t ctrl, double rate, int *level);
+
+/* The request queue of the serving experiment in virtual time: one accelerator, first come first
+ * served.  When the accelerator is free it takes every request that has arrived by then, oldest
+ * first, up to max_batch (max_batch = 1: the plain single-server queue), serves the batch for
+ * service_host[level][batch - 1] seconds and completes all its requests together.  With a
+ * controller, a dispatch that starts at least window_s after the previous decision (the first is
+ * due at time window_s) first shows the controller the rate = arrivals in the last window_s
+ * before the dispatch / window_s; the controller's level is left where the run ended.  Without
+ * one (ctrl NULL) every batch runs at fixed_level.
+ *   arrival_host  [n]  seconds, ascending        service_host [n_levels][max_batch] seconds
+ *   response_host [n]  completion - arrival      level_host   [n] level that served each request
+ * n == 0 is a successful no-op.  Errors: FLEXIQ_ERR_INVALID_ARG (NULL, sizes, unsorted arrivals,
+ * level out of range, n_levels different from the controller's). */
+int flexiq_serving_simulate(flexiq_controller_t ctrl, int fixed_level, int64_t n, const double *arrival_host,
+                            int n_levels, int max_batch, const double *service_host, double *response_host,
+                            int32_t *level_host);
+
 /* Test hooks: copy the layer's derived tables to host buffers (any may be NULL).
  *   sw_host [K/G][N] uint8 weight extraction positions (slab order),
  *   w8_host [N][Kw] int8 slab-order weights, w4_host [N][Kw/2] packed 4-bit weights,

@@ -27,6 +27,8 @@ EXPORTS = [
     "flexiq_mixed_gemm_to_slab", "flexiq_mixed_conv_to_slab", "flexiq_reorder_channels",
     "flexiq_calib_channel_ranges", "flexiq_calib_channel_histogram", "flexiq_calib_ranges_from_histogram",
     "flexiq_calib_weight_absmax", "flexiq_calib_prepare", "flexiq_calib_absmax_ema",
+    "flexiq_controller_create", "flexiq_controller_destroy", "flexiq_controller_level", "flexiq_controller_update",
+    "flexiq_serving_simulate",
     "flexiq_layer_export", "flexiq_force_tile", "flexiq_check_status", "flexiq_last_error",
 ]
 
@@ -72,6 +74,12 @@ def lib():
         L.flexiq_calib_absmax_ema.argtypes = [vp, i32, i64, f32, vp, vp]
         L.flexiq_layer_export.argtypes = [vp, vp, vp, vp]
         L.flexiq_check_status.argtypes = [vp]
+        f64 = C.c_double
+        L.flexiq_controller_create.argtypes = [C.POINTER(vp), i32, i32, vp, vp, f64, f64, i32]
+        L.flexiq_controller_destroy.argtypes = [vp]
+        L.flexiq_controller_level.argtypes = [vp, C.POINTER(i32)]
+        L.flexiq_controller_update.argtypes = [vp, f64, C.POINTER(i32)]
+        L.flexiq_serving_simulate.argtypes = [vp, i32, i64, vp, i32, i32, vp, vp, vp]
         _lib = L
     return _lib
 
@@ -337,3 +345,63 @@ class Layer:
             Y = torch.empty((Nb, P, Q, self.N), dtype=dt, device=self.device)
         flexiq_mixed_conv(self.h, x4, x8, x_shift, Nb, H, W, x_scale, y_scale, out_mode, Y)
         return Y
+
+
+# ------------------------------------------------------------------ ratio controller and request queue (host only)
+def _np_ptr(a):
+    return C.c_void_p(a.ctypes.data)
+
+
+class Controller:
+    """Run-time ratio controller (flexiq_controller_*): levels are the ratios l / (n_levels - 1)."""
+
+    def __init__(self, rate_grid, latency, threshold, window_s, initial_level=0):
+        import numpy as np
+        self.rate_grid = np.ascontiguousarray(rate_grid, dtype=np.float64)
+        self.latency = np.ascontiguousarray(latency, dtype=np.float64)
+        if self.latency.ndim != 2 or self.latency.shape[1] != self.rate_grid.size:
+            raise ValueError("latency must be [n_levels][n_rates]")
+        self.n_levels = self.latency.shape[0]
+        h = C.c_void_p()
+        _check(lib().flexiq_controller_create(C.byref(h), self.n_levels, self.rate_grid.size, _np_ptr(self.rate_grid),
+                                              _np_ptr(self.latency), float(threshold), float(window_s), int(initial_level)))
+        self.h = h
+
+    @property
+    def level(self) -> int:
+        v = C.c_int()
+        _check(lib().flexiq_controller_level(self.h, C.byref(v)))
+        return v.value
+
+    def update(self, rate: float) -> int:
+        v = C.c_int()
+        _check(lib().flexiq_controller_update(self.h, float(rate), C.byref(v)))
+        return v.value
+
+    def ratio(self) -> float:
+        return self.level / max(1, self.n_levels - 1)
+
+    def close(self):
+        if self.h is not None and self.h.value:
+            _check(lib().flexiq_controller_destroy(self.h))
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def flexiq_serving_simulate(ctrl, fixed_level, arrival, service, max_batch):
+    """Request queue in virtual time; returns (response seconds [n], level [n])."""
+    import numpy as np
+    arrival = np.ascontiguousarray(arrival, dtype=np.float64)
+    service = np.ascontiguousarray(service, dtype=np.float64)
+    if service.ndim != 2 or service.shape[1] != max_batch:
+        raise ValueError("service must be [n_levels][max_batch]")
+    response = np.zeros(arrival.size, dtype=np.float64)
+    level = np.zeros(arrival.size, dtype=np.int32)
+    _check(lib().flexiq_serving_simulate(ctrl.h if ctrl is not None else None, int(fixed_level), arrival.size, _np_ptr(arrival),
+                                         service.shape[0], int(max_batch), _np_ptr(service), _np_ptr(response), _np_ptr(level)))
+    return response, level
