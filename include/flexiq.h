@@ -99,6 +99,15 @@ int flexiq_layer_destroy(flexiq_layer_t layer);
  * its slabs. */
 int flexiq_layer_set_lowbit_path(flexiq_layer_t layer, int lowbit_path);
 
+/* Brings the layer's private weight operand to the ratio in force, in stream order (a copy of the
+ * channel groups that changed sides since the last mixed_* call; nothing when none did).  The
+ * mixed_* calls do this themselves; the explicit call is for CUDA graphs: a graph captured while
+ * ratio r was in force holds no such copy, so before it is replayed after another ratio was used,
+ * set r again (flexiq_set_lowbit_ratio) and call this on the replaying stream.  One graph per ratio
+ * and problem size can then be kept and replayed in any order (Sec. 7: the ratio changes at run
+ * time without re-packing the weights). */
+int flexiq_layer_sync_ratio(flexiq_layer_t layer, void *stream);
+
 /* Run-time ratio switch (Sec. 7, "Low-bitwidth Ratio Adjustment"): sets
  * max_4bit_ch = K_lo = ceil(ratio * n_g - 1e-4) * G, clamped to [0, K].  Host-only, one
  * integer, no data movement.  Takes effect for calls enqueued afterwards.

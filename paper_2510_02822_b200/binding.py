@@ -22,7 +22,7 @@ REORDER_TO_SLAB, REORDER_FROM_SLAB = 0, 1
 
 EXPORTS = [
     "flexiq_layer_create_linear", "flexiq_layer_create_conv", "flexiq_layer_destroy",
-    "flexiq_layer_set_lowbit_path", "flexiq_set_lowbit_ratio", "flexiq_get_max_4bit_ch",
+    "flexiq_layer_set_lowbit_path", "flexiq_layer_sync_ratio", "flexiq_set_lowbit_ratio", "flexiq_get_max_4bit_ch",
     "flexiq_x4_pitch", "flexiq_quantize_lower", "flexiq_quantize_lower_dynamic_noalloc", "flexiq_mixed_gemm", "flexiq_mixed_conv",
     "flexiq_mixed_gemm_to_slab", "flexiq_mixed_conv_to_slab", "flexiq_reorder_channels",
     "flexiq_calib_channel_ranges", "flexiq_calib_channel_histogram", "flexiq_calib_ranges_from_histogram",
@@ -56,6 +56,7 @@ def lib():
         L.flexiq_layer_create_conv.argtypes = [C.POINTER(vp), i32, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         L.flexiq_layer_destroy.argtypes = [vp]
         L.flexiq_layer_set_lowbit_path.argtypes = [vp, i32]
+        L.flexiq_layer_sync_ratio.argtypes = [vp, vp]
         L.flexiq_set_lowbit_ratio.argtypes = [vp, f32]
         L.flexiq_get_max_4bit_ch.argtypes = [vp, C.POINTER(i32)]
         L.flexiq_x4_pitch.argtypes = [vp, i32, C.POINTER(i64)]
@@ -278,6 +279,10 @@ class Layer:
 
     def set_lowbit_ratio(self, ratio):
         flexiq_set_lowbit_ratio(self.h, ratio)
+
+    def sync_ratio(self):
+        """Weight operand to the ratio in force, on the current stream (needed only before a CUDA-graph replay)."""
+        _check(lib().flexiq_layer_sync_ratio(self.h, _stream()))
 
     @property
     def K_lo(self):

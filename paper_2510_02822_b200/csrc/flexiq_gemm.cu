@@ -1003,6 +1003,22 @@ static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const
     return FLEXIQ_OK;
 }
 
+// Masked path: the weight operand wf follows the ratio lazily.  Only the channel groups that changed
+// sides since the last update are copied (from w8m when they became low-bit, from w8 when they
+// returned to 8 bits), in stream order.
+static int sync_weight_operand(Layer *L, cudaStream_t st)
+{
+    const int C_lo = L->K_lo;
+    if (L->wf_K_lo == C_lo) return FLEXIQ_OK;
+    const int k_from = C_lo < L->wf_K_lo ? C_lo : L->wf_K_lo, k_to = C_lo < L->wf_K_lo ? L->wf_K_lo : C_lo;
+    const long long total = (long long)L->N * L->R * L->S * ((k_to - k_from) >> 4);
+    patch_weights_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(L->wf, C_lo > L->wf_K_lo ? L->w8m : L->w8, L->N,
+                                                                          L->R * L->S, L->C, k_from, k_to);
+    FLEXIQ_CUDA_TRY(cudaGetLastError());
+    L->wf_K_lo = C_lo;
+    return FLEXIQ_OK;
+}
+
 static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_t *x_shift, long long M, int Nb, int H,
                      int W, float x_scale, float y_scale, int out_mode, void *Y, cudaStream_t st,
                      const Layer *next = nullptr, int relu = 0, int out_order = 0)
@@ -1041,14 +1057,8 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
         // Masked path: activations are one slab [rows][C] and the weights one operand wf, so the
         // mainloop is a plain 8-bit GEMM over whole K blocks whatever the ratio.  wf follows the
         // ratio lazily: only the channel groups that changed sides are copied, in stream order.
-        if (L->wf_K_lo != C_lo) {
-            const int k_from = C_lo < L->wf_K_lo ? C_lo : L->wf_K_lo, k_to = C_lo < L->wf_K_lo ? L->wf_K_lo : C_lo;
-            const long long total = (long long)L->N * L->R * L->S * ((k_to - k_from) >> 4);
-            patch_weights_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(L->wf, C_lo > L->wf_K_lo ? L->w8m : L->w8, L->N,
-                                                                                  L->R * L->S, L->C, k_from, k_to);
-            FLEXIQ_CUDA_TRY(cudaGetLastError());
-            L->wf_K_lo = C_lo;
-        }
+        int rcw = sync_weight_operand(L, st);
+        if (rcw) return rcw;
     }
     GemmParams p{};
     p.M = M; p.N = L->N; p.C = L->C; p.C_lo = packed ? C_lo : 0; p.C_hi = packed ? C_hi : L->C;
@@ -1256,4 +1266,14 @@ extern "C" int flexiq_check_status(void *stream)
         return set_error(FLEXIQ_ERR_TIMEOUT, "a bounded device-side wait expired (status word 0x%x)", word);
     }
     return FLEXIQ_OK;
+}
+
+extern "C" int flexiq_layer_sync_ratio(flexiq_layer_t layer, void *stream)
+{
+    Layer *L = as_layer(layer);
+    if (!L) return set_error(FLEXIQ_ERR_INVALID_ARG, "not a live flexiq layer handle");
+    if (L->lowbit_path == FLEXIQ_LOWBIT_PACKED_U4 && L->K_lo > 0) return FLEXIQ_OK;  // that path reads w4 and w8 as they are
+    int rc = check_device_sm100();
+    if (rc) return rc;
+    return sync_weight_operand(L, reinterpret_cast<cudaStream_t>(stream));
 }
