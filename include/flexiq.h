@@ -338,6 +338,48 @@ int flexiq_serving_simulate(flexiq_controller_t ctrl, int fixed_level, int64_t n
                             int n_levels, int max_batch, const double *service_host, double *response_host,
                             int32_t *level_host);
 
+/* ---------------------------------------------------------------------------------------------
+ * Evolutionary selection of the low-bitwidth channel groups (Sec. 4.2, Algorithm 1).
+ *
+ * A chromosome is one flag (uint8 0/1) per channel group, layer after layer: groups_host[l] flags
+ * for layer l, `total` = their sum; 1 = computed from 4-bit values.  score_host[total] is the error
+ * estimation score of each group (activation range x largest weight range, flexiq_calib_prepare's
+ * score_dev; 0 <= score < 2^31).  locked_host (or NULL) marks groups that every chromosome keeps
+ * set: the selection of the next smaller ratio, so that selections stay nested across ratios.
+ * The fitness of a chromosome is the caller's: run the model with each layer's selected groups
+ * first in group_perm and K_lo = their number, and take the squared distance of its outputs from
+ * the 8-bit model's (flexiq_sq_distance_i8); smaller is fitter.
+ *
+ * Randomness is counter based (splitmix64 finaliser over seed, generation, individual, draw index),
+ * so a run is reproducible from `seed`.  Probabilities "inversely proportional to the score" are the
+ * integer weights 2^32 / (1 + score); a flag to clear is drawn with weight 1 + score.
+ *
+ * flexiq_evo_init: population_host [N][total] receives the seeds: chromosome 0 is the greedy
+ *   selection (per layer its per_layer_target_host[l] lowest scores, ties by index, locked first),
+ *   the others set the locked flags and then draw flags over the whole model, low scores preferred,
+ *   until they hold as many as chromosome 0; *target_out = that number.
+ * flexiq_evo_next_generation: distance_host [N] = fitness of population_host's chromosomes.  The k
+ *   fittest are copied unchanged (rank order, ties by index); the other N - k places are filled pair
+ *   by pair: two parents drawn among the r fittest, one crossover point at a layer boundary, the two
+ *   children that swap the parts right of it (an odd last place takes the first child); then each
+ *   child is mutated: every set, unlocked flag is cleared with probability mutation_bp / 10000
+ *   (100 = the paper's 1 %) and as many flags of the same layer that were unset are set, low scores
+ *   preferred; finally flags are cleared (high scores first in probability) or set until the
+ *   chromosome holds `target` flags again.  generation >= 0 numbers the call.
+ * Host-only, no device work.  Errors: FLEXIQ_ERR_INVALID_ARG. */
+int flexiq_evo_init(int n_layers, const int32_t *groups_host, const int64_t *score_host,
+                    const uint8_t *locked_host, const int32_t *per_layer_target_host, int N, uint64_t seed,
+                    uint8_t *population_host, int64_t *target_out);
+int flexiq_evo_next_generation(int n_layers, const int32_t *groups_host, const int64_t *score_host,
+                               const uint8_t *locked_host, int64_t target, int N, int k, int r,
+                               int mutation_bp, uint64_t seed, int generation, const int64_t *distance_host,
+                               const uint8_t *population_host, uint8_t *next_population_host);
+
+/* Fitness reduction (Sec. 4.2: L2 distance from the outputs of the high-bitwidth model), exact:
+ * *out_dev = sum over i < n of (A[i] - B[i])^2 for int8 tensors, as int64.  out_dev is zeroed and
+ * written in stream order; A_dev, B_dev 16-byte aligned; n == 0 gives 0. */
+int flexiq_sq_distance_i8(const int8_t *A_dev, const int8_t *B_dev, int64_t n, int64_t *out_dev, void *stream);
+
 /* Test hooks: copy the layer's derived tables to host buffers (any may be NULL).
  *   sw_host [K/G][N] uint8 weight extraction positions (slab order),
  *   w8_host [N][Kw] int8 slab-order weights, w4_host [N][Kw/2] packed 4-bit weights,

@@ -28,7 +28,7 @@ EXPORTS = [
     "flexiq_calib_channel_ranges", "flexiq_calib_channel_histogram", "flexiq_calib_ranges_from_histogram",
     "flexiq_calib_weight_absmax", "flexiq_calib_prepare", "flexiq_calib_absmax_ema",
     "flexiq_controller_create", "flexiq_controller_destroy", "flexiq_controller_level", "flexiq_controller_update",
-    "flexiq_serving_simulate",
+    "flexiq_serving_simulate", "flexiq_evo_init", "flexiq_evo_next_generation", "flexiq_sq_distance_i8",
     "flexiq_layer_export", "flexiq_force_tile", "flexiq_check_status", "flexiq_last_error",
 ]
 
@@ -81,6 +81,10 @@ def lib():
         L.flexiq_controller_level.argtypes = [vp, C.POINTER(i32)]
         L.flexiq_controller_update.argtypes = [vp, f64, C.POINTER(i32)]
         L.flexiq_serving_simulate.argtypes = [vp, i32, i64, vp, i32, i32, vp, vp, vp]
+        u64 = C.c_uint64
+        L.flexiq_evo_init.argtypes = [i32, vp, vp, vp, vp, i32, u64, vp, C.POINTER(i64)]
+        L.flexiq_evo_next_generation.argtypes = [i32, vp, vp, vp, i64, i32, i32, i32, i32, u64, i32, vp, vp, vp]
+        L.flexiq_sq_distance_i8.argtypes = [vp, vp, i64, vp, vp]
         _lib = L
     return _lib
 
@@ -410,3 +414,52 @@ def flexiq_serving_simulate(ctrl, fixed_level, arrival, service, max_batch):
     _check(lib().flexiq_serving_simulate(ctrl.h if ctrl is not None else None, int(fixed_level), arrival.size, _np_ptr(arrival),
                                          service.shape[0], int(max_batch), _np_ptr(service), _np_ptr(response), _np_ptr(level)))
     return response, level
+
+
+# ------------------------------------------------------------------ evolutionary selection (Sec. 4.2, Algorithm 1)
+def _evo_args(groups, score, locked):
+    import numpy as np
+    groups = np.ascontiguousarray(groups, dtype=np.int32)
+    score = np.ascontiguousarray(score, dtype=np.int64)
+    if score.size != int(groups.sum()):
+        raise ValueError("score must hold one value per group of every layer")
+    if locked is not None:
+        locked = np.ascontiguousarray(locked, dtype=np.uint8)
+        if locked.size != score.size:
+            raise ValueError("locked must hold one flag per group")
+    return groups, score, locked
+
+
+def flexiq_evo_init(groups, score, per_layer_target, N, seed, locked=None):
+    """Seed population [N][total] uint8 and the number of set flags every chromosome holds."""
+    import numpy as np
+    groups, score, locked = _evo_args(groups, score, locked)
+    tgt = np.ascontiguousarray(per_layer_target, dtype=np.int32)
+    if tgt.size != groups.size:
+        raise ValueError("per_layer_target must hold one value per layer")
+    pop = np.zeros((int(N), score.size), dtype=np.uint8)
+    target = C.c_int64()
+    _check(lib().flexiq_evo_init(groups.size, _np_ptr(groups), _np_ptr(score), None if locked is None else _np_ptr(locked),
+                                 _np_ptr(tgt), int(N), int(seed), _np_ptr(pop), C.byref(target)))
+    return pop, target.value
+
+
+def flexiq_evo_next_generation(pop, distance, groups, score, target, k, r, mutation_bp, seed, generation, locked=None):
+    import numpy as np
+    groups, score, locked = _evo_args(groups, score, locked)
+    pop = np.ascontiguousarray(pop, dtype=np.uint8)
+    distance = np.ascontiguousarray(distance, dtype=np.int64)
+    if pop.ndim != 2 or pop.shape[1] != score.size or distance.size != pop.shape[0]:
+        raise ValueError("pop must be [N][total] and distance [N]")
+    nxt = np.zeros_like(pop)
+    _check(lib().flexiq_evo_next_generation(groups.size, _np_ptr(groups), _np_ptr(score), None if locked is None else _np_ptr(locked),
+                                            int(target), pop.shape[0], int(k), int(r), int(mutation_bp), int(seed), int(generation),
+                                            _np_ptr(distance), _np_ptr(pop), _np_ptr(nxt)))
+    return nxt
+
+
+def flexiq_sq_distance_i8(A, B, out):
+    """out (int64 device tensor, one element) = sum (A - B)^2 over two int8 device tensors."""
+    if A.numel() != B.numel():
+        raise ValueError("A and B differ in size")
+    _check(lib().flexiq_sq_distance_i8(_ptr(A), _ptr(B), A.numel(), _ptr(out), _stream()))

@@ -8,7 +8,7 @@ _DIR = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_DIR)
 CSRC = os.path.join(_DIR, "csrc")
 LIB = os.path.join(_DIR, "libflexiq.so")
-SOURCES = ["flexiq_layer.cu", "flexiq_prologue.cu", "flexiq_gemm.cu", "flexiq_reorder.cu", "flexiq_calib.cu", "flexiq_serving.cu"]
+SOURCES = ["flexiq_layer.cu", "flexiq_prologue.cu", "flexiq_gemm.cu", "flexiq_reorder.cu", "flexiq_calib.cu", "flexiq_serving.cu", "flexiq_evolution.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "--fmad=false",  # the epilogue spells out its fused multiply-adds; nothing else may contract

@@ -5,6 +5,7 @@ import itertools
 
 import numpy as np
 
+import helpers
 from oracle import evolution as ev
 
 
@@ -126,33 +127,8 @@ def test_selection_perm_puts_selected_groups_first():
     assert perm == [1, 2, 4, 0, 3] and n_low == 3
 
 
-def _tiny_stack(seed=50, M=48, dims=(64, 96, 64), G=16, small=False):
-    import oracle
-    from paper_2510_02822_b200 import inputs
-    layers, X0 = [], None
-    K = dims[0]
-    for l, N in enumerate(dims[1:] + (dims[-1],)):
-        c = inputs.ranged_linear(f"evo{l}", M, K, N, G, seed=seed + l, group_structured=True)
-        Wq = np.clip(c.Wq, -7, 7) if small else c.Wq
-        if X0 is None:
-            X0 = c.X * (np.float32(0.05) if small else np.float32(1.0))
-        layers.append(dict(Wq=Wq, w_scale=c.w_scale, bias=c.bias, x_scale=c.x_scale, y_scale=c.y_scale, G=G,
-                           sx_group=np.zeros(K // G, np.uint8)))
-        K = N
-    # chain the scales: a layer's output scale is the next layer's input scale
-    for l in range(len(layers) - 1):
-        layers[l + 1]["x_scale"] = layers[l]["y_scale"]
-    q = oracle.quantize(X0, layers[0]["x_scale"])
-    for L in layers:  # static positions from the 8-bit chain's own activations
-        lo, hi = oracle.channel_ranges(q)
-        L["sx_group"] = np.zeros_like(oracle.static_positions(lo, hi, G)) if small else oracle.static_positions(lo, hi, G)
-        acc = q.astype(np.int64) @ L["Wq"].astype(np.int64)
-        q = oracle.epilogue_i8(acc.astype(np.int32), L["x_scale"], L["w_scale"], L["bias"], L["y_scale"])
-    return layers, X0, [L["Wq"].shape[0] // G for L in layers], q
-
-
 def test_stack_fitness_reduces_to_the_8bit_chain_and_to_zero_when_lossless():
-    layers, X, groups, y8 = _tiny_stack()
+    layers, X, groups, y8 = helpers.tiny_stack()
     none = [0] * sum(groups)
     assert np.array_equal(ev.stack_forward(layers, X, none, groups), y8)        # no low group: the plain int8 chain
     allset = [1] * sum(groups)
@@ -161,7 +137,7 @@ def test_stack_fitness_reduces_to_the_8bit_chain_and_to_zero_when_lossless():
     half = ev.greedy_seed(groups, [1] * sum(groups), [g // 2 for g in groups])
     assert 0 < ev.sq_distance(ev.stack_forward(layers, X, half, groups), y8)
     # values that fit four bits on both sides (positions 0): every selection is lossless
-    layers, X, groups, y8 = _tiny_stack(small=True)
+    layers, X, groups, y8 = helpers.tiny_stack(small=True)
     q0 = __import__("oracle").quantize(X, layers[0]["x_scale"])
     assert np.abs(q0).max() <= 7
     first = [1] * groups[0] + [0] * (sum(groups) - groups[0])

@@ -1,0 +1,84 @@
+"""Evolutionary selection on the GPU (Sec. 4.2, Algorithm 1): the distance kernel against numpy
+integers, the chain fitness against the oracle's, and a whole search, generation by generation."""
+import numpy as np
+import pytest
+import torch
+
+import helpers
+from oracle import evolution as ev
+from paper_2510_02822_b200 import binding as fx
+from paper_2510_02822_b200 import evolution as gpu_ev
+from paper_2510_02822_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def dev():
+    return torch.device("cuda:0")
+
+
+@pytest.mark.parametrize("n", [0, 1, 15, 16, 17, 4101, 1000003, 40 * 1024 * 1024 + 7])
+def test_sq_distance_is_exact(dev, n):
+    a = (inputs.uniform(60, 0, n) * 256).astype(np.int64) - 128
+    b = (inputs.uniform(60, 1, n) * 256).astype(np.int64) - 128
+    if n > 2:
+        a[0], b[0] = -128, 127      # the largest difference
+        a[n - 1], b[n - 1] = 127, -128
+    A = torch.from_numpy(a.astype(np.int8)).to(dev)
+    B = torch.from_numpy(b.astype(np.int8)).to(dev)
+    out = torch.full((1,), -5, dtype=torch.int64, device=dev)
+    fx.flexiq_sq_distance_i8(A, B, out)
+    assert int(out.item()) == int(((a - b) ** 2).sum())
+
+
+def test_chain_fitness_matches_oracle(dev):
+    layers, X, groups, y8 = helpers.tiny_stack(M=200, dims=(128, 192, 96))
+    fit = gpu_ev.ChainFitness(layers, X, dev)
+    assert fit.groups == groups
+    assert np.array_equal(fit.Y8.cpu().numpy(), y8)
+    pop = ev.init_population(groups, [int(v * 500) for v in inputs.uniform(61, 0, sum(groups))], [g // 2 for g in groups], 6, seed=3)
+    pop.append([1] * sum(groups))
+    want = [ev.sq_distance(ev.stack_forward(layers, X, c, groups), y8) for c in pop]
+    assert fit.distances(pop) == want
+    assert min(want) > 0
+    fit.close()
+    fx.flexiq_check_status()
+
+
+def test_search_matches_oracle_generation_by_generation(dev):
+    layers, X, groups, y8 = helpers.tiny_stack(seed=70, M=96, dims=(96, 128, 64))
+    score = [int(v * 3000) for v in inputs.uniform(62, 0, sum(groups))]
+    tgt = [max(1, g // 2) for g in groups]
+    N, k, r, bp, gens, seed = 8, 2, 4, 1500, 5, 17
+
+    def fitness(flags):
+        return ev.sq_distance(ev.stack_forward(layers, X, flags, groups), y8)
+
+    want_flags, want_dist, want_hist = ev.run(fitness, groups, score, tgt, N, k, r, bp, gens, seed)
+    fit = gpu_ev.ChainFitness(layers, X, dev)
+    flags, dist, hist, _ = gpu_ev.search(fit, score, tgt, N, k, r, bp, gens, seed)
+    assert hist == want_hist
+    assert dist == want_dist and flags.tolist() == want_flags
+    assert all(b <= a for a, b in zip(hist, hist[1:]))
+    fit.close()
+    fx.flexiq_check_status()
+
+
+def test_nested_search_keeps_smaller_selections(dev):
+    layers, X, groups, y8 = helpers.tiny_stack(seed=80, M=64, dims=(128, 128, 128))
+    score = [int(v * 3000) for v in inputs.uniform(63, 0, sum(groups))]
+    fit = gpu_ev.ChainFitness(layers, X, dev)
+    results, perms = gpu_ev.nested_search(fit, score, [0.25, 0.5, 0.75], 6, 2, 3, 1000, 3, seed=5)
+    off = np.concatenate([[0], np.cumsum(groups)])
+    for a, b in zip(results, results[1:]):
+        assert np.all(b["flags"] >= a["flags"])
+    for res in results:
+        assert int(res["flags"].sum()) == sum(int(np.ceil(res["ratio"] * g - 1e-4)) for g in groups)
+    # the stored order serves every ratio: the groups selected at a ratio are a prefix of the layer's order
+    for l, perm in enumerate(perms):
+        assert sorted(perm.tolist()) == list(range(groups[l]))
+        for res in results:
+            sel = set(np.flatnonzero(res["flags"][off[l]:off[l + 1]]).tolist())
+            assert set(perm[:len(sel)].tolist()) == sel
+    fit.close()
