@@ -94,6 +94,15 @@ int flexiq_layer_create_conv(flexiq_layer_t *out, int Cin, int Cout, int R, int 
 
 int flexiq_layer_destroy(flexiq_layer_t layer);
 
+/* Re-runs the layout post-processing of an existing handle for another group order (and static
+ * activation positions): what flexiq_layer_create_* does with group_perm_host / x_shift_host,
+ * without allocating or synchronising -- the inner loop of the selection search (Sec. 4.2), which
+ * tries many selections on the same weights.  Wq_dev is the original-order weight tensor again
+ * (the handle keeps only slab-order copies).  Stream-ordered after earlier calls on `stream`; the
+ * ratio in force is kept.  Slabs written for the previous order no longer fit the handle. */
+int flexiq_layer_set_group_perm(flexiq_layer_t layer, const int8_t *Wq_dev, const int32_t *group_perm_host,
+                                const uint8_t *x_shift_host, void *stream);
+
 /* Chooses FLEXIQ_LOWBIT_MASKED_I8 (default) or FLEXIQ_LOWBIT_PACKED_U4 for the layer.
  * Must be the same for a flexiq_quantize_lower call and the mixed_* call that consumes
  * its slabs. */

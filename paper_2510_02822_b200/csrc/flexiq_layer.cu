@@ -158,6 +158,19 @@ __global__ void prep_weights_kernel(const int8_t *__restrict__ Wq, int is_conv, 
         }
 }
 
+static int validate_perm(const int32_t *perm, int n_g)
+{
+    char *seen = (char *)calloc((size_t)n_g, 1);
+    bool ok = true;
+    for (int j = 0; j < n_g && ok; ++j) {
+        if (perm[j] < 0 || perm[j] >= n_g || seen[perm[j]]) ok = false;
+        else seen[perm[j]] = 1;
+    }
+    free(seen);
+    if (!ok) return set_error(FLEXIQ_ERR_INVALID_ARG, "group_perm_host is not a permutation of 0..%d", n_g - 1);
+    return FLEXIQ_OK;
+}
+
 static int validate_common(flexiq_layer_t *out, int C, int N, int G, const int8_t *Wq, const float *w_scale,
                            const int32_t *perm)
 {
@@ -169,16 +182,7 @@ static int validate_common(flexiq_layer_t *out, int C, int N, int G, const int8_
     if (C % G != 0) return set_error(FLEXIQ_ERR_INVALID_ARG, "input channels %d not a multiple of group_size %d", C, G);
     if (N % 16 != 0) return set_error(FLEXIQ_ERR_INVALID_ARG, "output channels %d not a multiple of 16", N);
     if (!Wq || !w_scale || !perm) return set_error(FLEXIQ_ERR_INVALID_ARG, "Wq_dev, w_scale_dev and group_perm_host must not be NULL");
-    const int n_g = C / G;
-    char *seen = (char *)calloc((size_t)n_g, 1);
-    bool ok = true;
-    for (int j = 0; j < n_g && ok; ++j) {
-        if (perm[j] < 0 || perm[j] >= n_g || seen[perm[j]]) ok = false;
-        else seen[perm[j]] = 1;
-    }
-    free(seen);
-    if (!ok) return set_error(FLEXIQ_ERR_INVALID_ARG, "group_perm_host is not a permutation of 0..%d", n_g - 1);
-    return FLEXIQ_OK;
+    return validate_perm(perm, C / G);
 }
 
 static void free_layer(Layer *L)
@@ -207,6 +211,44 @@ int encode_weight_maps(Layer *L)
     return FLEXIQ_OK;
 }
 
+// The layout post-processing of a handle for a group order (Sec. 5): uploads the order, the
+// activation positions in slab order and the chunk tables, and rebuilds the slab-order weights, their
+// positions and the 4-bit cache from the original-order weights.  Stream-ordered, allocates nothing
+// on the device; the host arrays are staged by the copies before they return.
+static int layout_layer(Layer *L, const int8_t *Wq, const int32_t *perm, const uint8_t *x_shift, cudaStream_t stream)
+{
+    const int n_g = L->n_g, C = L->C, G = L->G, N = L->N;
+    memcpy(L->perm_host, perm, sizeof(int32_t) * n_g);
+    for (int j = 0; j < n_g; ++j) L->sx_host[j] = x_shift ? x_shift[perm[j]] : 0;  // slab order
+    FLEXIQ_CUDA_TRY(cudaMemcpyAsync(L->perm, L->perm_host, sizeof(int32_t) * n_g, cudaMemcpyHostToDevice, stream));
+    FLEXIQ_CUDA_TRY(cudaMemcpyAsync(L->sx, L->sx_host, n_g, cudaMemcpyHostToDevice, stream));
+    // chunk table: original chunk c lies in original group c*16/G, which is slab group j with perm[j] = that group
+    const int n_c = C / 16, cpg = G / 16;
+    int32_t *ent = (int32_t *)malloc(sizeof(int32_t) * (2 * n_c + n_g));
+    if (!ent) return set_error(FLEXIQ_ERR_CUDA, "out of host memory");
+    for (int j = 0; j < n_g; ++j) {
+        for (int i = 0; i < cpg; ++i) {
+            ent[perm[j] * cpg + i] = (j * cpg + i) | ((int32_t)L->sx_host[j] << 24);
+            ent[n_c + j * cpg + i] = (j * cpg + i) | ((int32_t)L->sx_host[j] << 24);
+        }
+        ent[2 * n_c + perm[j]] = j;
+    }
+    cudaError_t e1 = cudaMemcpyAsync(L->chunk_ent, ent, sizeof(int32_t) * n_c, cudaMemcpyHostToDevice, stream);
+    if (e1 == cudaSuccess) e1 = cudaMemcpyAsync(L->chunk_ent_slab, ent + n_c, sizeof(int32_t) * n_c, cudaMemcpyHostToDevice, stream);
+    if (e1 == cudaSuccess) e1 = cudaMemcpyAsync(L->inv_perm, ent + 2 * n_c, sizeof(int32_t) * n_g, cudaMemcpyHostToDevice, stream);
+    free(ent);  // pageable source: staged before the call returned
+    FLEXIQ_CUDA_TRY(e1);
+    const size_t wbytes = (size_t)N * L->Kw;
+    const long long total = (long long)n_g * N;
+    const int threads = 128;
+    prep_weights_kernel<<<(unsigned)((total + threads - 1) / threads), threads, 0, stream>>>(
+        Wq, L->is_conv, C, N, G, L->R * L->S, L->perm, L->w8, L->w8m, L->w4, L->w4_pitch, L->sw);
+    FLEXIQ_CUDA_TRY(cudaGetLastError());
+    FLEXIQ_CUDA_TRY(cudaMemcpyAsync(L->wf, L->w8, wbytes, cudaMemcpyDeviceToDevice, stream));  // all groups at 8 bits;
+    L->wf_K_lo = 0;                                                                             // the next mixed call brings the low groups along
+    return FLEXIQ_OK;
+}
+
 static int create_common(flexiq_layer_t *out, int is_conv, int C, int N, int R, int S, int stride, int pad,
                          int G, const int8_t *Wq, const float *w_scale, const float *bias,
                          const int32_t *perm, const uint8_t *x_shift, void *stream_)
@@ -232,9 +274,6 @@ static int create_common(flexiq_layer_t *out, int is_conv, int C, int N, int R, 
     cudaGetDevice(&L->device);
     L->perm_host = (int32_t *)malloc(sizeof(int32_t) * n_g);
     L->sx_host = (uint8_t *)malloc(n_g);
-    memcpy(L->perm_host, perm, sizeof(int32_t) * n_g);
-    for (int j = 0; j < n_g; ++j) L->sx_host[j] = x_shift ? x_shift[perm[j]] : 0;  // slab order
-
     const size_t wbytes = (size_t)N * L->Kw;
 #define TRY_OR_FREE(expr)                                                                        \
     do {                                                                                         \
@@ -257,36 +296,17 @@ static int create_common(flexiq_layer_t *out, int is_conv, int C, int N, int R, 
     TRY_OR_FREE(cudaMalloc(&L->alpha, sizeof(float) * N));
     TRY_OR_FREE(cudaMalloc(&L->beta, sizeof(float) * N));
     L->cache_mode = -1;
-    TRY_OR_FREE(cudaMemcpyAsync(L->perm, L->perm_host, sizeof(int32_t) * n_g, cudaMemcpyHostToDevice, stream));
-    TRY_OR_FREE(cudaMemcpyAsync(L->sx, L->sx_host, n_g, cudaMemcpyHostToDevice, stream));
     {
-        // chunk table: original chunk c lies in original group c*16/G, which is slab group j with perm[j] = that group
-        const int n_c = C / 16, cpg = G / 16;
-        int32_t *ent = (int32_t *)malloc(sizeof(int32_t) * n_c * 2);
-        for (int j = 0; j < n_g; ++j)
-            for (int i = 0; i < cpg; ++i) {
-                ent[perm[j] * cpg + i] = (j * cpg + i) | ((int32_t)L->sx_host[j] << 24);
-                ent[n_c + j * cpg + i] = (j * cpg + i) | ((int32_t)L->sx_host[j] << 24);
-            }
+        const int n_c = C / 16;
         cudaError_t e1 = cudaMalloc(&L->chunk_ent, sizeof(int32_t) * n_c);
         if (e1 == cudaSuccess) e1 = cudaMalloc(&L->chunk_ent_slab, sizeof(int32_t) * n_c);
-        if (e1 == cudaSuccess) e1 = cudaMemcpy(L->chunk_ent, ent, sizeof(int32_t) * n_c, cudaMemcpyHostToDevice);
-        if (e1 == cudaSuccess) e1 = cudaMemcpy(L->chunk_ent_slab, ent + n_c, sizeof(int32_t) * n_c, cudaMemcpyHostToDevice);
         if (e1 == cudaSuccess) e1 = cudaMalloc(&L->inv_perm, sizeof(int32_t) * n_g);
-        for (int j = 0; j < n_g; ++j) ent[perm[j]] = j;
-        if (e1 == cudaSuccess) e1 = cudaMemcpy(L->inv_perm, ent, sizeof(int32_t) * n_g, cudaMemcpyHostToDevice);
-        free(ent);
         TRY_OR_FREE(e1);
     }
     TRY_OR_FREE(cudaMemcpyAsync(L->w_scale, w_scale, sizeof(float) * N, cudaMemcpyDeviceToDevice, stream));
     if (bias) TRY_OR_FREE(cudaMemcpyAsync(L->bias, bias, sizeof(float) * N, cudaMemcpyDeviceToDevice, stream));
-    const long long total = (long long)n_g * N;
-    const int threads = 128;
-    prep_weights_kernel<<<(unsigned)((total + threads - 1) / threads), threads, 0, stream>>>(
-        Wq, is_conv, C, N, G, R * S, L->perm, L->w8, L->w8m, L->w4, L->w4_pitch, L->sw);
-    TRY_OR_FREE(cudaGetLastError());
-    TRY_OR_FREE(cudaMemcpyAsync(L->wf, L->w8, wbytes, cudaMemcpyDeviceToDevice, stream));  // ratio 0: all groups at 8 bits
-    L->wf_K_lo = 0;
+    rc = layout_layer(L, Wq, perm, x_shift, stream);
+    if (rc) { free_layer(L); return rc; }
     TRY_OR_FREE(cudaStreamSynchronize(stream));
 #undef TRY_OR_FREE
     rc = encode_weight_maps(L);
@@ -318,6 +338,22 @@ int flexiq_layer_create_conv(flexiq_layer_t *out, int Cin, int Cout, int R, int 
 {
     return create_common(out, 1, Cin, Cout, R, S, stride, pad, group_size, Wq_dev, w_scale_dev, bias_dev,
                          group_perm_host, x_shift_host, stream);
+}
+
+int flexiq_layer_set_group_perm(flexiq_layer_t layer, const int8_t *Wq_dev, const int32_t *group_perm_host,
+                                const uint8_t *x_shift_host, void *stream)
+{
+    Layer *L = as_layer(layer);
+    if (!L) return set_error(FLEXIQ_ERR_INVALID_ARG, "not a live flexiq layer handle");
+    if (!Wq_dev || !group_perm_host) return set_error(FLEXIQ_ERR_INVALID_ARG, "Wq_dev and group_perm_host must not be NULL");
+    int rc = validate_perm(group_perm_host, L->n_g);
+    if (rc) return rc;
+    if (x_shift_host)
+        for (int g = 0; g < L->n_g; ++g)
+            if (x_shift_host[g] > 4) return set_error(FLEXIQ_ERR_INVALID_ARG, "x_shift_host[%d] = %d exceeds 4", g, x_shift_host[g]);
+    rc = check_device_sm100();
+    if (rc) return rc;
+    return layout_layer(L, Wq_dev, group_perm_host, x_shift_host, reinterpret_cast<cudaStream_t>(stream));
 }
 
 int flexiq_layer_destroy(flexiq_layer_t layer)

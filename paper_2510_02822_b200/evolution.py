@@ -5,8 +5,8 @@ the fitness of a chromosome is measured with the hot path itself: every layer of
 quantized linears is created with the chromosome's selected groups first in its group order and
 K_lo = their number, the chain runs (prologue + mixed GEMM per layer, int8 between layers) and
 flexiq_sq_distance_i8 gives the exact squared distance of the last layer's outputs from those of
-the 8-bit chain.  Layer handles are cached per (layer, selection): crossover moves whole layers
-between chromosomes, so most selections of a generation have been seen before.
+the 8-bit chain.  One handle per layer serves every chromosome: flexiq_layer_set_group_perm lays it
+out again for the next selection without allocating or synchronising.
 
     python -m paper_2510_02822_b200.evolution [--model deits|vitb] [--blocks 2] [--batch 4]
                                               [--population 16] [--generations 10] [--ratios 0.25 0.5 0.75]
@@ -42,7 +42,7 @@ class ChainFitness:
     layers[l] = dict(Wq [K, N] int8, w_scale, bias, x_scale, y_scale, G, sx_group [K/G]); layer l + 1
     takes layer l's int8 output as its quantized input (x_scale of l + 1 = y_scale of l)."""
 
-    def __init__(self, layers, X, dev, cache_limit=4096):
+    def __init__(self, layers, X, dev):
         self.dev = dev
         self.layers = layers
         self.M = X.shape[0]
@@ -53,26 +53,27 @@ class ChainFitness:
                            for L in layers]
         self.slab = [torch.empty(self.M * L["Wq"].shape[0] + 16, dtype=torch.uint8, device=dev) for L in layers]
         self.Y = [torch.empty((self.M, L["Wq"].shape[1]), dtype=torch.int8, device=dev) for L in layers]
-        self.cache = {}
-        self.cache_limit = cache_limit
+        self.handles = [None] * len(layers)
+        self.current = [None] * len(layers)
         self.created = 0
         self.evaluated = 0
         self.Y8 = self.outputs(np.zeros(int(self.off[-1]), dtype=np.uint8)).clone()
 
     def _layer(self, l, flags_layer):
-        key = (l, bytes(np.asarray(flags_layer, dtype=np.uint8)))
-        h = self.cache.get(key)
-        if h is None:
-            if len(self.cache) >= self.cache_limit:
-                for old in self.cache.values():
-                    old.close()
-                self.cache.clear()
+        """The handle of layer l laid out for this selection: one handle per layer, re-laid out in place
+        (flexiq_layer_set_group_perm: no allocation, no synchronisation) when the selection changes."""
+        key = bytes(np.asarray(flags_layer, dtype=np.uint8))
+        h = self.handles[l]
+        if key != self.current[l]:
             perm, n_low = selection_perm(flags_layer)
             Wq, ws, b = self.dev_params[l]
-            h = fx.Layer(Wq, ws, b, perm, np.asarray(self.layers[l]["sx_group"], dtype=np.uint8), self.layers[l]["G"])
+            xs = np.asarray(self.layers[l]["sx_group"], dtype=np.uint8)
+            if h is None:
+                h = self.handles[l] = fx.Layer(Wq, ws, b, perm, xs, self.layers[l]["G"])
+            else:
+                h.set_group_perm(Wq, perm, xs)
             h.set_lowbit_ratio(n_low / self.groups[l])
-            assert h.K_lo == n_low * self.layers[l]["G"]
-            self.cache[key] = h
+            self.current[l] = key
             self.created += 1
         return h
 
@@ -95,9 +96,11 @@ class ChainFitness:
         return [int(v) for v in out.cpu().tolist()]
 
     def close(self):
-        for h in self.cache.values():
-            h.close()
-        self.cache.clear()
+        for h in self.handles:
+            if h is not None:
+                h.close()
+        self.handles = [None] * len(self.layers)
+        self.current = [None] * len(self.layers)
 
 
 def search(fit: ChainFitness, score, per_layer_target, N, k, r, rate_bp, generations, seed, locked=None):
@@ -216,7 +219,7 @@ def main():
                           "history": res["history"], "per_layer_ratio": [round(v, 3) for v in per_layer],
                           "s_per_generation": round(float(np.mean(res["seconds"])), 4)}), flush=True)
     print(json.dumps({"step": "done", "wall_s": round(time.time() - t0, 2), "chromosomes_evaluated": fit.evaluated,
-                      "layer_handles_created": fit.created}), flush=True)
+                      "layer_layouts": fit.created}), flush=True)
     # the stored group order serves every ratio: check the nesting on the first layer
     for t in range(1, len(results)):
         assert np.all(results[t]["flags"] >= results[t - 1]["flags"])

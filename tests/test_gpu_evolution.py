@@ -82,3 +82,34 @@ def test_nested_search_keeps_smaller_selections(dev):
             sel = set(np.flatnonzero(res["flags"][off[l]:off[l + 1]]).tolist())
             assert set(perm[:len(sel)].tolist()) == sel
     fit.close()
+
+
+def test_relayout_in_place_matches_a_fresh_layer(dev):
+    """flexiq_layer_set_group_perm: the handle laid out again for another order and other static
+    positions computes what the oracle computes for that order, at the ratio that was in force."""
+    import oracle
+    case = inputs.ranged_linear("relay", 260, 256, 176, 16, seed=91, group_structured=True)
+    perm_a, sxg, _, _ = helpers.prepare_linear(case)
+    L = fx.Layer(torch.from_numpy(case.Wq).to(dev), torch.from_numpy(case.w_scale).to(dev), torch.from_numpy(case.bias).to(dev), perm_a, sxg, case.G)
+    L.set_lowbit_ratio(0.5)
+    X = torch.from_numpy(case.X).to(dev)
+    Wq = torch.from_numpy(case.Wq).to(dev)
+    x4, x8 = L.alloc_slabs(case.M)
+    Y = torch.empty((case.M, case.N), dtype=torch.int8, device=dev)
+    q = oracle.quantize(case.X, case.x_scale)
+    n_g = case.K // case.G
+    orders = [perm_a, np.arange(n_g, dtype=np.int32)[::-1].copy(), np.roll(np.arange(n_g, dtype=np.int32), 5)]
+    shifts = [sxg, np.minimum(sxg + 1, 4).astype(np.uint8), sxg]
+    for ratio in (0.5, 0.25, 1.0):
+        L.set_lowbit_ratio(ratio)
+        for perm, xs in zip(orders, shifts):
+            L.set_group_perm(Wq, perm, xs)
+            fx.flexiq_quantize_lower(L.h, X, fx.DTYPE_F32, case.M, case.x_scale, 0, x4, x8)
+            fx.flexiq_mixed_gemm(L.h, x4, x8, None, case.M, case.x_scale, case.y_scale, fx.OUT_REQUANT_I8, Y)
+            sw = oracle.weight_positions_linear(case.Wq, case.G, perm)
+            acc = oracle.mixed_gemm_acc(q, case.Wq, case.G, perm, xs[perm].copy(), sw, oracle.n_low(ratio, n_g))
+            assert np.array_equal(Y.cpu().numpy(), oracle.epilogue_i8(acc, case.x_scale, case.w_scale, case.bias, case.y_scale))
+    with pytest.raises(fx.FlexiqError):
+        L.set_group_perm(Wq, np.zeros(n_g, dtype=np.int32))
+    fx.flexiq_check_status()
+    L.close()
