@@ -2,6 +2,7 @@
 
     python -m paper_2510_02822_b200.profile_case --layer vitb_qkv --ratio 0.5 --iters 3
     python -m paper_2510_02822_b200.profile_case --layer vitb_fc2 --aux reorder       # residual reorder of the layer's input
+    python -m paper_2510_02822_b200.profile_case --layer vitb_fc2 --aux distance      # squared-distance reduction (selection fitness)
 
 Prints the average device time of the prologue and of the mixed GEMM (CUDA events on the
 launching stream).  Layers: vitb_{qkv,proj,fc1,fc2}, vitl_{...}, deits_{...} (append
@@ -46,7 +47,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=1)
     ap.add_argument("--path", default="masked", choices=["masked", "packed"])
     ap.add_argument("--out", default="i8", choices=["i8", "f32", "i32"])
-    ap.add_argument("--aux", default="", choices=["", "reorder", "calib"], help="run an auxiliary kernel on the layer's input instead: the residual reorder operator or the calibration range kernels")
+    ap.add_argument("--aux", default="", choices=["", "reorder", "calib", "distance"], help="run an auxiliary kernel on the layer's input instead: the residual reorder operator, the calibration range kernels, or the squared-distance reduction (on the int8 view of the input and a shifted copy)")
     args = ap.parse_args()
     dev = torch.device("cuda:0")
     c, is_conv = make_case(args.layer)
@@ -65,9 +66,15 @@ def main():
         lo = torch.empty(L.K, dtype=torch.int32, device=dev)
         hi = torch.empty(L.K, dtype=torch.int32, device=dev)
         Yr = torch.empty_like(Xq)
+        if args.aux == "distance":
+            A8 = Xq.view(torch.int8).reshape(-1)
+            B8 = torch.roll(A8, 16)
+            d_out = torch.zeros(1, dtype=torch.int64, device=dev)
 
         def aux():
-            if args.aux == "reorder":
+            if args.aux == "distance":
+                fx.flexiq_sq_distance_i8(A8, B8, d_out)
+            elif args.aux == "reorder":
                 L.reorder_channels(Xq, fx.REORDER_TO_SLAB, Y=Yr)
             else:
                 fx.flexiq_calib_channel_ranges(Xq, fx._dtype_code(Xq), Xq.shape[0], L.K, c.x_scale, False, lo, hi)
@@ -82,7 +89,7 @@ def main():
         e1.record(stream)
         torch.cuda.synchronize()
         t = e0.elapsed_time(e1) / args.iters
-        moved = Xq.numel() * Xq.element_size() * (2 if args.aux == "reorder" else 1)
+        moved = Xq.numel() * Xq.element_size() * (1 if args.aux == "calib" else 2)
         print(f"{args.layer} {args.aux}: {t * 1e3:.1f} us, {moved / t / 1e6:.0f} GB/s")
         L.close()
         return
