@@ -296,6 +296,31 @@ def test_vit_b_full_size_sampled_rows(dev, layer):
     L.close()
 
 
+def test_vit_l_full_size_sampled_rows(dev):
+    """The largest configuration (ViT-L/16, batch 128: M = 25216) at full size: fc2, K = 4096."""
+    name, K, N = inputs.VIT_L_LAYERS[3]
+    case = inputs.vit_linear(f"cfg5_{name}", 128 * 197, K, N, 16, seed=5003)
+    perm, sxg, sxs, sw = helpers.prepare_linear(case)
+    L = _layer(case, dev, perm, sxg)
+    X = torch.from_numpy(case.X).to(dev)
+    rows = np.unique(np.concatenate([np.arange(0, case.M, 197), np.arange(case.M - 40, case.M), np.arange(250, 262)])).astype(np.int64)
+    q_rows = oracle.quantize(case.X[rows], case.x_scale)
+    for r in (0.25, 1.0):
+        L.set_lowbit_ratio(r)
+        nl = oracle.n_low(r, K // 16)
+        x4, x8, _ = L.quantize_lower(X, case.x_scale)
+        acc_e = oracle.mixed_gemm_acc(q_rows, case.Wq, 16, perm, sxs, sw, nl)
+        y8 = L.mixed_gemm(x4, x8, case.M, case.x_scale, case.y_scale, fx.OUT_REQUANT_I8)
+        yf = L.mixed_gemm(x4, x8, case.M, case.x_scale, case.y_scale, fx.OUT_DEQUANT_F32)
+        torch.cuda.synchronize()
+        fx.flexiq_check_status()
+        assert np.array_equal(y8.cpu().numpy()[rows], oracle.epilogue_i8(acc_e, case.x_scale, case.w_scale, case.bias, case.y_scale))
+        want = oracle.epilogue_f32(acc_e, case.x_scale, case.w_scale, case.bias)
+        got = yf.cpu().numpy()[rows]
+        assert np.all(np.abs(got - want) <= 1e-6 * np.maximum(1.0, np.abs(want)))
+    L.close()
+
+
 @pytest.mark.parametrize("K", [240, 256, 1024])
 def test_extreme_accumulators(dev, K):
     """The largest accumulator magnitudes a layer can produce (all operands at -128 / 127) survive the
