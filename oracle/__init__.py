@@ -237,6 +237,19 @@ def epilogue_f32(acc, x_scale, w_scale, bias) -> np.ndarray:
     return out.reshape(acc.shape)
 
 
+def epilogue_f16(acc, x_scale, w_scale, bias) -> np.ndarray:
+    """16-bit floating-point output (the operators between the quantized layers run in fp16): the fp32
+    epilogue value rounded once more to fp16, to nearest even (numpy's float32 -> float16 conversion)."""
+    return epilogue_f32(acc, x_scale, w_scale, bias).astype(np.float16)
+
+
+def epilogue_bf16_bits(acc, x_scale, w_scale, bias) -> np.ndarray:
+    """The same for bfloat16, returned as the 16-bit patterns (numpy has no bfloat16): the upper half of
+    the fp32 pattern after adding half an ulp of the kept part, ties to the even pattern (finite values)."""
+    u = epilogue_f32(acc, x_scale, w_scale, bias).view(np.uint32).astype(np.uint64)
+    return ((u + 0x7FFF + ((u >> 16) & 1)) >> 16).astype(np.uint16)
+
+
 def reorder_channels(x, G: int, perm, to_slab: bool = True) -> np.ndarray:
     x = np.ascontiguousarray(x)
     K = x.shape[-1]

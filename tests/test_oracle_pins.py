@@ -443,3 +443,35 @@ def test_weight_positions_never_saturate():
             if sw[j, n] > 0:
                 t = blk[:, n] >> (int(sw[j, n]) - 1)
                 assert t.min() < -8 or t.max() > 7
+
+
+def test_epilogue_half_precision_roundings():
+    """fp16 / bf16 outputs = the fp32 value rounded to nearest even: hand-picked ties, and a library
+    conversion (torch on the CPU) as an independent reference for both formats."""
+    import torch
+    ws = np.ones(16, np.float32)
+    # acc * 2^-12: 4097 -> 1 + 2^-12 (rounds down to 1 in fp16: spacing 2^-10), 4098 -> 1 + 2^-11 is the tie -> even (1.0),
+    # 4102 -> 1 + 3 * 2^-11 is the tie above 1 + 2^-10 -> even (1 + 2^-9)
+    acc = np.array([[4096, 4097, 4098, 4099, 4102, -4098, 4128, 4160, 0, 1, -1, 70000, 123456, -99999, 33, 65]], np.int32)
+    s = float(2.0 ** -12)
+    f32 = oracle.epilogue_f32(acc, s, ws, None)
+    f16 = oracle.epilogue_f16(acc, s, ws, None)
+    assert f16.dtype == np.float16
+    assert f16[0, :6].tolist() == [1.0, 1.0, 1.0, 1.0 + 2.0 ** -10, 1.0 + 2.0 ** -9, -1.0]
+    assert np.array_equal(f16, torch.from_numpy(f32).to(torch.float16).numpy())
+    # bf16 keeps 8 significant bits: spacing 2^-7 at 1.0; 1 + 2^-8 (acc 4112) is a tie -> 1.0; 1 + 3 * 2^-8 (4144) -> 1 + 2^-6
+    acc_b = np.array([[4096, 4112, 4113, 4144, 4128, -4112, 12345678, -7654321, 0, 5, 4111, 4145, 1 << 30, -(1 << 30), 77, 99]], np.int32)
+    f32b = oracle.epilogue_f32(acc_b, s, ws, None)
+    bits = oracle.epilogue_bf16_bits(acc_b, s, ws, None)
+    as_f32 = (bits.astype(np.uint32) << 16).view(np.float32)
+    assert as_f32[0, :6].tolist() == [1.0, 1.0, 1.0 + 2.0 ** -7, 1.0 + 2.0 ** -6, 1.0 + 2.0 ** -7, -1.0]
+    want = torch.from_numpy(f32b).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    assert np.array_equal(bits, want)
+    rng = np.random.default_rng(0)
+    acc_r = rng.integers(-2 ** 24, 2 ** 24, (64, 16)).astype(np.int32)
+    wsr = rng.uniform(0.5, 2.0, 16).astype(np.float32)
+    br = rng.normal(0, 1, 16).astype(np.float32)
+    f = oracle.epilogue_f32(acc_r, 3.1e-4, wsr, br)
+    assert np.array_equal(oracle.epilogue_f16(acc_r, 3.1e-4, wsr, br), torch.from_numpy(f).to(torch.float16).numpy())
+    assert np.array_equal(oracle.epilogue_bf16_bits(acc_r, 3.1e-4, wsr, br),
+                          torch.from_numpy(f).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16))
