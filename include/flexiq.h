@@ -50,6 +50,11 @@ extern "C" {
 #define FLEXIQ_OUT_ACC_I32 0    /* raw int32 accumulators                       */
 #define FLEXIQ_OUT_REQUANT_I8 1 /* int8, re-quantized with y_scale (Eq. 1)      */
 #define FLEXIQ_OUT_DEQUANT_F32 2 /* fp32, de-quantized                          */
+/* 16-bit floating-point outputs (the evaluation runs the operators between the quantized layers,
+ * normalisation and GELU, in 16-bit floating point): the DEQUANT_F32 value rounded once more, to
+ * nearest even.  (3 is not a public mode.) */
+#define FLEXIQ_OUT_DEQUANT_F16 4
+#define FLEXIQ_OUT_DEQUANT_BF16 5
 
 /* How the low-bit slice travels from the prologue to the mainloop (layer property).
  * PACKED : two 4-bit values per byte (half the bytes); the mainloop widens them to the
@@ -187,6 +192,7 @@ int flexiq_quantize_lower_dynamic_noalloc(flexiq_layer_t layer, const void *X_de
  *   REQUANT_I8 : clip(round_half_even(fma(float(acc), (x_scale*w_scale[n])/y_scale,
  *                                        bias[n]/y_scale)), -128, 127)
  *   DEQUANT_F32: fma(float(acc), x_scale*w_scale[n], bias[n])
+ *   DEQUANT_F16 / DEQUANT_BF16: that fp32 value converted to fp16 / bf16, round to nearest even
  *   X4_dev/X8_dev  slabs written by flexiq_quantize_lower at the layer's current ratio
  *   x_shift_dev    [K/G] uint8 slab-order activation positions (dynamic mode) or NULL for
  *                  the layer's static ones.  Only the PACKED path reads it; on the MASKED

@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_DIR, "libflexiq.so")
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4
 DTYPE_F32, DTYPE_F16, DTYPE_BF16, DTYPE_I8 = 0, 1, 2, 3
 OUT_ACC_I32, OUT_REQUANT_I8, OUT_DEQUANT_F32 = 0, 1, 2
+OUT_DEQUANT_F16, OUT_DEQUANT_BF16 = 4, 5
 LOWBIT_MASKED_I8, LOWBIT_PACKED_U4 = 0, 1
 ORDER_ORIGINAL, ORDER_NEXT_SLAB = 0, 1
 REORDER_TO_SLAB, REORDER_FROM_SLAB = 0, 1
@@ -323,7 +324,8 @@ class Layer:
     def mixed_gemm(self, x4, x8, M, x_scale, y_scale, out_mode, Y=None, x_shift=None):
         import torch
         if Y is None:
-            dt = {OUT_ACC_I32: torch.int32, OUT_REQUANT_I8: torch.int8, OUT_DEQUANT_F32: torch.float32}[out_mode]
+            dt = {OUT_ACC_I32: torch.int32, OUT_REQUANT_I8: torch.int8, OUT_DEQUANT_F32: torch.float32,
+                  OUT_DEQUANT_F16: torch.float16, OUT_DEQUANT_BF16: torch.bfloat16}[out_mode]
             Y = torch.empty((M, self.N), dtype=dt, device=self.device)
         flexiq_mixed_gemm(self.h, x4, x8, x_shift, M, x_scale, y_scale, out_mode, Y)
         return Y
@@ -358,7 +360,8 @@ class Layer:
         P = (H + 2 * pad - self.R) // stride + 1
         Q = (W + 2 * pad - self.S) // stride + 1
         if Y is None:
-            dt = {OUT_ACC_I32: torch.int32, OUT_REQUANT_I8: torch.int8, OUT_DEQUANT_F32: torch.float32}[out_mode]
+            dt = {OUT_ACC_I32: torch.int32, OUT_REQUANT_I8: torch.int8, OUT_DEQUANT_F32: torch.float32,
+                  OUT_DEQUANT_F16: torch.float16, OUT_DEQUANT_BF16: torch.bfloat16}[out_mode]
             Y = torch.empty((Nb, P, Q, self.N), dtype=dt, device=self.device)
         flexiq_mixed_conv(self.h, x4, x8, x_shift, Nb, H, W, x_scale, y_scale, out_mode, Y)
         return Y

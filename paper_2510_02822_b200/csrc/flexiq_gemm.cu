@@ -9,12 +9,16 @@
 // cta_group::2) per 256-row tile:
 //   warp 0       TMA producer (tiled loads for linear layers, im2col loads for convs)
 //   warp 1       TMEM allocation + MMA issue (one elected lane)
-//   warps 2..17  epilogue, four per TMEM lane quadrant: tcgen05.ld, scale / bias / round / clip, int8
-//                tiles staged in shared memory and written by tiled bulk stores (fp32 / int32: direct
-//                256-bit stores); on the packed path eight of them widen 4-bit tiles instead
+//   warps 2..17  epilogue, four per TMEM lane quadrant: tcgen05.ld, scale / bias / round / clip, the
+//                results staged in shared memory 32 rows x 32 bytes at a time and written by tiled bulk
+//                stores (the fused boundary in original channel order scatters 16-byte chunks directly);
+//                on the packed path eight of them widen 4-bit tiles instead
 // Two TMEM accumulators let the epilogue of tile i overlap the mainloop of tile i+1.
 // Every wait is bounded; an expired wait raises the status word and the CTA drains.
 #include "flexiq_internal.h"
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include "sm100_ptx.cuh"
 
 #include <stdlib.h>
@@ -144,6 +148,17 @@ __device__ __forceinline__ unsigned requant4(float y0, float y1, float y2, float
     return pack2_sat_s8(__float2int_rn(y1), __float2int_rn(y0), top);
 }
 
+// two fp32 -> two fp16 (or bf16) values, round to nearest even, the first in the low half
+template <bool BF16> __device__ __forceinline__ uint32_t pack2_f16(float lo, float hi)
+{
+    if (BF16) {
+        const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<const uint32_t *>(&v);
+    }
+    const __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&v);
+}
+
 // 16 accumulator columns of one row -> 16 output values, through the per-channel factors.
 //   REQUANT_I8 : 16 bytes (one 128-bit word);  DEQUANT_F32 / ACC_I32 : 64 bytes.
 template <int MODE>
@@ -248,13 +263,14 @@ struct EpilogueCtx {
 // One epilogue warp: TMEM lane quadrant `quad` (32 rows, lane = row), column slot `part` (32 or 64
 // columns per pass; two passes when only eight warps drain the tile) of every tile of this CTA.
 // Per pass: fetch the columns' factors, read the whole slice of the accumulator into registers,
-// hand the accumulator back, then scale / round / clip; int8 results are staged in shared memory
-// and leave through tiled bulk stores, 4-byte results go straight to global memory row by row.
+// hand the accumulator back, then scale / round / clip; the results are staged in shared memory (32 rows
+// x 32 bytes: 32 int8, 16 half-precision or 8 four-byte columns) and leave through tiled bulk stores.
 template <int CG, int MODE>
 __device__ __forceinline__ void epilogue_role(const GemmParams &p, const EpilogueCtx &x, int quad, int part, int lane)
 {
     constexpr bool kScaled = MODE != FLEXIQ_OUT_ACC_I32;
-    constexpr int kElem = (MODE == FLEXIQ_OUT_REQUANT_I8 || MODE == kOutNextSlab) ? 1 : 4;  // output bytes per element
+    constexpr bool kHalf = MODE == FLEXIQ_OUT_DEQUANT_F16 || MODE == FLEXIQ_OUT_DEQUANT_BF16;
+    constexpr int kElem = (MODE == FLEXIQ_OUT_REQUANT_I8 || MODE == kOutNextSlab) ? 1 : (kHalf ? 2 : 4);  // output bytes per element
     const int BN = p.BN;
     // Columns per warp and pass: 64 (tiles of 192 or 256 columns) or 32 (128 or 64), so that every staged
     // box is 32 columns = whole sectors; with 192 or 64 columns the last column slot of a lane quadrant has no
@@ -372,6 +388,66 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                         }
                     }
                 }
+            } else if (kHalf && p.tma_store) {
+                // 16-bit outputs: 32 rows x 16 columns (32 bytes per row: the same 1 KB swizzled box) per store
+                const long long row0 = row - lane;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t *r = h == 0 ? ra : rb;
+#pragma unroll
+                    for (int g = 0; g < 2; ++g) {
+                        const int n = nw + 32 * h + 16 * g;
+                        if (32 * h < cols && n < p.N && row0 < p.M) {   // warp-uniform
+                            uint32_t w[16], hw[8];
+                            finish16<FLEXIQ_OUT_DEQUANT_F32>(r + 16 * g, x.fac + 32 * h + 16 * g, x.fac + 64 + 32 * h + 16 * g, w);
+#pragma unroll
+                            for (int q = 0; q < 8; ++q)
+                                hw[q] = pack2_f16<MODE == FLEXIQ_OUT_DEQUANT_BF16>(__uint_as_float(w[2 * q]), __uint_as_float(w[2 * q + 1]));
+                            if (lane == 0) ptx::bulk_wait_read_all();    // the previous store has read the buffer
+                            __syncwarp();
+                            const uint32_t dst = x.store_stage + (uint32_t)lane * 32u;
+                            const uint32_t sw16 = ((uint32_t)lane >> 2 & 1u) << 4;
+                            ptx::st_shared_128(dst + sw16, hw[0], hw[1], hw[2], hw[3]);
+                            ptx::st_shared_128(dst + (sw16 ^ 16u), hw[4], hw[5], hw[6], hw[7]);
+                            ptx::fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == 0) {
+                                ptx::tma_store_2d(x.map_y, x.store_stage, 2 * n, (int)row0);
+                                ptx::bulk_commit_group();
+                            }
+                        }
+                    }
+                }
+            } else if (kElem == 4 && p.tma_store) {
+                // 4-byte outputs: 32 rows x 8 columns per store (the same 32-byte rows)
+                const long long row0 = row - lane;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t *r = h == 0 ? ra : rb;
+#pragma unroll
+                    for (int g = 0; g < 2; ++g) {
+                        const int n = nw + 32 * h + 16 * g;
+                        if (32 * h < cols && n < p.N && row0 < p.M) {   // warp-uniform
+                            uint32_t w[16];
+                            finish16<MODE>(r + 16 * g, x.fac + 32 * h + 16 * g, x.fac + 64 + 32 * h + 16 * g, w);
+                            const uint32_t dst = x.store_stage + (uint32_t)lane * 32u;
+                            const uint32_t sw16 = ((uint32_t)lane >> 2 & 1u) << 4;
+#pragma unroll
+                            for (int b = 0; b < 2; ++b) {
+                                if (lane == 0) ptx::bulk_wait_read_all();
+                                __syncwarp();
+                                ptx::st_shared_128(dst + sw16, w[8 * b], w[8 * b + 1], w[8 * b + 2], w[8 * b + 3]);
+                                ptx::st_shared_128(dst + (sw16 ^ 16u), w[8 * b + 4], w[8 * b + 5], w[8 * b + 6], w[8 * b + 7]);
+                                ptx::fence_proxy_async_smem();
+                                __syncwarp();
+                                if (lane == 0) {
+                                    ptx::tma_store_2d(x.map_y, x.store_stage, 4 * (n + 8 * b), (int)row0);
+                                    ptx::bulk_commit_group();
+                                }
+                            }
+                        }
+                    }
+                }
             } else
             if (row < p.M) {
                 uint8_t *yrow = static_cast<uint8_t *>(p.Y) + (row * p.N + nw) * kElem;
@@ -407,6 +483,24 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                                 st_global_128(yrow + 32 * h, w[0], w[1], w[2], w[3]);
                                 if (second) st_global_128(yrow + 32 * h + 16, w[4], w[5], w[6], w[7]);
                             }
+                        } else if (kHalf) {
+                            // 16-bit floating-point outputs: the fp32 result of the fma, rounded once more (to nearest even)
+#pragma unroll
+                            for (int g = 0; g < 2; ++g) {
+                                if (g == 0 || second) {
+                                    uint32_t w[16], hw[8];
+                                    finish16<FLEXIQ_OUT_DEQUANT_F32>(r + 16 * g, x.fac + 32 * h + 16 * g, x.fac + 64 + 32 * h + 16 * g, w);
+#pragma unroll
+                                    for (int q = 0; q < 8; ++q)
+                                        hw[q] = pack2_f16<MODE == FLEXIQ_OUT_DEQUANT_BF16>(__uint_as_float(w[2 * q]), __uint_as_float(w[2 * q + 1]));
+                                    uint8_t *dst = yrow + (32 * h + 16 * g) * 2;
+                                    if (y32) st_global_256(dst, hw);    // rows of 2-byte elements with N % 16 == 0 are 32-byte aligned
+                                    else {
+                                        st_global_128(dst, hw[0], hw[1], hw[2], hw[3]);
+                                        st_global_128(dst + 16, hw[4], hw[5], hw[6], hw[7]);
+                                    }
+                                }
+                            }
                         } else {
 #pragma unroll
                             for (int g = 0; g < 2; ++g) {
@@ -431,7 +525,7 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
         }
         if ((buf ^= 1) == 0) buf_phase ^= 1;
     }
-    if ((MODE == FLEXIQ_OUT_REQUANT_I8 || MODE == kOutNextSlab) && p.tma_store && lane == 0) ptx::bulk_wait_all();  // the staged stores are performed
+    if (p.tma_store && lane == 0) ptx::bulk_wait_all();  // the staged stores are performed
     if (quad == 2 && part == 0 && lane == 0) { PROF_STORE(8, prof_wait); PROF_STORE(9, clock64() - prof_start); PROF_STORE(10, prof_ld); PROF_STORE(11, prof_math); }
 }
 
@@ -749,6 +843,8 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             if (p.out_mode == FLEXIQ_OUT_REQUANT_I8) epilogue_role<CG, FLEXIQ_OUT_REQUANT_I8>(p, x, warp & 3, e >> 2, lane);
             else if (p.out_mode == FLEXIQ_OUT_DEQUANT_F32) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_F32>(p, x, warp & 3, e >> 2, lane);
             else if (p.out_mode == kOutNextSlab) epilogue_role<CG, kOutNextSlab>(p, x, warp & 3, e >> 2, lane);
+            else if (p.out_mode == FLEXIQ_OUT_DEQUANT_F16) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_F16>(p, x, warp & 3, e >> 2, lane);
+            else if (p.out_mode == FLEXIQ_OUT_DEQUANT_BF16) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_BF16>(p, x, warp & 3, e >> 2, lane);
             else epilogue_role<CG, FLEXIQ_OUT_ACC_I32>(p, x, warp & 3, e >> 2, lane);
         } else if (PK) {
             // --------------------------------------------------------- expanders (packed path)
@@ -1033,7 +1129,8 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
         if (out_order != FLEXIQ_ORDER_ORIGINAL && out_order != FLEXIQ_ORDER_NEXT_SLAB)
             return set_error(FLEXIQ_ERR_INVALID_ARG, "unknown out_order %d", out_order);
         out_mode = kOutNextSlab;
-    } else if (out_mode < FLEXIQ_OUT_ACC_I32 || out_mode > FLEXIQ_OUT_DEQUANT_F32)
+    } else if (out_mode != FLEXIQ_OUT_ACC_I32 && out_mode != FLEXIQ_OUT_REQUANT_I8 && out_mode != FLEXIQ_OUT_DEQUANT_F32 &&
+               out_mode != FLEXIQ_OUT_DEQUANT_F16 && out_mode != FLEXIQ_OUT_DEQUANT_BF16)
         return set_error(FLEXIQ_ERR_INVALID_ARG, "unknown out_mode %d", out_mode);
     if ((out_mode == FLEXIQ_OUT_REQUANT_I8 || next) && !(y_scale > 0.0f))
         return set_error(FLEXIQ_ERR_INVALID_ARG, "y_scale %g must be positive", (double)y_scale);
@@ -1114,7 +1211,9 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     }
     // the per-output-channel factors depend on the call's scales: recomputed (one tiny launch,
     // stream-ordered before the GEMM) only when they differ from the previous call's
-    const int fmode = next ? FLEXIQ_OUT_REQUANT_I8 : out_mode;  // the fused boundary re-quantizes with the same factors
+    // the fused boundary re-quantizes with the REQUANT factors; the three floating-point outputs share theirs
+    const int fmode = next ? FLEXIQ_OUT_REQUANT_I8
+                           : ((out_mode == FLEXIQ_OUT_DEQUANT_F16 || out_mode == FLEXIQ_OUT_DEQUANT_BF16) ? FLEXIQ_OUT_DEQUANT_F32 : out_mode);
     if (fmode != FLEXIQ_OUT_ACC_I32 &&
         !(L->cache_mode == fmode && L->cache_xs == x_scale && (fmode == FLEXIQ_OUT_DEQUANT_F32 || L->cache_ys == y_scale))) {
         scale_vectors_kernel<<<(L->N + 255) / 256, 256, 0, st>>>(L->N, x_scale, y_scale, fmode == FLEXIQ_OUT_REQUANT_I8,
@@ -1126,11 +1225,14 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     // activation maps (per call: they depend on the caller's buffers, M and the ratio);
     // an empty slab borrows the other one's map and is never addressed
     CUtensorMap a_lo, a_hi;
-    const bool staged = (out_mode == FLEXIQ_OUT_REQUANT_I8 || (next && out_order == FLEXIQ_ORDER_NEXT_SLAB)) && !direct_stores_only();
+    const bool half_out = out_mode == FLEXIQ_OUT_DEQUANT_F16 || out_mode == FLEXIQ_OUT_DEQUANT_BF16;
+    const bool word_out = out_mode == FLEXIQ_OUT_DEQUANT_F32 || out_mode == FLEXIQ_OUT_ACC_I32;
+    const int y_elem = half_out ? 2 : (word_out ? 4 : 1);
+    const bool staged = (!next || out_order == FLEXIQ_ORDER_NEXT_SLAB) && !direct_stores_only();
     const void *slab = packed_path ? static_cast<const void *>(X8) : static_cast<const void *>(X4);
     Layer::CallMaps &cm = L->call_maps;
     const bool cached = !packed && cm.slab == slab && cm.M == M && cm.Nb == Nb && cm.H == H && cm.W == W && cm.bk == p.BK &&
-                        cm.im2col == (int)p.im2col && (!staged || (cm.staged && cm.Y == Y));
+                        cm.im2col == (int)p.im2col && (!staged || (cm.staged && cm.Y == Y && cm.y_elem == y_elem));
     if (cached) {
         a_lo = a_hi = cm.a;
     } else if (!packed) {
@@ -1163,13 +1265,17 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     if (staged && cached) {
         y_map = cm.y;
         y_map16 = cm.y16;
+    } else if (staged && y_elem > 1) {
+        // rows of N 2- or 4-byte values addressed in bytes: a box is 32 bytes (16 or 8 columns) x 32 rows
+        if ((rc = make_map_2d(&y_map, Y, (uint64_t)L->N * y_elem, (uint64_t)M, (uint64_t)L->N * y_elem, 32, 32, 32))) return rc;
+        y_map16 = y_map;
     } else if (staged) {
         if (L->N >= 32 && (rc = make_map_2d(&y_map, Y, (uint64_t)L->N, (uint64_t)M, (uint64_t)L->N, 32, 32, 32))) return rc;
         if ((rc = make_map_2d(&y_map16, Y, (uint64_t)L->N, (uint64_t)M, (uint64_t)L->N, 16, 32, 0))) return rc;
     }
     if (!packed && !cached) {
         cm.slab = slab; cm.Y = staged ? Y : nullptr; cm.M = M; cm.Nb = Nb; cm.H = H; cm.W = W; cm.bk = p.BK; cm.im2col = p.im2col;
-        cm.staged = staged; cm.a = a_hi; cm.y = y_map; cm.y16 = y_map16;
+        cm.staged = staged; cm.y_elem = y_elem; cm.a = a_hi; cm.y = y_map; cm.y16 = y_map16;
     }
     const int bi = weight_map_index(bn / cg);  // box rows = the B rows one CTA loads
     if (packed) return launch_kernel<1, 1>(a_lo, a_hi, L->map_w4[bi], L->map_w8[bi], y_map, y_map16, p, sms, st);

@@ -65,7 +65,7 @@ struct Layer {
     struct CallMaps {
         const void *slab, *Y;
         long long M;
-        int Nb, H, W, bk, im2col, staged;
+        int Nb, H, W, bk, im2col, staged, y_elem;
         CUtensorMap a, y, y16;
     } call_maps;
 };

@@ -46,7 +46,7 @@ def main():
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=1)
     ap.add_argument("--path", default="masked", choices=["masked", "packed"])
-    ap.add_argument("--out", default="i8", choices=["i8", "f32", "i32"])
+    ap.add_argument("--out", default="i8", choices=["i8", "f32", "i32", "f16", "bf16"])
     ap.add_argument("--aux", default="", choices=["", "reorder", "calib", "distance"], help="run an auxiliary kernel on the layer's input instead: the residual reorder operator, the calibration range kernels, or the squared-distance reduction (on the int8 view of the input and a shifted copy)")
     args = ap.parse_args()
     dev = torch.device("cuda:0")
@@ -58,7 +58,8 @@ def main():
     L.set_lowbit_path(fx.LOWBIT_PACKED_U4 if args.path == "packed" else fx.LOWBIT_MASKED_I8)
     L.set_lowbit_ratio(args.ratio)
     X = torch.from_numpy(c.X).to(dev)
-    mode = {"i8": fx.OUT_REQUANT_I8, "f32": fx.OUT_DEQUANT_F32, "i32": fx.OUT_ACC_I32}[args.out]
+    mode = {"i8": fx.OUT_REQUANT_I8, "f32": fx.OUT_DEQUANT_F32, "i32": fx.OUT_ACC_I32, "f16": fx.OUT_DEQUANT_F16,
+            "bf16": fx.OUT_DEQUANT_BF16}[args.out]
     M = X.numel() // L.K
     stream = torch.cuda.current_stream()
     if args.aux:

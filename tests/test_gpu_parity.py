@@ -29,7 +29,8 @@ def _layer(case, dev, perm, sx_group, conv=False, path=fx.LOWBIT_MASKED_I8):
 
 def _check_outputs(L, case, x4, x8, acc_e, dev, conv=False, x_shift=None):
     shape = acc_e.shape
-    for mode, dt in ((fx.OUT_ACC_I32, torch.int32), (fx.OUT_REQUANT_I8, torch.int8), (fx.OUT_DEQUANT_F32, torch.float32)):
+    for mode, dt in ((fx.OUT_ACC_I32, torch.int32), (fx.OUT_REQUANT_I8, torch.int8), (fx.OUT_DEQUANT_F32, torch.float32),
+                     (fx.OUT_DEQUANT_F16, torch.float16), (fx.OUT_DEQUANT_BF16, torch.bfloat16)):
         Y, guard_ok = helpers.with_guard(torch, shape, dt, dev)
         if conv:
             L.mixed_conv(x4, x8, case.Nb, case.H, case.W, case.x_scale, case.y_scale, mode, Y=Y, x_shift=x_shift)
@@ -38,7 +39,15 @@ def _check_outputs(L, case, x4, x8, acc_e, dev, conv=False, x_shift=None):
         torch.cuda.synchronize()
         fx.flexiq_check_status()
         guard_ok()
+        if mode == fx.OUT_DEQUANT_BF16:
+            # 16-bit patterns: both sides round the same fp32 value to nearest even
+            assert np.array_equal(Y.view(torch.int16).cpu().numpy().view(np.uint16),
+                                  oracle.epilogue_bf16_bits(acc_e, case.x_scale, case.w_scale, case.bias))
+            continue
         got = Y.cpu().numpy()
+        if mode == fx.OUT_DEQUANT_F16:
+            assert np.array_equal(got.view(np.uint16), oracle.epilogue_f16(acc_e, case.x_scale, case.w_scale, case.bias).view(np.uint16))
+            continue
         if mode == fx.OUT_ACC_I32:
             assert np.array_equal(got, acc_e)
         elif mode == fx.OUT_REQUANT_I8:
