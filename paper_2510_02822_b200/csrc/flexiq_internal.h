@@ -50,6 +50,13 @@ struct Layer {
     int32_t *chunk_ent_slab;  // [C/16] the same for a producer that already emits slab order: c | position << 24
     float *w_scale;  // [N]
     float *bias;     // [N] or nullptr
+    // perm, inv_perm, chunk_ent, chunk_ent_slab and sx live in ONE device block so that a layout uploads
+    // them with a single copy from the pinned mirror below
+    void *tables;             // the device block
+    void *tables_host;        // pinned mirror, same layout
+    size_t tables_bytes;
+    cudaEvent_t tables_event; // recorded after the upload: the mirror may be rewritten once it has passed
+    int tables_in_flight;
     // host copies
     int32_t *perm_host;
     uint8_t *sx_host;

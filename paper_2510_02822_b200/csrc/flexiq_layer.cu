@@ -188,8 +188,11 @@ static int validate_common(flexiq_layer_t *out, int C, int N, int G, const int8_
 static void free_layer(Layer *L)
 {
     if (!L) return;
-    cudaFree(L->w8); cudaFree(L->w8m); cudaFree(L->w4); cudaFree(L->wf); cudaFree(L->sw); cudaFree(L->sx);
-    cudaFree(L->perm); cudaFree(L->inv_perm); cudaFree(L->chunk_ent); cudaFree(L->chunk_ent_slab); cudaFree(L->w_scale); cudaFree(L->bias); cudaFree(L->alpha); cudaFree(L->beta);
+    if (L->tables_in_flight) cudaEventSynchronize(L->tables_event);
+    cudaFree(L->w8); cudaFree(L->w8m); cudaFree(L->w4); cudaFree(L->wf); cudaFree(L->sw);
+    cudaFree(L->tables); cudaFree(L->w_scale); cudaFree(L->bias); cudaFree(L->alpha); cudaFree(L->beta);
+    if (L->tables_host) cudaFreeHost(L->tables_host);
+    if (L->tables_event) cudaEventDestroy(L->tables_event);
     free(L->perm_host); free(L->sx_host);
     L->magic = 0;
     free(L);
@@ -214,30 +217,30 @@ int encode_weight_maps(Layer *L)
 // The layout post-processing of a handle for a group order (Sec. 5): uploads the order, the
 // activation positions in slab order and the chunk tables, and rebuilds the slab-order weights, their
 // positions and the 4-bit cache from the original-order weights.  Stream-ordered, allocates nothing
-// on the device; the host arrays are staged by the copies before they return.
+// on the device, does not wait for the stream: the tables go up in one copy from a pinned mirror.
 static int layout_layer(Layer *L, const int8_t *Wq, const int32_t *perm, const uint8_t *x_shift, cudaStream_t stream)
 {
     const int n_g = L->n_g, C = L->C, G = L->G, N = L->N;
+    // the pinned mirror is free again once the previous upload has read it (normally long ago)
+    if (L->tables_in_flight) FLEXIQ_CUDA_TRY(cudaEventSynchronize(L->tables_event));
     memcpy(L->perm_host, perm, sizeof(int32_t) * n_g);
     for (int j = 0; j < n_g; ++j) L->sx_host[j] = x_shift ? x_shift[perm[j]] : 0;  // slab order
-    FLEXIQ_CUDA_TRY(cudaMemcpyAsync(L->perm, L->perm_host, sizeof(int32_t) * n_g, cudaMemcpyHostToDevice, stream));
-    FLEXIQ_CUDA_TRY(cudaMemcpyAsync(L->sx, L->sx_host, n_g, cudaMemcpyHostToDevice, stream));
-    // chunk table: original chunk c lies in original group c*16/G, which is slab group j with perm[j] = that group
     const int n_c = C / 16, cpg = G / 16;
-    int32_t *ent = (int32_t *)malloc(sizeof(int32_t) * (2 * n_c + n_g));
-    if (!ent) return set_error(FLEXIQ_ERR_CUDA, "out of host memory");
+    int32_t *h_perm = static_cast<int32_t *>(L->tables_host), *h_inv = h_perm + n_g, *h_ent = h_inv + n_g, *h_ent_slab = h_ent + n_c;
+    uint8_t *h_sx = reinterpret_cast<uint8_t *>(h_ent_slab + n_c);
+    // chunk table: original chunk c lies in original group c*16/G, which is slab group j with perm[j] = that group
     for (int j = 0; j < n_g; ++j) {
+        h_perm[j] = perm[j];
+        h_inv[perm[j]] = j;
+        h_sx[j] = L->sx_host[j];
         for (int i = 0; i < cpg; ++i) {
-            ent[perm[j] * cpg + i] = (j * cpg + i) | ((int32_t)L->sx_host[j] << 24);
-            ent[n_c + j * cpg + i] = (j * cpg + i) | ((int32_t)L->sx_host[j] << 24);
+            h_ent[perm[j] * cpg + i] = (j * cpg + i) | ((int32_t)L->sx_host[j] << 24);
+            h_ent_slab[j * cpg + i] = (j * cpg + i) | ((int32_t)L->sx_host[j] << 24);
         }
-        ent[2 * n_c + perm[j]] = j;
     }
-    cudaError_t e1 = cudaMemcpyAsync(L->chunk_ent, ent, sizeof(int32_t) * n_c, cudaMemcpyHostToDevice, stream);
-    if (e1 == cudaSuccess) e1 = cudaMemcpyAsync(L->chunk_ent_slab, ent + n_c, sizeof(int32_t) * n_c, cudaMemcpyHostToDevice, stream);
-    if (e1 == cudaSuccess) e1 = cudaMemcpyAsync(L->inv_perm, ent + 2 * n_c, sizeof(int32_t) * n_g, cudaMemcpyHostToDevice, stream);
-    free(ent);  // pageable source: staged before the call returned
-    FLEXIQ_CUDA_TRY(e1);
+    FLEXIQ_CUDA_TRY(cudaMemcpyAsync(L->tables, L->tables_host, L->tables_bytes, cudaMemcpyHostToDevice, stream));
+    FLEXIQ_CUDA_TRY(cudaEventRecord(L->tables_event, stream));
+    L->tables_in_flight = 1;
     const size_t wbytes = (size_t)N * L->Kw;
     const long long total = (long long)n_g * N;
     const int threads = 128;
@@ -289,20 +292,24 @@ static int create_common(flexiq_layer_t *out, int is_conv, int C, int N, int R, 
     TRY_OR_FREE(cudaMalloc(&L->w4, (size_t)N * L->w4_pitch));
     TRY_OR_FREE(cudaMemsetAsync(L->w4, 0, (size_t)N * L->w4_pitch, stream));
     TRY_OR_FREE(cudaMalloc(&L->sw, (size_t)n_g * N));
-    TRY_OR_FREE(cudaMalloc(&L->sx, (size_t)n_g));
-    TRY_OR_FREE(cudaMalloc(&L->perm, sizeof(int32_t) * n_g));
+    {
+        // [perm n_g | inv_perm n_g | chunk_ent n_c | chunk_ent_slab n_c] int32, then sx [n_g] bytes
+        const int n_c = C / 16;
+        L->tables_bytes = sizeof(int32_t) * (2 * (size_t)n_g + 2 * (size_t)n_c) + (size_t)n_g;
+        TRY_OR_FREE(cudaMalloc(&L->tables, L->tables_bytes));
+        TRY_OR_FREE(cudaMallocHost(&L->tables_host, L->tables_bytes));
+        TRY_OR_FREE(cudaEventCreateWithFlags(&L->tables_event, cudaEventDisableTiming));
+        L->perm = static_cast<int32_t *>(L->tables);
+        L->inv_perm = L->perm + n_g;
+        L->chunk_ent = L->inv_perm + n_g;
+        L->chunk_ent_slab = L->chunk_ent + n_c;
+        L->sx = reinterpret_cast<uint8_t *>(L->chunk_ent_slab + n_c);
+    }
     TRY_OR_FREE(cudaMalloc(&L->w_scale, sizeof(float) * N));
     if (bias) TRY_OR_FREE(cudaMalloc(&L->bias, sizeof(float) * N));
     TRY_OR_FREE(cudaMalloc(&L->alpha, sizeof(float) * N));
     TRY_OR_FREE(cudaMalloc(&L->beta, sizeof(float) * N));
     L->cache_mode = -1;
-    {
-        const int n_c = C / 16;
-        cudaError_t e1 = cudaMalloc(&L->chunk_ent, sizeof(int32_t) * n_c);
-        if (e1 == cudaSuccess) e1 = cudaMalloc(&L->chunk_ent_slab, sizeof(int32_t) * n_c);
-        if (e1 == cudaSuccess) e1 = cudaMalloc(&L->inv_perm, sizeof(int32_t) * n_g);
-        TRY_OR_FREE(e1);
-    }
     TRY_OR_FREE(cudaMemcpyAsync(L->w_scale, w_scale, sizeof(float) * N, cudaMemcpyDeviceToDevice, stream));
     if (bias) TRY_OR_FREE(cudaMemcpyAsync(L->bias, bias, sizeof(float) * N, cudaMemcpyDeviceToDevice, stream));
     rc = layout_layer(L, Wq, perm, x_shift, stream);
