@@ -113,3 +113,53 @@ def test_relayout_in_place_matches_a_fresh_layer(dev):
         L.set_group_perm(Wq, np.zeros(n_g, dtype=np.int32))
     fx.flexiq_check_status()
     L.close()
+
+
+def test_relayout_in_place_conv_and_fused_tables(dev):
+    """The same for a convolution handle, and for the chunk tables a producer layer uses when it writes
+    this layer's slab directly (fused boundary): they follow the new order too."""
+    import oracle
+    case = inputs.resnet_conv("relay_c", 2, 14, 128, 64, 3, seed=93)
+    perm_a, sxg, _, _ = helpers.prepare_conv(case)
+    L = fx.Layer(torch.from_numpy(case.Wq).to(dev), torch.from_numpy(case.w_scale).to(dev), torch.from_numpy(case.bias).to(dev),
+                 perm_a, sxg, case.G, conv=(case.stride, case.pad))
+    Wq = torch.from_numpy(case.Wq).to(dev)
+    X = torch.from_numpy(case.X).to(dev)
+    q = oracle.quantize(case.X, case.x_scale)
+    n_g = case.C // case.G
+    perm_b = np.roll(np.arange(n_g, dtype=np.int32)[::-1].copy(), 3)
+    for perm in (perm_b, perm_a):
+        L.set_group_perm(Wq, perm, sxg)
+        L.set_lowbit_ratio(0.5)
+        x4, x8, _ = L.quantize_lower(X, case.x_scale)
+        y = L.mixed_conv(x4, x8, case.Nb, case.H, case.W, case.x_scale, case.y_scale, fx.OUT_REQUANT_I8)
+        sw = oracle.weight_positions_conv(case.Wq, case.G, perm)
+        acc = oracle.mixed_conv_acc(q, case.Wq, case.stride, case.pad, case.G, perm, sxg[perm].copy(), sw, oracle.n_low(0.5, n_g))
+        assert np.array_equal(y.cpu().numpy(), oracle.epilogue_i8(acc, case.x_scale, case.w_scale, case.bias, case.y_scale))
+    L.close()
+    # producer -> consumer chain: the consumer is laid out again, the producer's epilogue follows its new tables
+    a = inputs.ranged_linear("relay_a", 200, 128, 192, 16, seed=94, group_structured=True)
+    b = inputs.ranged_linear("relay_b", 200, 192, 96, 16, seed=95, group_structured=True)
+    pa, sa, sas, swa = helpers.prepare_linear(a)
+    pb, sb, _, _ = helpers.prepare_linear(b)
+    LA = fx.Layer(torch.from_numpy(a.Wq).to(dev), torch.from_numpy(a.w_scale).to(dev), torch.from_numpy(a.bias).to(dev), pa, sa, 16)
+    LB = fx.Layer(torch.from_numpy(b.Wq).to(dev), torch.from_numpy(b.w_scale).to(dev), torch.from_numpy(b.bias).to(dev), pb, sb, 16)
+    WB = torch.from_numpy(b.Wq).to(dev)
+    XA = torch.from_numpy(a.X).to(dev)
+    qa = oracle.quantize(a.X, a.x_scale)
+    next_scale = a.y_scale
+    for perm in (pb, np.arange(192 // 16, dtype=np.int32)[::-1].copy()):
+        LB.set_group_perm(WB, perm, sb)
+        for L_, r in ((LA, 0.5), (LB, 0.5)):
+            L_.set_lowbit_ratio(r)
+        x4, x8, _ = LA.quantize_lower(XA, a.x_scale)
+        slab = LA.mixed_gemm_to_slab(x4, x8, a.M, a.x_scale, LB, next_scale)
+        yb = LB.mixed_gemm(slab, None, a.M, next_scale, b.y_scale, fx.OUT_REQUANT_I8)
+        acc_a = oracle.mixed_gemm_acc(qa, a.Wq, 16, pa, sas, swa, oracle.n_low(0.5, 128 // 16))
+        qb = oracle.epilogue_i8(acc_a, a.x_scale, a.w_scale, a.bias, next_scale)
+        swb = oracle.weight_positions_linear(b.Wq, 16, perm)
+        acc_b = oracle.mixed_gemm_acc(qb, b.Wq, 16, perm, sb[perm].copy(), swb, oracle.n_low(0.5, 192 // 16))
+        assert np.array_equal(yb.cpu().numpy(), oracle.epilogue_i8(acc_b, next_scale, b.w_scale, b.bias, b.y_scale))
+    fx.flexiq_check_status()
+    LA.close()
+    LB.close()
