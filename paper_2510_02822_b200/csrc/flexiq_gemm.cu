@@ -644,7 +644,9 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                 // several filter taps per stage: one barrier round trip pays for all of them
                 for (int tap0 = 0; tap0 < p.T && ok; tap0 += p.tps) {
                     const int nt = min(p.tps, p.T - tap0);
+                    PROF_T0(tq0);
                     if (!__all_sync(0xffffffffu, wait_bounded(empty0 + 8 * stage, phase ^ 1, abort_flag, 1))) { ok = false; break; }
+                    PROF_ADD(prof_wait, tq0);
                     if (ptx::elect_one()) {
                         const uint32_t sa = stage0 + stage * stage_bytes;
                         if (leader) ptx::mbar_expect_tx_s(full0 + 8 * stage, (uint32_t)(CG * nt * (a_sub + b_sub)));
@@ -770,14 +772,29 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                     const int ks = (p.C + 31) >> 5;  // K steps of one tap (C <= BK)
                     for (int tap0 = 0; tap0 < p.T && ok; tap0 += p.tps) {
                         const int nt = min(p.tps, p.T - tap0);
+                        PROF_T0(tq1);
                         if (!__all_sync(0xffffffffu, wait_bounded(full0 + 8 * stage, phase, abort_flag, 3))) { ok = false; break; }
+                        PROF_ADD(prof_wait_full, tq1);
                         const uint32_t a_lo = a_lo0 + stage * stage_step, b_lo = b_lo0 + stage * stage_step;
                         if (ptx::elect_one()) {
-                            for (int i = 0; i < nt; ++i)
-                                for (int k = 0; k < ks; ++k) {
-                                    ptx::mma_i8_s<CG>(d_tmem, a_lo + i * (a_sub >> 4) + 2 * k, b_lo + i * (b_sub >> 4) + 2 * k, desc_hi, idesc, acc);
-                                    acc = 1;
-                                }
+                            const uint32_t a_step = (uint32_t)(a_sub >> 4), b_step = (uint32_t)(b_sub >> 4);
+                            if (nt == 3 && ks == 2) {
+                                // three taps of 64 channels (a filter row of the 64-channel 3x3 convolutions): the issuing
+                                // lane's instruction stream bounds these small MMAs, so no loop around them
+                                ptx::mma_i8_s<CG>(d_tmem, a_lo, b_lo, desc_hi, idesc, acc);
+                                ptx::mma_i8_s<CG>(d_tmem, a_lo + 2, b_lo + 2, desc_hi, idesc, 1);
+                                ptx::mma_i8_s<CG>(d_tmem, a_lo + a_step, b_lo + b_step, desc_hi, idesc, 1);
+                                ptx::mma_i8_s<CG>(d_tmem, a_lo + a_step + 2, b_lo + b_step + 2, desc_hi, idesc, 1);
+                                ptx::mma_i8_s<CG>(d_tmem, a_lo + 2 * a_step, b_lo + 2 * b_step, desc_hi, idesc, 1);
+                                ptx::mma_i8_s<CG>(d_tmem, a_lo + 2 * a_step + 2, b_lo + 2 * b_step + 2, desc_hi, idesc, 1);
+                            } else {
+                                uint32_t a2 = acc;
+                                for (int i = 0; i < nt; ++i)
+                                    for (int k = 0; k < ks; ++k) {
+                                        ptx::mma_i8_s<CG>(d_tmem, a_lo + i * a_step + 2 * k, b_lo + i * b_step + 2 * k, desc_hi, idesc, a2);
+                                        a2 = 1;
+                                    }
+                            }
                             ptx::mma_commit_s<CG>(empty0 + 8 * stage);
                         }
                         __syncwarp();
