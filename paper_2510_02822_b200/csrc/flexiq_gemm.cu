@@ -134,6 +134,41 @@ struct TileWalk {
     }
 };
 
+// Output pixel coordinates (image n, row h, column w) of a running row index that advances by a fixed
+// number of rows per step, plus one block of rows when the tile walk wraps to the next block row.
+struct PixelWalk {
+    int n, h, w;
+    int dn, dh, dw, en, eh, ew;
+    __device__ __forceinline__ static void split(long long idx, int P, int Q, int &n_, int &h_, int &w_)
+    {
+        const long long pq = (long long)P * Q;
+        n_ = (int)(idx / pq);
+        const int rem = (int)(idx - (long long)n_ * pq);
+        h_ = rem / Q;
+        w_ = rem - h_ * Q;
+    }
+    __device__ __forceinline__ void init(long long first_row, long long step_rows, long long block_rows, int P, int Q)
+    {
+        split(first_row, P, Q, n, h, w);
+        split(step_rows, P, Q, dn, dh, dw);
+        split(block_rows, P, Q, en, eh, ew);
+    }
+    __device__ __forceinline__ void add(int an, int ah, int aw, int P, int Q)
+    {
+        w += aw;
+        if (w >= Q) { w -= Q; ++h; }
+        h += ah;
+        if (h >= P) { h -= P; ++n; }
+        n += an;
+    }
+    // one step of the tile walk that moved to another block row; extra = 1 when it also wrapped
+    __device__ __forceinline__ void advance(int extra, int P, int Q)
+    {
+        add(dn, dh, dw, P, Q);
+        if (extra > 0) add(en, eh, ew, P, Q);
+    }
+};
+
 // two int32 -> two saturated int8 in the low half, upper half taken from c's low half
 __device__ __forceinline__ unsigned pack2_sat_s8(int hi, int lo, unsigned c)
 {
@@ -629,19 +664,25 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
         PROF_DECL(prof_wait);
         PROF_T0(prof_start);
         TileWalk tw;
-        for (tw.init(first_tile, tile_step, num_tiles, p.n_tiles); tw.left > 0 && ok; tw.next()) {
+        tw.init(first_tile, tile_step, num_tiles, p.n_tiles);
+        // Output pixel (image, row, column) of this CTA's first row in the current tile, kept up to date by
+        // additions: the divisions are done once per kernel, not once per tile, in this single-lane loop.
+        PixelWalk pw;
+        if (p.im2col) pw.init(((long long)tw.m_blk * CG + cta_rank) * BM, (long long)tw.step_m * CG * BM, (long long)CG * BM, p.P, p.Q);
+        int prev_m = tw.m_blk;
+        for (; tw.left > 0 && ok; tw.next()) {
             const long long m0 = ((long long)tw.m_blk * CG + cta_rank) * BM;
             const int n0 = tw.n_blk * BN + (int)cta_rank * b_rows;
             int pix_w = 0, pix_h = 0, pix_n = 0;
             if (p.im2col) {
-                const long long pq = (long long)p.P * p.Q;
-                pix_n = (int)(m0 / pq);
-                const int rem = (int)(m0 - (long long)pix_n * pq);
-                pix_h = (rem / p.Q) * p.stride - p.pad;
-                pix_w = (rem % p.Q) * p.stride - p.pad;
+                if (tw.m_blk != prev_m) { pw.advance(tw.m_blk - prev_m - tw.step_m, p.P, p.Q); prev_m = tw.m_blk; }
+                pix_n = pw.n;
+                pix_h = pw.h * p.stride - p.pad;
+                pix_w = pw.w * p.stride - p.pad;
             }
             if (p.tps > 1) {
                 // several filter taps per stage: one barrier round trip pays for all of them
+                int tap_s = 0, tap_r = 0, tap_k = 0;   // running tap coordinates: no division in the issuing lane's loop
                 for (int tap0 = 0; tap0 < p.T && ok; tap0 += p.tps) {
                     const int nt = min(p.tps, p.T - tap0);
                     PROF_T0(tq0);
@@ -651,12 +692,17 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                         const uint32_t sa = stage0 + stage * stage_bytes;
                         if (leader) ptx::mbar_expect_tx_s(full0 + 8 * stage, (uint32_t)(CG * nt * (a_sub + b_sub)));
                         const uint32_t bar = full0_lead + 8 * stage;
+                        int ts = tap_s, tr = tap_r, tk = tap_k;
                         for (int i = 0; i < nt; ++i) {
-                            const int tap = tap0 + i;
-                            ptx::tma_load_im2col_4d_s<CG>(sa + i * a_sub, &mapA_hi, bar, 0, pix_w, pix_h, pix_n,
-                                                          (uint16_t)(tap % p.S), (uint16_t)(tap / p.S));
-                            ptx::tma_load_2d_s<CG>(sa + b_off + i * b_sub, &mapB_hi, bar, tap * p.C, n0);
+                            ptx::tma_load_im2col_4d_s<CG>(sa + i * a_sub, &mapA_hi, bar, 0, pix_w, pix_h, pix_n, (uint16_t)ts, (uint16_t)tr);
+                            ptx::tma_load_2d_s<CG>(sa + b_off + i * b_sub, &mapB_hi, bar, tk, n0);
+                            tk += p.C;
+                            if (++ts == p.S) { ts = 0; ++tr; }
                         }
+                    }
+                    for (int i = 0; i < nt; ++i) {
+                        tap_k += p.C;
+                        if (++tap_s == p.S) { tap_s = 0; ++tap_r; }
                     }
                     __syncwarp();
                     ++issued;
