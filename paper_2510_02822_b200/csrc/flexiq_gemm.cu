@@ -79,6 +79,10 @@ struct GemmParams {
     int next_K_lo;             // the next layer's max_4bit_ch
     int relu;                  // clamp at zero before the re-quantization
     int tma_store;             // int8 output leaves through shared memory and tiled bulk stores (mapY)
+    // Resident weights (convolutions on the multi-tap path whose output channels fit one tile): every tap's
+    // weight tile is loaded once per CTA and stays in shared memory in front of the ring, whose stages then hold
+    // activation taps only: half as many copies per tile for the producer lane, which bounds these layers.
+    int b_res;
     // packed low-bit path only: positions the expander warps shift the 4-bit values back to
     const uint8_t *sx;   // [n_g] activation positions, slab order
     const uint8_t *sw;   // [n_g][N] weight positions
@@ -601,7 +605,8 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
     const int b_rows = BN / CG;                       // rows of the B tile this CTA loads
     // one stage = tps sub-tiles of A (BM x BK each) followed by tps sub-tiles of B (b_rows x BK each)
     const int a_sub = BM * p.BK, b_sub = b_rows * p.BK, b_off = p.tps * a_sub;
-    const int stage_bytes = p.tps * (a_sub + b_sub);
+    const int stage_bytes = p.b_res ? p.tps * a_sub : p.tps * (a_sub + b_sub);
+    const int ring_off = p.b_res ? ((p.T * b_sub + 1023) & ~1023) : 0;   // resident weight tiles lie in front of the ring
     const int num_tiles = p.m_tiles * p.n_tiles;
     const uint32_t cta_rank = CG == 2 ? ptx::cluster_ctarank() : 0u;
     const bool leader = cta_rank == 0;
@@ -651,7 +656,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             ptx::prefetch_tmap(&mapB_hi);
         }
         const uint32_t tx_bytes = (uint32_t)(CG * (BM * p.BK + b_rows * p.BK));  // both CTAs' loads
-        const uint32_t stage0 = ptx::smem_u32(stage_base);
+        const uint32_t stage0 = ptx::smem_u32(stage_base) + (uint32_t)ring_off;
         const uint32_t empty0 = ptx::smem_u32(empty_bar);
         const uint32_t full0 = ptx::smem_u32(full_bar);
         const uint32_t full0_lead = CG == 2 ? ptx::mapa(full0, 0) : full0;  // transaction bytes go to the leader's barrier
@@ -665,6 +670,15 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
         PROF_T0(prof_start);
         TileWalk tw;
         tw.init(first_tile, tile_step, num_tiles, p.n_tiles);
+        if (p.b_res && tw.left > 0 && ptx::elect_one()) {
+            // all taps' weight tiles of this CTA's (only) column block, once
+            const uint32_t bar = ptx::smem_u32(&raw_full[0]);
+            if (leader) ptx::mbar_expect_tx_s(bar, (uint32_t)(CG * p.T * b_sub));
+            const uint32_t bar_lead = CG == 2 ? ptx::mapa(bar, 0) : bar;
+            for (int t = 0; t < p.T; ++t)
+                ptx::tma_load_2d_s<CG>(ptx::smem_u32(stage_base) + t * b_sub, &mapB_hi, bar_lead, t * p.C, (int)cta_rank * b_rows);
+        }
+        __syncwarp();
         // Output pixel (image, row, column) of this CTA's first row in the current tile, kept up to date by
         // additions: the divisions are done once per kernel, not once per tile, in this single-lane loop.
         PixelWalk pw;
@@ -690,12 +704,12 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                     PROF_ADD(prof_wait, tq0);
                     if (ptx::elect_one()) {
                         const uint32_t sa = stage0 + stage * stage_bytes;
-                        if (leader) ptx::mbar_expect_tx_s(full0 + 8 * stage, (uint32_t)(CG * nt * (a_sub + b_sub)));
+                        if (leader) ptx::mbar_expect_tx_s(full0 + 8 * stage, (uint32_t)(CG * nt * (p.b_res ? a_sub : a_sub + b_sub)));
                         const uint32_t bar = full0_lead + 8 * stage;
                         int ts = tap_s, tr = tap_r, tk = tap_k;
                         for (int i = 0; i < nt; ++i) {
                             ptx::tma_load_im2col_4d_s<CG>(sa + i * a_sub, &mapA_hi, bar, 0, pix_w, pix_h, pix_n, (uint16_t)ts, (uint16_t)tr);
-                            ptx::tma_load_2d_s<CG>(sa + b_off + i * b_sub, &mapB_hi, bar, tk, n0);
+                            if (!p.b_res) ptx::tma_load_2d_s<CG>(sa + b_off + i * b_sub, &mapB_hi, bar, tk, n0);
                             tk += p.C;
                             if (++ts == p.S) { ts = 0; ++tr; }
                         }
@@ -791,7 +805,9 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
         // The whole warp walks the loops; one elected lane issues the MMAs and their commits.
         if (leader) {
             const uint32_t idesc = ptx::idesc_i8(BM * CG, BN);
-            const uint64_t adesc0 = ptx::smem_desc(ptx::smem_u32(stage_base), p.BK);
+            const uint64_t adesc0 = ptx::smem_desc(ptx::smem_u32(stage_base) + (uint32_t)ring_off, p.BK);
+            const uint32_t bres_lo = (uint32_t)ptx::smem_desc(ptx::smem_u32(stage_base), p.BK);   // resident weight tiles
+            bool bres_ready = false;
             const uint32_t desc_hi = (uint32_t)(adesc0 >> 32);
             const uint32_t a_lo0 = (uint32_t)adesc0;
             const uint32_t b_lo0 = a_lo0 + (uint32_t)(b_off >> 4);
@@ -821,7 +837,12 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                         PROF_T0(tq1);
                         if (!__all_sync(0xffffffffu, wait_bounded(full0 + 8 * stage, phase, abort_flag, 3))) { ok = false; break; }
                         PROF_ADD(prof_wait_full, tq1);
-                        const uint32_t a_lo = a_lo0 + stage * stage_step, b_lo = b_lo0 + stage * stage_step;
+                        if (p.b_res && !bres_ready) {
+                            if (!__all_sync(0xffffffffu, wait_bounded(&raw_full[0], 0, abort_flag, 6))) { ok = false; break; }
+                            bres_ready = true;
+                        }
+                        const uint32_t a_lo = a_lo0 + stage * stage_step;
+                        const uint32_t b_lo = p.b_res ? bres_lo + (uint32_t)tap0 * (uint32_t)(b_sub >> 4) : b_lo0 + stage * stage_step;
                         if (ptx::elect_one()) {
                             const uint32_t a_step = (uint32_t)(a_sub >> 4), b_step = (uint32_t)(b_sub >> 4);
                             if (nt == 3 && ks == 2) {
@@ -1266,6 +1287,11 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
         if (p.tps < 1) p.tps = 1;
     }
     p.stages = kStageRegion / (p.tps * (BM + bn / cg) * p.BK);
+    if (p.tps > 1 && p.n_tiles == 1) {
+        const int b_all = ((p.T * (bn / cg) * p.BK + 1023) / 1024) * 1024;
+        const int st = (kStageRegion - b_all) / (p.tps * BM * p.BK);
+        if (b_all <= 65536 && st >= 4) { p.b_res = 1; p.stages = st; }
+    }
     if (p.stages > kMaxStages) p.stages = kMaxStages;
     if (packed) {  // room for the ring of raw 4-bit tiles behind the operand ring
         const int raw = kRawStages * (BM + bn) * (p.BK / 2);
