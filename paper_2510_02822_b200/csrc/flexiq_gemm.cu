@@ -43,7 +43,7 @@ __device__ long long g_prof[16];
 
 constexpr int BM = 128;
 constexpr int kNumWorkWarps = 16;                     // epilogue warps (+ expander warps on the packed path)
-constexpr int kThreads = 32 * (2 + kNumWorkWarps);
+constexpr int kThreads = 32 * (3 + kNumWorkWarps);      // producer, two MMA warps (the second one last), work warps
 constexpr int kRawStages = 2;                         // packed path: ring of raw 4-bit tiles in front of the operand ring
 constexpr uint32_t kSpinLimit = 1u << 21;              // parked waits of <= 1 us each: about two seconds at most
 constexpr int kStageRegion = 196608;                  // shared memory given to the operand ring
@@ -595,7 +595,8 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
     uint64_t *tmem_empty = tmem_full + 2;
     uint64_t *raw_full = tmem_empty + 2;
     uint64_t *raw_empty = raw_full + kRawStages;
-    uint32_t *tmem_ptr_s = reinterpret_cast<uint32_t *>(raw_empty + kRawStages);
+    uint64_t *turn_bar = raw_empty + kRawStages;     // hand-over between the two MMA warps: one phase per tile
+    uint32_t *tmem_ptr_s = reinterpret_cast<uint32_t *>(turn_bar + 1);
     constexpr int kEpiWarps = PK ? 8 : 16;
     constexpr int kExpWarps = PK ? 8 : 0;
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_ptr_s + 1);
@@ -627,6 +628,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             ptx::mbar_init(&raw_full[r], 1);
             ptx::mbar_init(&raw_empty[r], PK ? kExpWarps : 1);
         }
+        ptx::mbar_init(turn_bar, 1);
         *abort_flag = 0;
         ptx::fence_mbar_init();
     }
@@ -800,9 +802,17 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                 }
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------------------------------------- MMA issuer
+    } else if (warp == 1 || (!PK && warp == 2 + kNumWorkWarps)) {
+        // ------------------------------------------------------------- MMA issuers
         // The whole warp walks the loops; one elected lane issues the MMAs and their commits.
+        // Two warps take the CTA's tiles in turn (even tiles and accumulator 0, odd tiles and accumulator 1;
+        // on the packed path one warp takes them all): a lone warp shows the latency of every instruction, and
+        // the bookkeeping of a tile boundary (≈ 500 cycles) then runs behind the other warp's MMAs.  The waits
+        // on the ring stay in ring order: a warp starts on its tile's first stage only after the other has
+        // passed the wait for its own last stage (one barrier phase per tile), so the parity of a ring barrier
+        // means what it means to a single consumer.
+        const bool duo = !PK;
+        const int my = warp == 1 ? 0 : 1;
         if (leader) {
             const uint32_t idesc = ptx::idesc_i8(BM * CG, BN);
             const uint64_t adesc0 = ptx::smem_desc(ptx::smem_u32(stage_base) + (uint32_t)ring_off, p.BK);
@@ -816,17 +826,28 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             const uint32_t full0 = ptx::smem_u32(full_bar);
             const int ks_full = p.BK >> 5;
             uint32_t stage = 0, phase = 0;
-            int buf = 0;
+            int buf = duo ? my : 0;
             uint32_t buf_phase = 0;
             bool ok = true;
             PROF_DECL(prof_wait_acc);
             PROF_DECL(prof_wait_full);
             PROF_T0(prof_start);
+            const int tile_slots = p.tps > 1 ? (p.T + p.tps - 1) / p.tps : p.T * (p.nb_lo + p.nb_hi);  // ring stages per tile
+            int ti = 0;                                          // index of the tile in this CTA's sequence
             TileWalk tw;
-            for (tw.init(first_tile, tile_step, num_tiles, p.n_tiles); tw.left > 0 && ok; tw.next()) {
+            for (tw.init(first_tile, tile_step, num_tiles, p.n_tiles); tw.left > 0 && ok; tw.next(), ++ti) {
+                if (duo && (ti & 1) != my) {
+                    // the other warp's tile: step over its ring stages
+                    stage += (uint32_t)tile_slots;
+                    while (stage >= (uint32_t)p.stages) { stage -= (uint32_t)p.stages; phase ^= 1; }
+                    continue;
+                }
+                int slot = 0;                                    // stages of this tile passed so far
                 PROF_T0(t0);
                 if (!__all_sync(0xffffffffu, wait_bounded(&tmem_empty[buf], buf_phase ^ 1, abort_flag, 2))) break;
                 PROF_ADD(prof_wait_acc, t0);
+                // the other warp has passed the wait for the last stage of the tile before this one
+                if (duo && ti > 0 && !__all_sync(0xffffffffu, wait_bounded(turn_bar, (uint32_t)((ti - 1) & 1), abort_flag, 7))) break;
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)buf * buf_stride;
                 uint32_t acc = 0;
@@ -837,6 +858,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                         PROF_T0(tq1);
                         if (!__all_sync(0xffffffffu, wait_bounded(full0 + 8 * stage, phase, abort_flag, 3))) { ok = false; break; }
                         PROF_ADD(prof_wait_full, tq1);
+                        if (duo && ++slot == tile_slots && lane == 0) ptx::mbar_arrive(turn_bar);   // the other warp may go on
                         if (p.b_res && !bres_ready) {
                             if (!__all_sync(0xffffffffu, wait_bounded(&raw_full[0], 0, abort_flag, 6))) { ok = false; break; }
                             bres_ready = true;
@@ -878,6 +900,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                             PROF_T0(t1);
                             if (!__all_sync(0xffffffffu, wait_bounded(full0 + 8 * stage, phase, abort_flag, 3))) { ok = false; break; }
                             PROF_ADD(prof_wait_full, t1);
+                            if (duo && ++slot == tile_slots && lane == 0) ptx::mbar_arrive(turn_bar);   // the other warp may go on
                             const uint32_t a_lo = a_lo0 + stage * stage_step, b_lo = b_lo0 + stage * stage_step;
                             const int ks = cb == nb - 1 ? ks_last : ks_full;
                             if (ptx::elect_one()) {
@@ -904,11 +927,14 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                 }
                 if (ok && ptx::elect_one()) ptx::mma_commit_s<CG>(ptx::smem_u32(&tmem_full[buf]));
                 __syncwarp();
-                if ((buf ^= 1) == 0) buf_phase ^= 1;
+                if (duo) buf_phase ^= 1;                         // this warp's accumulator again at its next tile
+                else if ((buf ^= 1) == 0) buf_phase ^= 1;
             }
+            if (my == 0) {
             PROF_STORE(4, prof_wait_acc);
             PROF_STORE(5, prof_wait_full);
             PROF_STORE(6, clock64() - prof_start);
+            }
         }
     } else {
         if (warp < 2 + kEpiWarps) {
@@ -930,7 +956,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             else if (p.out_mode == FLEXIQ_OUT_DEQUANT_F16) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_F16>(p, x, warp & 3, e >> 2, lane);
             else if (p.out_mode == FLEXIQ_OUT_DEQUANT_BF16) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_BF16>(p, x, warp & 3, e >> 2, lane);
             else epilogue_role<CG, FLEXIQ_OUT_ACC_I32>(p, x, warp & 3, e >> 2, lane);
-        } else if (PK) {
+        } else if (PK && warp < 2 + kNumWorkWarps) {
             // --------------------------------------------------------- expanders (packed path)
             // Widen each raw 4-bit tile into the operand ring: 8 packed bytes -> one 16-byte unit
             // (nibble << position) at its swizzled place, activations shifted by sx[group], weights
