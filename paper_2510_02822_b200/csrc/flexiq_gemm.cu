@@ -8,7 +8,8 @@
 // registers for the shift.  A persistent, warp-specialised CTA per SM, or a CTA pair (cluster of two,
 // cta_group::2) per 256-row tile:
 //   warp 0       TMA producer (tiled loads for linear layers, im2col loads for convs)
-//   warp 1       TMEM allocation + MMA issue (one elected lane)
+//   warp 1, 18   MMA issue (one elected lane each), tiles taken in turn with one accumulator each; warp 1
+//                also allocates TMEM (on the packed path warp 1 issues alone)
 //   warps 2..17  epilogue, four per TMEM lane quadrant: tcgen05.ld, scale / bias / round / clip, the
 //                results staged in shared memory 32 rows x 32 bytes at a time and written by tiled bulk
 //                stores (the fused boundary in original channel order scatters 16-byte chunks directly);
