@@ -575,7 +575,10 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
 // accumulator rows held in its own TMEM.  Operand traffic from L2 per MAC drops by a third.
 // PK = 1 (single CTA only): the low slab arrives as packed 4-bit tiles; eight expander warps
 // widen them into the operand ring (eight epilogue warps remain).
-template <int CG, int PK>
+// KIND 0: linear layers and 1x1 convolutions (plain 2-D copies, one K block per stage); KIND 1: everything a
+// convolution may need (im2col copies, several taps per stage, resident weight tiles).  The issuing warps'
+// instruction streams are on the critical path of a tile, so the first kind carries none of the second's code.
+template <int CG, int PK, int KIND>
 __global__ void __launch_bounds__(kThreads, 1)
 mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_constant__ CUtensorMap mapA_hi,
                   const __grid_constant__ CUtensorMap mapB_lo, const __grid_constant__ CUtensorMap mapB_hi,
@@ -604,11 +607,14 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int BN = p.BN;
+    const bool k_im2col = KIND != 0 && p.im2col;      // compile-time false for KIND 0: the branches below fold away
+    const int k_tps = KIND != 0 ? p.tps : 1;
+    const bool k_bres = KIND != 0 && p.b_res;
     const int b_rows = BN / CG;                       // rows of the B tile this CTA loads
     // one stage = tps sub-tiles of A (BM x BK each) followed by tps sub-tiles of B (b_rows x BK each)
-    const int a_sub = BM * p.BK, b_sub = b_rows * p.BK, b_off = p.tps * a_sub;
-    const int stage_bytes = p.b_res ? p.tps * a_sub : p.tps * (a_sub + b_sub);
-    const int ring_off = p.b_res ? ((p.T * b_sub + 1023) & ~1023) : 0;   // resident weight tiles lie in front of the ring
+    const int a_sub = BM * p.BK, b_sub = b_rows * p.BK, b_off = k_tps * a_sub;
+    const int stage_bytes = k_bres ? k_tps * a_sub : k_tps * (a_sub + b_sub);
+    const int ring_off = k_bres ? ((p.T * b_sub + 1023) & ~1023) : 0;   // resident weight tiles lie in front of the ring
     const int num_tiles = p.m_tiles * p.n_tiles;
     const uint32_t cta_rank = CG == 2 ? ptx::cluster_ctarank() : 0u;
     const bool leader = cta_rank == 0;
@@ -673,7 +679,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
         PROF_T0(prof_start);
         TileWalk tw;
         tw.init(first_tile, tile_step, num_tiles, p.n_tiles);
-        if (p.b_res && tw.left > 0 && ptx::elect_one()) {
+        if (k_bres && tw.left > 0 && ptx::elect_one()) {
             // all taps' weight tiles of this CTA's (only) column block, once
             const uint32_t bar = ptx::smem_u32(&raw_full[0]);
             if (leader) ptx::mbar_expect_tx_s(bar, (uint32_t)(CG * p.T * b_sub));
@@ -685,34 +691,34 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
         // Output pixel (image, row, column) of this CTA's first row in the current tile, kept up to date by
         // additions: the divisions are done once per kernel, not once per tile, in this single-lane loop.
         PixelWalk pw;
-        if (p.im2col) pw.init(((long long)tw.m_blk * CG + cta_rank) * BM, (long long)tw.step_m * CG * BM, (long long)CG * BM, p.P, p.Q);
+        if (k_im2col) pw.init(((long long)tw.m_blk * CG + cta_rank) * BM, (long long)tw.step_m * CG * BM, (long long)CG * BM, p.P, p.Q);
         int prev_m = tw.m_blk;
         for (; tw.left > 0 && ok; tw.next()) {
             const long long m0 = ((long long)tw.m_blk * CG + cta_rank) * BM;
             const int n0 = tw.n_blk * BN + (int)cta_rank * b_rows;
             int pix_w = 0, pix_h = 0, pix_n = 0;
-            if (p.im2col) {
+            if (k_im2col) {
                 if (tw.m_blk != prev_m) { pw.advance(tw.m_blk - prev_m - tw.step_m, p.P, p.Q); prev_m = tw.m_blk; }
                 pix_n = pw.n;
                 pix_h = pw.h * p.stride - p.pad;
                 pix_w = pw.w * p.stride - p.pad;
             }
-            if (p.tps > 1) {
+            if (k_tps > 1) {
                 // several filter taps per stage: one barrier round trip pays for all of them
                 int tap_s = 0, tap_r = 0, tap_k = 0;   // running tap coordinates: no division in the issuing lane's loop
-                for (int tap0 = 0; tap0 < p.T && ok; tap0 += p.tps) {
-                    const int nt = min(p.tps, p.T - tap0);
+                for (int tap0 = 0; tap0 < p.T && ok; tap0 += k_tps) {
+                    const int nt = min(k_tps, p.T - tap0);
                     PROF_T0(tq0);
                     if (!__all_sync(0xffffffffu, wait_bounded(empty0 + 8 * stage, phase ^ 1, abort_flag, 1))) { ok = false; break; }
                     PROF_ADD(prof_wait, tq0);
                     if (ptx::elect_one()) {
                         const uint32_t sa = stage0 + stage * stage_bytes;
-                        if (leader) ptx::mbar_expect_tx_s(full0 + 8 * stage, (uint32_t)(CG * nt * (p.b_res ? a_sub : a_sub + b_sub)));
+                        if (leader) ptx::mbar_expect_tx_s(full0 + 8 * stage, (uint32_t)(CG * nt * (k_bres ? a_sub : a_sub + b_sub)));
                         const uint32_t bar = full0_lead + 8 * stage;
                         int ts = tap_s, tr = tap_r, tk = tap_k;
                         for (int i = 0; i < nt; ++i) {
                             ptx::tma_load_im2col_4d_s<CG>(sa + i * a_sub, &mapA_hi, bar, 0, pix_w, pix_h, pix_n, (uint16_t)ts, (uint16_t)tr);
-                            if (!p.b_res) ptx::tma_load_2d_s<CG>(sa + b_off + i * b_sub, &mapB_hi, bar, tk, n0);
+                            if (!k_bres) ptx::tma_load_2d_s<CG>(sa + b_off + i * b_sub, &mapB_hi, bar, tk, n0);
                             tk += p.C;
                             if (++ts == p.S) { ts = 0; ++tr; }
                         }
@@ -747,7 +753,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                                 const uint32_t ra = raw0 + rstage * raw_bytes;
                                 const uint32_t bar = ptx::smem_u32(&raw_full[rstage]);
                                 ptx::mbar_expect_tx_s(bar, raw_bytes);
-                                if (p.im2col)
+                                if (k_im2col)
                                     ptx::tma_load_im2col_4d_s<1>(ra, ma, bar, xa >> 1, pix_w, pix_h, pix_n, (uint16_t)tap_s, (uint16_t)tap_r);
                                 else
                                     ptx::tma_load_2d_s<1>(ra, ma, bar, xa >> 1, (int)m0);
@@ -769,7 +775,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                             if (leader) ptx::mbar_expect_tx_s(full0 + 8 * stage, tx_bytes);
                             if (PK) ptx::mbar_arrive_count(&full_bar[stage], PK ? kExpWarps - 1 : 0);  // stand in for the expander warps
                             const uint32_t bar = full0_lead + 8 * stage;
-                            if (p.im2col)
+                            if (k_im2col)
                                 ptx::tma_load_im2col_4d_s<CG>(sa, ma, bar, xa, pix_w, pix_h, pix_n, (uint16_t)tap_s, (uint16_t)tap_r);
                             else
                                 ptx::tma_load_2d_s<CG>(sa, ma, bar, xa, (int)m0);
@@ -833,7 +839,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             PROF_DECL(prof_wait_acc);
             PROF_DECL(prof_wait_full);
             PROF_T0(prof_start);
-            const int tile_slots = p.tps > 1 ? (p.T + p.tps - 1) / p.tps : p.T * (p.nb_lo + p.nb_hi);  // ring stages per tile
+            const int tile_slots = k_tps > 1 ? (p.T + k_tps - 1) / k_tps : p.T * (p.nb_lo + p.nb_hi);  // ring stages per tile
             int ti = 0;                                          // index of the tile in this CTA's sequence
             TileWalk tw;
             for (tw.init(first_tile, tile_step, num_tiles, p.n_tiles); tw.left > 0 && ok; tw.next(), ++ti) {
@@ -852,20 +858,20 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                 ptx::tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)buf * buf_stride;
                 uint32_t acc = 0;
-                if (p.tps > 1) {
+                if (k_tps > 1) {
                     const int ks = (p.C + 31) >> 5;  // K steps of one tap (C <= BK)
-                    for (int tap0 = 0; tap0 < p.T && ok; tap0 += p.tps) {
-                        const int nt = min(p.tps, p.T - tap0);
+                    for (int tap0 = 0; tap0 < p.T && ok; tap0 += k_tps) {
+                        const int nt = min(k_tps, p.T - tap0);
                         PROF_T0(tq1);
                         if (!__all_sync(0xffffffffu, wait_bounded(full0 + 8 * stage, phase, abort_flag, 3))) { ok = false; break; }
                         PROF_ADD(prof_wait_full, tq1);
                         if (duo && ++slot == tile_slots && lane == 0) ptx::mbar_arrive(turn_bar);   // the other warp may go on
-                        if (p.b_res && !bres_ready) {
+                        if (k_bres && !bres_ready) {
                             if (!__all_sync(0xffffffffu, wait_bounded(&raw_full[0], 0, abort_flag, 6))) { ok = false; break; }
                             bres_ready = true;
                         }
                         const uint32_t a_lo = a_lo0 + stage * stage_step;
-                        const uint32_t b_lo = p.b_res ? bres_lo + (uint32_t)tap0 * (uint32_t)(b_sub >> 4) : b_lo0 + stage * stage_step;
+                        const uint32_t b_lo = k_bres ? bres_lo + (uint32_t)tap0 * (uint32_t)(b_sub >> 4) : b_lo0 + stage * stage_step;
                         if (ptx::elect_one()) {
                             const uint32_t a_step = (uint32_t)(a_sub >> 4), b_step = (uint32_t)(b_sub >> 4);
                             if (nt == 3 && ks == 2) {
@@ -892,7 +898,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                         if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
                     }
                 }
-                for (int part = 0; part < 2 && ok && p.tps == 1; ++part) {
+                for (int part = 0; part < 2 && ok && k_tps == 1; ++part) {
                     const int nb = part ? p.nb_hi : p.nb_lo;
                     if (nb == 0) continue;
                     const int ks_last = ((part ? p.C_hi : p.C_lo) - (nb - 1) * p.BK + 31) >> 5;
@@ -1178,15 +1184,15 @@ static int make_map_im2col(CUtensorMap *map, const void *base, int Cpart, long l
     return FLEXIQ_OK;
 }
 
-template <int CG, int PK>
+template <int CG, int PK, int KIND>
 static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const CUtensorMap &b_lo, const CUtensorMap &b_hi,
                          const CUtensorMap &y_map, const CUtensorMap &y_map16, const GemmParams &p, int sms, cudaStream_t st)
 {
-    static bool attr_set[64] = {};
+    static bool attr_set[64] = {};   // per instantiation
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 64 && !attr_set[dev]) {
-        FLEXIQ_CUDA_TRY(cudaFuncSetAttribute(mixed_gemm_kernel<CG, PK>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        FLEXIQ_CUDA_TRY(cudaFuncSetAttribute(mixed_gemm_kernel<CG, PK, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
         attr_set[dev] = true;
     }
     const long long tiles = (long long)p.m_tiles * p.n_tiles;
@@ -1206,7 +1212,7 @@ static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    FLEXIQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, mixed_gemm_kernel<CG, PK>, a_lo, a_hi, b_lo, b_hi, y_map, y_map16, p));
+    FLEXIQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, mixed_gemm_kernel<CG, PK, KIND>, a_lo, a_hi, b_lo, b_hi, y_map, y_map16, p));
     return FLEXIQ_OK;
 }
 
@@ -1394,9 +1400,13 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
         cm.staged = staged; cm.y_elem = y_elem; cm.a = a_hi; cm.y = y_map; cm.y16 = y_map16;
     }
     const int bi = weight_map_index(bn / cg);  // box rows = the B rows one CTA loads
-    if (packed) return launch_kernel<1, 1>(a_lo, a_hi, L->map_w4[bi], L->map_w8[bi], y_map, y_map16, p, sms, st);
-    if (cg == 2) return launch_kernel<2, 0>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], y_map, y_map16, p, sms, st);
-    return launch_kernel<1, 0>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], y_map, y_map16, p, sms, st);
+    const bool conv_kind = p.im2col || p.tps > 1 || p.b_res;
+    if (packed) return launch_kernel<1, 1, 1>(a_lo, a_hi, L->map_w4[bi], L->map_w8[bi], y_map, y_map16, p, sms, st);
+    if (cg == 2)
+        return conv_kind ? launch_kernel<2, 0, 1>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], y_map, y_map16, p, sms, st)
+                         : launch_kernel<2, 0, 0>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], y_map, y_map16, p, sms, st);
+    return conv_kind ? launch_kernel<1, 0, 1>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], y_map, y_map16, p, sms, st)
+                     : launch_kernel<1, 0, 0>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], y_map, y_map16, p, sms, st);
 }
 
 }  // namespace flexiq
