@@ -305,7 +305,7 @@ struct EpilogueCtx {
 // Per pass: fetch the columns' factors, read the whole slice of the accumulator into registers,
 // hand the accumulator back, then scale / round / clip; the results are staged in shared memory (32 rows
 // x 32 bytes: 32 int8, 16 half-precision or 8 four-byte columns) and leave through tiled bulk stores.
-template <int CG, int MODE>
+template <int CG, int MODE, bool SPLIT>
 __device__ __forceinline__ void epilogue_role(const GemmParams &p, const EpilogueCtx &x, int quad, int part, int lane)
 {
     constexpr bool kScaled = MODE != FLEXIQ_OUT_ACC_I32;
@@ -361,17 +361,22 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                 ptx::tc_fence_after_sync();
                 waited = true;
             }
-            const uint32_t taddr = x.tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)buf * x.buf_stride + (uint32_t)col0;
+            const uint32_t taddr = x.tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(SPLIT ? 2 * buf : buf) * x.buf_stride + (uint32_t)col0;
             PROF_T0(te0);
             uint32_t ra[32], rb[32];
             ptx::tmem_ld_32x32(taddr, ra);
-            if (cols == 64) ptx::tmem_ld_32x32(taddr + 32, rb);
+            if (SPLIT) ptx::tmem_ld_32x32(taddr + x.buf_stride, rb);   // the other MMA warp's partial sums (32-column passes only)
+            else if (cols == 64) ptx::tmem_ld_32x32(taddr + 32, rb);
             if (kScaled) {
                 __syncwarp();                                      // the previous reads of the table are done
                 reinterpret_cast<float4 *>(x.fac)[lane] = f;
                 __syncwarp();
             }
             ptx::tmem_ld_wait();
+            if (SPLIT) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) ra[i] += rb[i];
+            }
             PROF_ADD(prof_ld, te0);
             PROF_T0(te1);
             if (pass + 1 == passes) {
@@ -578,7 +583,12 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
 // KIND 0: linear layers and 1x1 convolutions (plain 2-D copies, one K block per stage); KIND 1: everything a
 // convolution may need (im2col copies, several taps per stage, resident weight tiles).  The issuing warps'
 // instruction streams are on the critical path of a tile, so the first kind carries none of the second's code.
-template <int CG, int PK, int KIND>
+// SPLIT (tiles of at most 128 columns, one K block per stage, at least two stages per tile): the two MMA warps
+// take the ring's stages in turn INSIDE a tile, each into an accumulator of its own, and the epilogue adds the
+// two: for narrow MMAs (64 cycles each) the issuing warp's bookkeeping, not the pipe, bounds a K block, and two
+// warps halve it.  No accumulator is shared, so no order between the warps' MMAs is needed; their waits on
+// the ring stay in ring order (one hand-over phase per stage).
+template <int CG, int PK, int KIND, bool SPLIT>
 __global__ void __launch_bounds__(kThreads, 1)
 mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_constant__ CUtensorMap mapA_hi,
                   const __grid_constant__ CUtensorMap mapB_lo, const __grid_constant__ CUtensorMap mapB_hi,
@@ -619,8 +629,9 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
     const uint32_t cta_rank = CG == 2 ? ptx::cluster_ctarank() : 0u;
     const bool leader = cta_rank == 0;
     const int first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
-    const uint32_t tmem_cols = BN <= 64 ? 128u : (BN <= 128 ? 256u : 512u);
-    const uint32_t buf_stride = tmem_cols / 2;  // column offset of the second accumulator
+    // two accumulators (tiles in turn); SPLIT: two per tile, four in all
+    const uint32_t buf_stride = BN <= 64 ? 64u : (BN <= 128 ? 128u : 256u);  // column offset from one accumulator to the next
+    const uint32_t tmem_cols = (SPLIT ? 4u : 2u) * buf_stride;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
@@ -628,7 +639,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             ptx::mbar_init(&empty_bar[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
-            ptx::mbar_init(&tmem_full[b], 1);
+            ptx::mbar_init(&tmem_full[b], SPLIT ? 2 : 1);   // SPLIT: both MMA warps commit a tile
             ptx::mbar_init(&tmem_empty[b], CG * kEpiWarps);
         }
         for (int r = 0; r < kRawStages; ++r) {
@@ -833,7 +844,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             const uint32_t full0 = ptx::smem_u32(full_bar);
             const int ks_full = p.BK >> 5;
             uint32_t stage = 0, phase = 0;
-            int buf = duo ? my : 0;
+            int buf = (duo && !SPLIT) ? my : 0;
             uint32_t buf_phase = 0;
             bool ok = true;
             PROF_DECL(prof_wait_acc);
@@ -843,7 +854,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             int ti = 0;                                          // index of the tile in this CTA's sequence
             TileWalk tw;
             for (tw.init(first_tile, tile_step, num_tiles, p.n_tiles); tw.left > 0 && ok; tw.next(), ++ti) {
-                if (duo && (ti & 1) != my) {
+                if (!SPLIT && duo && (ti & 1) != my) {
                     // the other warp's tile: step over its ring stages
                     stage += (uint32_t)tile_slots;
                     while (stage >= (uint32_t)p.stages) { stage -= (uint32_t)p.stages; phase ^= 1; }
@@ -854,9 +865,10 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                 if (!__all_sync(0xffffffffu, wait_bounded(&tmem_empty[buf], buf_phase ^ 1, abort_flag, 2))) break;
                 PROF_ADD(prof_wait_acc, t0);
                 // the other warp has passed the wait for the last stage of the tile before this one
-                if (duo && ti > 0 && !__all_sync(0xffffffffu, wait_bounded(turn_bar, (uint32_t)((ti - 1) & 1), abort_flag, 7))) break;
+                if (!SPLIT && duo && ti > 0 && !__all_sync(0xffffffffu, wait_bounded(turn_bar, (uint32_t)((ti - 1) & 1), abort_flag, 7))) break;
                 ptx::tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + (uint32_t)buf * buf_stride;
+                const uint32_t d_tmem = tmem_base + (uint32_t)(SPLIT ? 2 * buf + my : buf) * buf_stride;
+                const int g0 = ti * tile_slots;                  // SPLIT: number of this tile's first stage in the CTA's sequence
                 uint32_t acc = 0;
                 if (k_tps > 1) {
                     const int ks = (p.C + 31) >> 5;  // K steps of one tap (C <= BK)
@@ -904,10 +916,21 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                     const int ks_last = ((part ? p.C_hi : p.C_lo) - (nb - 1) * p.BK + 31) >> 5;
                     for (int tap = 0; tap < p.T && ok; ++tap) {
                         for (int cb = 0; cb < nb; ++cb) {
+                            if (SPLIT) {
+                                const int g = g0 + slot;
+                                if ((g & 1) != my) {   // the other warp's stage
+                                    ++slot;
+                                    if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
+                                    continue;
+                                }
+                                // the other warp has passed its wait for the stage before this one
+                                if (g > 0 && !__all_sync(0xffffffffu, wait_bounded(turn_bar, (uint32_t)((g - 1) & 1), abort_flag, 7))) { ok = false; break; }
+                            }
                             PROF_T0(t1);
                             if (!__all_sync(0xffffffffu, wait_bounded(full0 + 8 * stage, phase, abort_flag, 3))) { ok = false; break; }
                             PROF_ADD(prof_wait_full, t1);
-                            if (duo && ++slot == tile_slots && lane == 0) ptx::mbar_arrive(turn_bar);   // the other warp may go on
+                            if (SPLIT) { ++slot; if (lane == 0) ptx::mbar_arrive(turn_bar); }
+                            else if (duo && ++slot == tile_slots && lane == 0) ptx::mbar_arrive(turn_bar);   // the other warp may go on
                             const uint32_t a_lo = a_lo0 + stage * stage_step, b_lo = b_lo0 + stage * stage_step;
                             const int ks = cb == nb - 1 ? ks_last : ks_full;
                             if (ptx::elect_one()) {
@@ -934,8 +957,8 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                 }
                 if (ok && ptx::elect_one()) ptx::mma_commit_s<CG>(ptx::smem_u32(&tmem_full[buf]));
                 __syncwarp();
-                if (duo) buf_phase ^= 1;                         // this warp's accumulator again at its next tile
-                else if ((buf ^= 1) == 0) buf_phase ^= 1;
+                if (duo && !SPLIT) buf_phase ^= 1;               // this warp's accumulator again at its next tile
+                else if ((buf ^= 1) == 0) buf_phase ^= 1;        // SPLIT: buf counts the tile's pair of accumulators
             }
             if (my == 0) {
             PROF_STORE(4, prof_wait_acc);
@@ -957,12 +980,12 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             x.map_y = &mapY; x.map_y16 = &mapY16;
             x.first_tile = first_tile; x.tile_step = tile_step; x.num_tiles = num_tiles;
             x.parts = kEpiWarps / 4; x.arrivals_on = 1;
-            if (p.out_mode == FLEXIQ_OUT_REQUANT_I8) epilogue_role<CG, FLEXIQ_OUT_REQUANT_I8>(p, x, warp & 3, e >> 2, lane);
-            else if (p.out_mode == FLEXIQ_OUT_DEQUANT_F32) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_F32>(p, x, warp & 3, e >> 2, lane);
-            else if (p.out_mode == kOutNextSlab) epilogue_role<CG, kOutNextSlab>(p, x, warp & 3, e >> 2, lane);
-            else if (p.out_mode == FLEXIQ_OUT_DEQUANT_F16) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_F16>(p, x, warp & 3, e >> 2, lane);
-            else if (p.out_mode == FLEXIQ_OUT_DEQUANT_BF16) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_BF16>(p, x, warp & 3, e >> 2, lane);
-            else epilogue_role<CG, FLEXIQ_OUT_ACC_I32>(p, x, warp & 3, e >> 2, lane);
+            if (p.out_mode == FLEXIQ_OUT_REQUANT_I8) epilogue_role<CG, FLEXIQ_OUT_REQUANT_I8, SPLIT>(p, x, warp & 3, e >> 2, lane);
+            else if (p.out_mode == FLEXIQ_OUT_DEQUANT_F32) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_F32, SPLIT>(p, x, warp & 3, e >> 2, lane);
+            else if (p.out_mode == kOutNextSlab) epilogue_role<CG, kOutNextSlab, SPLIT>(p, x, warp & 3, e >> 2, lane);
+            else if (p.out_mode == FLEXIQ_OUT_DEQUANT_F16) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_F16, SPLIT>(p, x, warp & 3, e >> 2, lane);
+            else if (p.out_mode == FLEXIQ_OUT_DEQUANT_BF16) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_BF16, SPLIT>(p, x, warp & 3, e >> 2, lane);
+            else epilogue_role<CG, FLEXIQ_OUT_ACC_I32, SPLIT>(p, x, warp & 3, e >> 2, lane);
         } else if (PK && warp < 2 + kNumWorkWarps) {
             // --------------------------------------------------------- expanders (packed path)
             // Widen each raw 4-bit tile into the operand ring: 8 packed bytes -> one 16-byte unit
@@ -1184,7 +1207,7 @@ static int make_map_im2col(CUtensorMap *map, const void *base, int Cpart, long l
     return FLEXIQ_OK;
 }
 
-template <int CG, int PK, int KIND>
+template <int CG, int PK, int KIND, bool SPLIT>
 static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const CUtensorMap &b_lo, const CUtensorMap &b_hi,
                          const CUtensorMap &y_map, const CUtensorMap &y_map16, const GemmParams &p, int sms, cudaStream_t st)
 {
@@ -1192,7 +1215,7 @@ static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 64 && !attr_set[dev]) {
-        FLEXIQ_CUDA_TRY(cudaFuncSetAttribute(mixed_gemm_kernel<CG, PK, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+        FLEXIQ_CUDA_TRY(cudaFuncSetAttribute(mixed_gemm_kernel<CG, PK, KIND, SPLIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
         attr_set[dev] = true;
     }
     const long long tiles = (long long)p.m_tiles * p.n_tiles;
@@ -1212,7 +1235,7 @@ static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    FLEXIQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, mixed_gemm_kernel<CG, PK, KIND>, a_lo, a_hi, b_lo, b_hi, y_map, y_map16, p));
+    FLEXIQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, mixed_gemm_kernel<CG, PK, KIND, SPLIT>, a_lo, a_hi, b_lo, b_hi, y_map, y_map16, p));
     return FLEXIQ_OK;
 }
 
@@ -1401,12 +1424,20 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     }
     const int bi = weight_map_index(bn / cg);  // box rows = the B rows one CTA loads
     const bool conv_kind = p.im2col || p.tps > 1 || p.b_res;
-    if (packed) return launch_kernel<1, 1, 1>(a_lo, a_hi, L->map_w4[bi], L->map_w8[bi], y_map, y_map16, p, sms, st);
-    if (cg == 2)
-        return conv_kind ? launch_kernel<2, 0, 1>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], y_map, y_map16, p, sms, st)
-                         : launch_kernel<2, 0, 0>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], y_map, y_map16, p, sms, st);
-    return conv_kind ? launch_kernel<1, 0, 1>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], y_map, y_map16, p, sms, st)
-                     : launch_kernel<1, 0, 0>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], y_map, y_map16, p, sms, st);
+    // One narrow tile per CTA and a long K: nothing overlaps across tiles, so the MMA warps share the tile
+    // (SPLIT).  With several tiles per CTA the warps already work side by side on tiles of their own, and the
+    // second accumulator's extra read in the epilogue would only cost (measured: +4 to +6 % on short-K shapes).
+    const bool split = !packed && bn <= 128 && p.tps == 1 && p.T * (p.nb_lo + p.nb_hi) >= 8 &&
+                       (long long)p.m_tiles * p.n_tiles <= sms / cg;
+    if (packed) return launch_kernel<1, 1, 1, false>(a_lo, a_hi, L->map_w4[bi], L->map_w8[bi], y_map, y_map16, p, sms, st);
+#define FLEXIQ_LAUNCH(CG_, KIND_, SPLIT_) launch_kernel<CG_, 0, KIND_, SPLIT_>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], y_map, y_map16, p, sms, st)
+    if (cg == 2) {
+        if (conv_kind) return split ? FLEXIQ_LAUNCH(2, 1, true) : FLEXIQ_LAUNCH(2, 1, false);
+        return split ? FLEXIQ_LAUNCH(2, 0, true) : FLEXIQ_LAUNCH(2, 0, false);
+    }
+    if (conv_kind) return split ? FLEXIQ_LAUNCH(1, 1, true) : FLEXIQ_LAUNCH(1, 1, false);
+    return split ? FLEXIQ_LAUNCH(1, 0, true) : FLEXIQ_LAUNCH(1, 0, false);
+#undef FLEXIQ_LAUNCH
 }
 
 }  // namespace flexiq

@@ -71,3 +71,32 @@ def test_random_conv(dev, seed):
         assert np.all(np.abs(got - exp) <= 1e-6 * np.abs(exp))
     L.close()
     fx.flexiq_check_status()
+
+
+@pytest.mark.parametrize("tile", [(0, 0), (1, 64), (1, 128), (2, 128)])
+@pytest.mark.parametrize("M,K,N,G", [(1, 1296, 176, 16), (300, 2304, 96, 64), (700, 1056, 240, 32)])
+def test_one_long_k_tile_per_cta(dev, tile, M, K, N, G):
+    """Few narrow tiles and many K blocks: each CTA has one tile, and its two MMA warps share the tile's K
+    blocks into accumulators of their own, which the epilogue adds.  Every output mode reads both."""
+    case = inputs.ranged_linear("s", M, K, N, G, seed=K + N, group_structured=True)
+    perm, sxg, sxs, sw = helpers.prepare_linear(case)
+    q = oracle.quantize(case.X, case.x_scale)
+    X = torch.from_numpy(case.X).to(dev)
+    L = fx.Layer(torch.from_numpy(case.Wq).to(dev), torch.from_numpy(case.w_scale).to(dev), torch.from_numpy(case.bias).to(dev), perm, sxg, G)
+    fx.flexiq_force_tile(*tile)
+    try:
+        for ratio in (0.0, 0.5, 1.0):
+            L.set_lowbit_ratio(ratio)
+            x4, x8, _ = L.quantize_lower(X, case.x_scale)
+            acc = oracle.mixed_gemm_acc(q, case.Wq, G, perm, sxs, sw, oracle.n_low(ratio, K // G))
+            assert np.array_equal(L.mixed_gemm(x4, x8, M, case.x_scale, case.y_scale, fx.OUT_ACC_I32).cpu().numpy(), acc)
+            assert np.array_equal(L.mixed_gemm(x4, x8, M, case.x_scale, case.y_scale, fx.OUT_REQUANT_I8).cpu().numpy(),
+                                  oracle.epilogue_i8(acc, case.x_scale, case.w_scale, case.bias, case.y_scale))
+            assert np.array_equal(L.mixed_gemm(x4, x8, M, case.x_scale, case.y_scale, fx.OUT_DEQUANT_F32).cpu().numpy(),
+                                  oracle.epilogue_f32(acc, case.x_scale, case.w_scale, case.bias))
+            y16 = L.mixed_gemm(x4, x8, M, case.x_scale, case.y_scale, fx.OUT_DEQUANT_F16).cpu().numpy()
+            assert np.array_equal(y16.view(np.uint16), oracle.epilogue_f16(acc, case.x_scale, case.w_scale, case.bias).view(np.uint16))
+    finally:
+        fx.flexiq_force_tile(0, 0)
+    L.close()
+    fx.flexiq_check_status()
