@@ -14,7 +14,9 @@
 //                results staged in shared memory 32 rows x 32 bytes at a time and written by tiled bulk
 //                stores (the fused boundary in original channel order scatters 16-byte chunks directly);
 //                on the packed path eight of them widen 4-bit tiles instead
-// Two TMEM accumulators let the epilogue of tile i overlap the mainloop of tile i+1.
+// Two TMEM accumulators let the epilogue of tile i overlap the mainloop of tile i+1.  Launches of one narrow,
+// long-K tile per CTA instead let the two MMA warps share the tile's K blocks (an accumulator each, summed
+// in the epilogue).
 // Every wait is bounded; an expired wait raises the status word and the CTA drains.
 #include "flexiq_internal.h"
 
