@@ -79,7 +79,8 @@ def _chain_linear(dev, M, K, N1, N2, G1, G2, ratios, relu, seed):
 
 @pytest.mark.parametrize("M,K,N1,N2,G1,G2,relu", [(300, 256, 272, 48, 16, 16, False), (129, 128, 64, 32, 16, 32, True),
                                                   (1000, 384, 1024, 80, 16, 64, False), (1, 64, 16, 16, 16, 16, True),
-                                                  (515, 192, 400, 64, 32, 16, True)])
+                                                  (515, 192, 400, 64, 32, 16, True),
+                                                  (260, 1280, 112, 48, 16, 16, False)])   # one long-K tile per CTA
 def test_linear_chain(dev, M, K, N1, N2, G1, G2, relu):
     _chain_linear(dev, M, K, N1, N2, G1, G2, [(0.0, 0.0), (0.5, 0.5), (1.0, 0.25), (0.25, 1.0)], relu, seed=M + N1)
 
