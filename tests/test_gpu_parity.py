@@ -253,6 +253,13 @@ def test_resnet50_conv_full_size_56(dev):
     _run_conv(case, dev, [0.0, 0.5, 1.0])
 
 
+def test_resnet50_conv_full_size_7(dev):
+    # 3x3, 512 -> 512 channels at 7x7, batch 32 as the sweep times it: 104 tiles, one per CTA, the two MMA
+    # warps sharing each tile's 36 K blocks
+    case = inputs.resnet_conv("c7", 32, 7, 512, 512, 3, seed=3007)
+    _run_conv(case, dev, [0.5])
+
+
 # ---------------------------------------------------------------- packed 4-bit slabs
 @pytest.mark.parametrize("M,K,N,G", [(300, 384, 272, 16), (129, 256, 48, 32), (1000, 1024, 400, 16), (257, 64, 64, 16),
                                      (700, 192, 512, 64)])
