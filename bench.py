@@ -247,6 +247,7 @@ def run_ours(args):
             "gemm_ms": round(ms_r, 4),
             "gemm_tops": round(sum(layer_ops(c) for c in cases) / (ms_r * 1e-3) / 1e12, 1),
             "gemm_gbs": round(sum(gemm_algorithmic_bytes(c, r) for c in cases) / (ms_r * 1e-3) / 1e9, 1),
+            "frac_of_peak": round(sum(layer_ops(c) for c in cases) / (ms_r * 1e-3) / 1e12 / int8_peak, 4),
         }
     traffic = None
     tpath = os.path.join(ROOT, "profiles", "mixed_gemm_vitb_dram_traffic.json")
