@@ -315,6 +315,7 @@ def run_ours(args):
                      "avg_launch_us": round(total_gemm_ms * 1e3 / (len(RATIOS) * len(cases)), 2),
                      "peak_note": f"2 x sustained bf16 cuBLAS ({peaks['source']}); burst-based peak {2 * peaks['bf16_burst']:.0f}; nominal 4500"},
         "per_ratio": per_ratio,
+        "gemm_time_non_increasing_in_ratio_within_2pct": all(group_ms[i + 1] <= 1.02 * group_ms[i] for i in range(len(RATIOS) - 1)),
         "e2e": {"value": round(e2e_tops, 2), "unit": "TOPS", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps},
         "gpu_launches": args.steps * len(RATIOS) * len(cases) * 2,
         "clocks": clocks,
