@@ -273,20 +273,24 @@ __device__ __forceinline__ void st_global_256(void *p, const uint32_t *w)
 }
 
 // Eight packed bytes (16 two's-complement nibbles, channel 2t in bits 0-3 of byte t) -> 16 int8
-// values (nibble << s), as four little-endian words.  Nibbles are spread to bytes with two
-// byte permutes per word; the sign extension ORs in bits s+4..7 where bit 3 of the nibble is set.
+// values (nibble << s), as four little-endian words.  A nibble n moved to the high half of a byte is the
+// int8 value 16 n, and n << s is that byte shifted right arithmetically by 4 - s: a logical shift of the
+// whole word (the low halves are zero, so nothing crosses a byte) plus the sign, replicated over each byte
+// by a byte permute, in the vacated top bits.
 __device__ __forceinline__ void unpack16(uint32_t w0, uint32_t w1, int s, uint32_t out[4])
 {
-    const uint32_t k = (16u >> s) - 1u;
+    const uint32_t r = 4u - (uint32_t)s;
+    const uint32_t top = 0x01010101u * ((0xff00u >> r) & 0xffu);   // the top r bits of every byte
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         const uint32_t w = h == 0 ? w0 : w1;
-        const uint32_t e = w & 0x0f0f0f0fu, o = (w >> 4) & 0x0f0f0f0fu;  // even / odd nibbles, one per byte
+        const uint32_t e = (w << 4) & 0xf0f0f0f0u, o = w & 0xf0f0f0f0u;  // even / odd nibbles, each in the high half of a byte
         const uint32_t x[2] = {__byte_perm(e, o, 0x5140), __byte_perm(e, o, 0x7362)};  // channel order
 #pragma unroll
         for (int q = 0; q < 2; ++q) {
-            const uint32_t fill = (((x[q] & 0x08080808u) << (s + 1)) & 0xf0f0f0f0u) * k;
-            out[2 * h + q] = (x[q] << s) | fill;
+            uint32_t sign;
+            asm("prmt.b32 %0, %1, 0, 0xba98;" : "=r"(sign) : "r"(x[q]));   // 0xff where the byte is negative
+            out[2 * h + q] = (x[q] >> r) | (sign & top);
         }
     }
 }
@@ -1014,22 +1018,37 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             for (tw.init(first_tile, tile_step, num_tiles, p.n_tiles); tw.left > 0 && ok; tw.next()) {
                 const int n0 = tw.n_blk * BN;
                 const bool liveB = hasB && n0 + rowB < p.N;
+                const int colB = liveB ? n0 + rowB : 0;      // a valid column of the position table for every thread
                 for (int part = 0; part < 2 && ok; ++part) {
                     const int nb = part ? p.nb_hi : p.nb_lo;
                     for (int tap = 0; tap < p.T && ok; ++tap) {
+                        // The positions of a K block's chunks come from global memory (the 221 KB of shared memory
+                        // leave almost no L1, so every fetch goes to L2): those of block cb + 1 are requested before
+                        // block cb is widened.  The requests are unconditional (clamped indices); what a thread does
+                        // not own is zeroed when the values are taken over.
+                        int nxB[8], nxA[4];
+                        const int last_chunk = (p.C_lo >> 4) - 1;
+                        auto request = [&](int cb) {
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) {
+                                const int chunk = min(cb * upr + (u < upr ? u : 0), last_chunk);
+                                nxB[u] = __ldg(p.sw + (size_t)(chunk >> cpg_log2) * p.N + colB);
+                            }
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const int chunk = min(cb * upr + uA0 + (k < (upr >> 1) ? k : 0), last_chunk);
+                                nxA[k] = __ldg(p.sx + (chunk >> cpg_log2));
+                            }
+                        };
+                        if (part == 0 && nb > 0) request(0);
                         for (int cb = 0; cb < nb; ++cb) {
                             if (part == 0) {
                                 int shB[8], shA[4];
 #pragma unroll
-                                for (int u = 0; u < 8; ++u) {
-                                    const int chunk = cb * upr + u;       // 16-channel chunk of the low slab
-                                    shB[u] = (u < upr && liveB && chunk * 16 < p.C_lo) ? __ldg(p.sw + (size_t)(chunk >> cpg_log2) * p.N + n0 + rowB) : 0;
-                                }
+                                for (int u = 0; u < 8; ++u) shB[u] = (u < upr && liveB && (cb * upr + u) * 16 < p.C_lo) ? nxB[u] : 0;
 #pragma unroll
-                                for (int k = 0; k < 4; ++k) {
-                                    const int chunk = cb * upr + uA0 + k;
-                                    shA[k] = (k < (upr >> 1) && chunk * 16 < p.C_lo) ? __ldg(p.sx + (chunk >> cpg_log2)) : 0;
-                                }
+                                for (int k = 0; k < 4; ++k) shA[k] = (k < (upr >> 1) && (cb * upr + uA0 + k) * 16 < p.C_lo) ? nxA[k] : 0;
+                                if (cb + 1 < nb) request(cb + 1);
                                 PROF_T0(tx0);
                                 bool w1 = wait_bounded(&raw_full[rstage], rphase, abort_flag, 6);
                                 PROF_ADD(prof_x_raw, tx0);
@@ -1323,8 +1342,9 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
             long long best = -1;
             const int bns[4] = {256, 192, 128, 64};
             for (int i = 0; i < 4; ++i) {
+                // the expander warps widen the tile's 128 + BN rows for every K block: that, not the MMAs, is a tile's time
                 const long long tiles = mt * ((L->N + bns[i] - 1) / bns[i]);
-                const long long cost = ((tiles + sms - 1) / sms) * bns[i];
+                const long long cost = ((tiles + sms - 1) / sms) * (BM + bns[i]);
                 if (best < 0 || cost < best) { best = cost; tc.bn = bns[i]; }
             }
         }
