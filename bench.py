@@ -309,7 +309,7 @@ def run_ours(args):
         "config": {"workload": WORKLOAD, "ratios": RATIOS, "l2": "working set per step (271 MB fp32 inputs + slabs + outputs) exceeds the 126 MB L2; no flush needed",
                    "lowbit_path": "masked_i8", "launch": "CUDA graph replay" if use_graph else "host launches"},
         "roofline": {"bound": "tensor", "achieved": round(achieved, 1), "peak": round(int8_peak, 1), "unit": "TOPS",
-                     "frac": round(achieved / int8_peak, 4), "traffic": traffic,
+                     "frac": round(achieved / int8_peak, 4), "traffic": None if traffic is None else int(round(traffic)),
                      "kernel": "mixed_gemm_kernel (all 20 launches of a step)",
                      "timing": "second pass: per ratio, rounds of the 4 GEMM launches alone inside one CUDA-event pair (ratios visited up then down, K/2 rounds each way); avg launch = total time / launches",
                      "avg_launch_us": round(total_gemm_ms * 1e3 / (len(RATIOS) * len(cases)), 2),
