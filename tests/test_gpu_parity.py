@@ -337,6 +337,69 @@ def test_vit_l_full_size_sampled_rows(dev):
     L.close()
 
 
+def test_rows_beyond_32_bit_byte_offsets(dev):
+    """M * K and M * N above 2^32 bytes (4.4 million rows of 1024 channels).  The int8 input is a seeded block
+    of 50,000 rows repeated -- a period that does not divide 2^32, so an offset that wrapped at 32 bits would
+    land on other rows.  Every slab and output row must equal the row one period earlier (checked on the device
+    for all rows); sampled rows of the first period, the rows around the 2^32-byte mark and the last rows equal
+    the oracle's."""
+    K, N, G, P = 1024, 1024, 16, 50_000
+    M = 88 * P + 12_345
+    case = inputs.vit_linear("big", P, K, N, G, seed=7000)
+    perm, sxg, sxs, sw = helpers.prepare_linear(case)
+    q = oracle.quantize(case.X, case.x_scale)
+    L = _layer(case, dev, perm, sxg)
+    X = torch.from_numpy(q).to(dev).repeat(89, 1)[:M]
+    assert X.is_contiguous() and M * K > 2 ** 32
+    L.set_lowbit_ratio(0.5)
+    nl = oracle.n_low(0.5, K // G)
+    x4, x8, _ = L.quantize_lower(X, case.x_scale)
+    y8 = L.mixed_gemm(x4, x8, M, case.x_scale, case.y_scale, fx.OUT_REQUANT_I8)
+    torch.cuda.synchronize()
+    fx.flexiq_check_status()
+    slab = x4.view(torch.int8)[:M * K].view(M, K)
+    for i in range(1, 89):
+        n = min(P, M - i * P)
+        assert torch.equal(y8[i * P:i * P + n], y8[:n]), f"output rows of period {i}"
+        assert torch.equal(slab[i * P:i * P + n], slab[:n]), f"slab rows of period {i}"
+    mark = 2 ** 32 // K
+    rows = np.unique(np.concatenate([np.arange(0, P, 197), np.arange(mark - 6, mark + 6), np.arange(M - 40, M)])).astype(np.int64)
+    acc_e = oracle.mixed_gemm_acc(q[rows % P], case.Wq, G, perm, sxs, sw, nl)
+    got = y8[torch.from_numpy(rows).to(dev)].cpu().numpy()
+    assert np.array_equal(got, oracle.epilogue_i8(acc_e, case.x_scale, case.w_scale, case.bias, case.y_scale))
+    L.close()
+
+
+def test_conv_beyond_32_bit_byte_offsets(dev):
+    """The same for the convolution path: 22,000 images of 56 x 56 x 64 (4.4 GB in, 4.4 GB out), a seeded block
+    of 7 images repeated (1,404,928 bytes: not a divisor of 2^32).  Every output image equals the image one
+    period earlier; the first period, the images around the 2^32-byte mark and the last ones equal the oracle's."""
+    Pd, Nb = 7, 22_000
+    case = inputs.resnet_conv("bigc", Pd, 56, 64, 64, 3, seed=7100)
+    perm, sxg, sxs, sw = helpers.prepare_conv(case)
+    q = oracle.quantize(case.X, case.x_scale)                      # [7][56][56][64] int8
+    L = _layer(case, dev, perm, sxg, conv=True)
+    X = torch.from_numpy(q).to(dev).repeat(Nb // Pd + 1, 1, 1, 1)[:Nb]
+    assert X.is_contiguous() and X.numel() > 2 ** 32
+    L.set_lowbit_ratio(0.5)
+    nl = oracle.n_low(0.5, case.C // case.G)
+    x4, x8, _ = L.quantize_lower(X, case.x_scale)
+    y = L.mixed_conv(x4, x8, Nb, case.H, case.W, case.x_scale, case.y_scale, fx.OUT_REQUANT_I8)
+    torch.cuda.synchronize()
+    fx.flexiq_check_status()
+    assert y.shape[0] == Nb and y.numel() > 2 ** 32
+    for i in range(1, Nb // Pd + 1):
+        n = min(Pd, Nb - i * Pd)
+        if n > 0:
+            assert torch.equal(y[i * Pd:i * Pd + n], y[:n]), f"images of period {i}"
+    acc_e = oracle.mixed_conv_acc(q, case.Wq, case.stride, case.pad, case.G, perm, sxs, sw, nl)
+    want = oracle.epilogue_i8(acc_e, case.x_scale, case.w_scale, case.bias, case.y_scale).reshape(Pd, *y.shape[1:])
+    mark = 2 ** 32 // (56 * 56 * 64)
+    for img in list(range(Pd)) + list(range(mark - 2, mark + 3)) + list(range(Nb - 3, Nb)):
+        assert np.array_equal(y[img].cpu().numpy(), want[img % Pd]), f"image {img}"
+    L.close()
+
+
 @pytest.mark.parametrize("K", [240, 256, 1024])
 def test_extreme_accumulators(dev, K):
     """The largest accumulator magnitudes a layer can produce (all operands at -128 / 127) survive the
