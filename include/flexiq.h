@@ -407,6 +407,11 @@ int flexiq_layer_export(flexiq_layer_t layer, uint8_t *sw_host, int8_t *w8_host,
  * tile_n >= 128).  cta_group 0 restores the automatic choice.  The paper has no counterpart. */
 int flexiq_force_tile(int cta_group, int tile_n);
 
+/* Test hook, host-only (no GPU needed): the tile shape the automatic choice takes for a masked-path layer of
+ * M rows, N output channels and k_blocks K blocks of block_k (128 or 64) bytes per tile on a GPU of sm_count
+ * SMs.  Writes the CTAs per tile (1 or 2) and the tile width.  The paper has no counterpart. */
+int flexiq_choose_tile(int64_t M, int N, int k_blocks, int block_k, int sm_count, int *cta_group_out, int *tile_n_out);
+
 /* Reads and clears the device status word raised by a bounded wait that expired.
  * Synchronises `stream`. */
 int flexiq_check_status(void *stream);

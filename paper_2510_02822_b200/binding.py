@@ -30,7 +30,7 @@ EXPORTS = [
     "flexiq_calib_weight_absmax", "flexiq_calib_prepare", "flexiq_calib_absmax_ema",
     "flexiq_controller_create", "flexiq_controller_destroy", "flexiq_controller_level", "flexiq_controller_update",
     "flexiq_serving_simulate", "flexiq_evo_init", "flexiq_evo_next_generation", "flexiq_sq_distance_i8",
-    "flexiq_layer_export", "flexiq_force_tile", "flexiq_check_status", "flexiq_last_error",
+    "flexiq_layer_export", "flexiq_force_tile", "flexiq_choose_tile", "flexiq_check_status", "flexiq_last_error",
 ]
 
 _lib = None
@@ -232,6 +232,13 @@ def flexiq_layer_export(h, sw_host=None, w8_host=None, w4_host=None):
 
 def flexiq_force_tile(cta_group, tile_n):
     _check(lib().flexiq_force_tile(cta_group, tile_n))
+
+
+def flexiq_choose_tile(M, N, k_blocks, block_k=128, sm_count=148):
+    """(CTAs per tile, tile width) of the automatic choice; host-only."""
+    cg, bn = C.c_int(0), C.c_int(0)
+    _check(lib().flexiq_choose_tile(C.c_int64(M), N, k_blocks, block_k, sm_count, C.byref(cg), C.byref(bn)))
+    return cg.value, bn.value
 
 
 def flexiq_check_status():

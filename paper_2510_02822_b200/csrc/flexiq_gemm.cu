@@ -1530,6 +1530,16 @@ extern "C" int flexiq_profile_counters(long long *out16)
 }
 #endif
 
+extern "C" int flexiq_choose_tile(int64_t M, int N, int k_blocks, int block_k, int sm_count, int *cta_group_out, int *tile_n_out)
+{
+    if (M <= 0 || N <= 0 || k_blocks <= 0 || sm_count <= 0 || (block_k != 128 && block_k != 64) || !cta_group_out || !tile_n_out)
+        return set_error(FLEXIQ_ERR_INVALID_ARG, "flexiq_choose_tile: M, N, k_blocks and sm_count must be positive, block_k 128 or 64, outputs non-NULL");
+    const TileChoice tc = choose_tile(M, N, k_blocks, block_k, sm_count);
+    *cta_group_out = tc.cg;
+    *tile_n_out = tc.bn;
+    return FLEXIQ_OK;
+}
+
 extern "C" int flexiq_force_tile(int cta_group, int tile_n)
 {
     if (cta_group == 0) { g_forced_tile = TileChoice{0, 0}; return FLEXIQ_OK; }

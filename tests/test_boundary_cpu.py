@@ -100,3 +100,24 @@ def test_inputs_are_seeded_and_shaped():
     assert abs(z.mean()) < 0.05 and abs(z.std() - 1) < 0.05
     v = inputs.vit_linear("v", 32, 768, 64, seed=5)
     assert 20 <= v.meta["outlier_channels"] <= 60  # about 5 % of 768
+
+
+def test_tile_choice_host_logic(lib):
+    """The automatic tile shape (host-only hook): what the benchmark's four ViT-B layers get on 148 SMs, and
+    properties that hold for every shape."""
+    M = 64 * 197
+    assert fx.flexiq_choose_tile(M, 2304, 6) == (2, 256)      # QKV: CTA pairs, 256 x 256
+    assert fx.flexiq_choose_tile(M, 3072, 6) == (2, 256)      # fc1
+    assert fx.flexiq_choose_tile(M, 768, 24) == (2, 192)      # fc2: 200 pair tiles fill three waves better than 150
+    assert fx.flexiq_choose_tile(M, 768, 6) == (1, 192)       # proj
+    rng = np.random.default_rng(5)
+    for _ in range(300):
+        m, n = int(rng.integers(1, 40000)), 16 * int(rng.integers(1, 300))
+        kb, bk, sms = int(rng.integers(1, 40)), int(rng.choice([64, 128])), int(rng.choice([74, 132, 148]))
+        cg, bn = fx.flexiq_choose_tile(m, n, kb, bk, sms)
+        assert cg in (1, 2) and bn in (64, 128, 192, 256)
+        assert not (cg == 2 and bn < 128)
+        assert (cg, bn) == fx.flexiq_choose_tile(m, n, kb, bk, sms)      # a pure function of its arguments
+    for bad in [(0, 64, 1, 128, 148), (5, 0, 1, 128, 148), (5, 64, 0, 128, 148), (5, 64, 1, 96, 148), (5, 64, 1, 128, 0)]:
+        with pytest.raises(fx.FlexiqError):
+            fx.flexiq_choose_tile(*bad)
