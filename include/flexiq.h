@@ -252,20 +252,20 @@ int flexiq_mixed_conv_to_slab(flexiq_layer_t layer, const uint8_t *X4_dev, const
 /* ---- Calibration on the device (off the hot path; produces what flexiq_layer_create_* takes) ----
  *
  * flexiq_calib_channel_ranges: per input channel the range [lo, hi] (lo <= 0 <= hi) of the
- *   Eq. 1-quantized calibration activations X_dev [M][K] ("estimating the value ranges of the
- *   activation channels using sampled calibration data", Sec. 4.2).  accumulate != 0 merges into
+ *   Eq. 1-quantized calibration activations X_dev [M][K] (Sec. 4.2 takes the channels' ranges
+ *   from a sample of calibration data).  accumulate != 0 merges into
  *   the ranges already in lo_dev / hi_dev (several calibration batches); 0 starts from [0, 0].
  *   lo_dev, hi_dev: [K] int32.  K % 16 == 0.
  * flexiq_calib_channel_histogram / flexiq_calib_ranges_from_histogram: ranges that cover a given
- *   share of each channel's values instead of all of them (Sec. 8.4 presumes ranges "to cover 99 %
- *   of neuron values for each channel").  The first counts the Eq. 1-quantized values per channel,
+ *   share of each channel's values instead of all of them (Sec. 8.4 presumes ranges holding 99 % of a
+ *   channel's values).  The first counts the Eq. 1-quantized values per channel,
  *   hist_dev [K][256] uint32 with bin q + 128 (accumulate as above); the second drops at most `tail`
  *   samples from each end of every channel's histogram -- the caller passes
  *   tail = floor(n * (1 - coverage) / 2) for n samples per channel -- and widens the result to
  *   contain zero.  tail = 0 gives the exact ranges of flexiq_calib_channel_ranges.
  * flexiq_calib_weight_absmax: wmax_dev[k] = max |w| over the output channels (and taps) of input
- *   channel k ("the corresponding weight parameters' channels across the output channel dimension
- *   to determine the maximum value range", Sec. 4.2).  Linear: Wq_dev [K][N], taps ignored;
+ *   channel k (Sec. 4.2 pairs an activation channel with the widest range of its weights over the
+ *   output channels).  Linear: Wq_dev [K][N], taps ignored;
  *   convolution (is_conv != 0): Wq_dev [N][taps][K].
  * flexiq_calib_prepare: from those three tables, per channel group of group_size channels
  *     x_shift_dev[g]  static extraction position of ORIGINAL group g: that of its widest channel
@@ -366,7 +366,7 @@ int flexiq_serving_simulate(flexiq_controller_t ctrl, int fixed_level, int64_t n
  * the 8-bit model's (flexiq_sq_distance_i8); smaller is fitter.
  *
  * Randomness is counter based (splitmix64 finaliser over seed, generation, individual, draw index),
- * so a run is reproducible from `seed`.  Probabilities "inversely proportional to the score" are the
+ * so a run is reproducible from `seed`.  Draws that should favour low scores (Sec. 4.2) use the
  * integer weights 2^32 / (1 + score); a flag to clear is drawn with weight 1 + score.
  *
  * flexiq_evo_init: population_host [N][total] receives the seeds: chromosome 0 is the greedy

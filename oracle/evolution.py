@@ -17,7 +17,7 @@ random ones that prefer low scores.
 Readings where the text is silent (each is also listed in the design notes):
   * randomness: a counter-based generator, draw(seed, generation, individual, n) = splitmix64
     finaliser of a mix of the four counters; every decision below says which draw it takes;
-  * "probability inversely proportional to the score": integer weight 2^32 // (1 + score);
+  * draws that favour low error scores (Sec. 4.2): integer weight 2^32 // (1 + score);
     a flag to CLEAR in a repair is drawn with weight 1 + score; weighted draws walk the
     candidates in index order with value = draw % total weight;
   * parents of a pair: two independent draws among the r fittest (they may coincide); the

@@ -20,8 +20,12 @@
  *                         masked-operand closed form, brute-force dot products.
  *   fqo_mixed_conv_acc    equals the GEMM on an explicit im2col matrix; ratio 0 equals a
  *                         float64 convolution of the int8 tensors.
- *   fqo_epilogue_*        the paper gives no epilogue formula: "parity unpinned"; pinned
- *                         only at alpha = 1, beta = 0 and at hand-computed ties.
+ *   fqo_weight_*_conv     brute force over every tap per (group, output channel): no weight
+ *                         saturates and one position less would; 1x1 equals the linear tables.
+ *   fqo_epilogue_*        the paper gives no epilogue formula, so the FORM (which factors, in
+ *                         which association) is a reading: "parity unpinned" by the paper.  The
+ *                         arithmetic of that form is pinned: exact rational arithmetic on the
+ *                         fp32 factors rounded once, at general scales and next to ties.
  */
 #include <math.h>
 #include <stdint.h>
@@ -92,8 +96,8 @@ void fqo_channel_ranges(const int8_t *qcal, int64_t Mc, int K, int32_t *lo, int3
 }
 
 /* Static activation position of every ORIGINAL channel group g (G consecutive channels):
- * the group's position is that of its widest channel (Sec. 7: "the group's bit
- * extraction position"). */
+ * the group's position is that of its widest channel (Sec. 7 speaks of one extraction
+ * position per group). */
 void fqo_static_positions(const int32_t *lo, const int32_t *hi, int K, int G, uint8_t *sx_group)
 {
     for (int g = 0; g < K / G; ++g) {
@@ -235,7 +239,7 @@ void fqo_dynamic_positions(const int8_t *q, int64_t M, int K, int G, const int32
 
 /* ------------------------------------------------------------------ Sec. 4.1, Fig. 3
  * Bit-lowering: shift the 8-bit value right by the extraction position (arithmetic
- * shift: "shifting and storing low four bits"; both worked examples are floors) and keep
+ * shift: Sec. 4.1 describes a shift followed by keeping four bits; both worked examples are floors) and keep
  * four bits.  A value outside the range the static position was chosen for saturates
  * (the paper calls such channels saturated) instead of wrapping: clamp to [-8, 7]. */
 int fqo_floor_shift(int v, int s)
@@ -449,8 +453,7 @@ void fqo_reorder_channels(const uint8_t *x, int64_t M, int K, int G, int elem_by
             }
 }
 
-/* Coverage-based channel ranges (Sec. 8.4: ranges presumed "to cover 99 % of neuron values for each
- * channel"): hist[c][q + 128] counts the quantized values of channel c; the range drops at most `tail`
+/* Coverage-based channel ranges (Sec. 8.4 presumes ranges that hold 99 % of a channel's values): hist[c][q + 128] counts the quantized values of channel c; the range drops at most `tail`
  * samples from each end (tail = floor(n * (1 - coverage) / 2) for n samples) and is widened to contain
  * zero.  tail = 0 is the exact min / max of fqo_channel_ranges. */
 void fqo_channel_histogram(const int8_t *q, int64_t M, int K, uint32_t *hist /*[K][256]*/)
@@ -474,8 +477,7 @@ void fqo_ranges_from_histogram(const uint32_t *hist, int K, int64_t tail, int32_
 }
 
 /* Unused-bit statistics (Sec. 8.4): an int8 value has 7 magnitude bits; a channel whose range needs
- * L of them leaves 7 - L unused ("maximum is less than 32 => the highest two bits are not used",
- * Sec. 4.1).  hist[u] counts the channels with u unused bits, u = 4 standing for four or more. */
+ * L of them leaves 7 - L unused (Sec. 4.1's example: values below 32 leave the top two unused).  hist[u] counts the channels with u unused bits, u = 4 standing for four or more. */
 void fqo_unused_bits_histogram(const int32_t *lo, const int32_t *hi, int K, int32_t *hist /*[5]*/)
 {
     for (int u = 0; u < 5; ++u) hist[u] = 0;

@@ -475,3 +475,155 @@ def test_epilogue_half_precision_roundings():
     assert np.array_equal(oracle.epilogue_f16(acc_r, 3.1e-4, wsr, br), torch.from_numpy(f).to(torch.float16).numpy())
     assert np.array_equal(oracle.epilogue_bf16_bits(acc_r, 3.1e-4, wsr, br),
                           torch.from_numpy(f).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16))
+
+
+# ------------------------------------------------------------------ convolution weight tables (Fig. 4, Sec. 4.1, 4.2)
+def _conv_weights(rng, Cout, R, S, Cin):
+    """Weights whose range differs by tap, by input channel and by output channel, so that a table taken over
+    one tap only, over the wrong axis, or per group instead of per (group, output channel) is wrong."""
+    tap = rng.choice([0.1, 0.3, 1.0], size=(1, R, S, 1))
+    tap.flat[rng.integers(tap.size)] = 1.0
+    cin = rng.choice([0.5, 1.0], size=(1, 1, 1, Cin))
+    cell = np.repeat(rng.choice([1, 3, 8, 20, 50], size=(Cout, 1, 1, Cin // 16)), 16, axis=3)  # per (output, group)
+    W = rng.standard_normal((Cout, R, S, Cin)) * tap * cin * cell
+    return W.clip(-128, 127).astype(np.int8)
+
+
+@pytest.mark.parametrize("R,S", [(3, 3), (1, 1), (1, 3)])
+def test_conv_weight_positions_cover_all_taps_and_are_tight(R, S):
+    """Fig. 4 / Sec. 4.1: one extraction position per (channel group, output channel); for a convolution the group's
+    weights are those of ALL taps.  The position is the smallest shift for which no weight of the group leaves
+    [-8, 7] (weights never saturate), checked by brute force over the taps."""
+    rng = np.random.default_rng(60 + R * S)
+    G, Cin, Cout = 16, 64, 12
+    Wq = _conv_weights(rng, Cout, R, S, Cin)
+    perm = rng.permutation(Cin // G).astype(np.int32)
+    sw = oracle.weight_positions_conv(Wq, G, perm)
+    assert sw.shape == (Cin // G, Cout) and sw.max() <= 4
+    seen = set()
+    for j, g in enumerate(perm):
+        for n in range(Cout):
+            blk = Wq[n, :, :, g * G:(g + 1) * G].astype(int)  # every tap, the group's G channels
+            s = int(sw[j, n])
+            assert (blk >> s).min() >= -8 and (blk >> s).max() <= 7, "a weight would saturate"
+            if s > 0:
+                t = blk >> (s - 1)
+                assert t.min() < -8 or t.max() > 7, "position is not the smallest that fits"
+            seen.add(s)
+    assert len(seen) >= 3  # the draw exercises several positions
+    if R * S > 1:
+        # the widest tap decides: positions from the centre tap alone are somewhere smaller
+        one_tap = oracle.weight_positions_conv(Wq[:, :1, :1].copy(), G, perm)
+        assert np.all(one_tap <= sw) and np.any(one_tap < sw)
+
+
+def test_conv_1x1_weight_tables_equal_the_linear_ones():
+    """A 1x1 convolution is the linear layer with the transposed weight matrix: both tables must agree."""
+    rng = np.random.default_rng(71)
+    G, Cin, Cout = 16, 80, 24
+    Wq = _conv_weights(rng, Cout, 1, 1, Cin)
+    perm = rng.permutation(Cin // G).astype(np.int32)
+    Wlin = Wq.reshape(Cout, Cin).T.copy()
+    assert np.array_equal(oracle.weight_positions_conv(Wq, G, perm), oracle.weight_positions_linear(Wlin, G, perm))
+    assert np.array_equal(oracle.weight_absmax_conv(Wq), oracle.weight_absmax_linear(Wlin))
+
+
+def test_conv_weight_absmax_over_outputs_and_taps():
+    """Sec. 4.2: a feature channel's maximum weight range, here over every output channel and every tap."""
+    rng = np.random.default_rng(72)
+    Wq = _conv_weights(rng, 10, 3, 3, 48)
+    Wq[3, 2, 0, 5] = -128  # |-128| = 128 does not fit int8: the table is int32
+    got = oracle.weight_absmax_conv(Wq)
+    assert got.dtype == np.int32 and got[5] == 128
+    assert np.array_equal(got, np.abs(Wq.astype(np.int32)).max(axis=(0, 1, 2)))
+    # one tap or one output channel alone gives something smaller somewhere
+    assert np.any(np.abs(Wq[:, 1, 1].astype(np.int32)).max(axis=0) < got)
+    assert np.any(np.abs(Wq[0].astype(np.int32)).max(axis=(0, 1)) < got)
+
+
+# ------------------------------------------------------------------ epilogue: ONE rounding at general scales
+def _round_to_f32(v):
+    """Exact rational -> nearest float32, ties to even, decided with exact comparisons."""
+    from fractions import Fraction
+    c = np.float32(float(v))
+    cands = [c, np.nextafter(c, np.float32(np.inf)), np.nextafter(c, np.float32(-np.inf))]
+    best = None
+    for x in cands:
+        d = abs(Fraction(float(x)) - v)
+        even = (int(np.float32(x).view(np.uint32)) & 1) == 0
+        if best is None or d < best[0] or (d == best[0] and even and not best[2]):
+            best = (d, x, even)
+    return np.float32(best[1])
+
+
+def test_epilogue_is_one_fused_rounding_at_general_scales():
+    """y = acc * alpha + beta rounded ONCE to fp32 (a fused multiply-add), then, for int8, to the nearest integer
+    (ties to even) and clipped.  The expectation is exact rational arithmetic on the fp32 factors; a product
+    rounded before the addition, a factor associated differently, or float(acc) rounded twice fails it."""
+    from fractions import Fraction
+    rng = np.random.default_rng(80)
+    N = 16
+    acc = np.concatenate([
+        rng.integers(-2 ** 24, 2 ** 24, (40, N)),
+        rng.integers(-2 ** 31, 2 ** 31, (40, N)),       # beyond 2^24: float(acc) itself rounds
+        rng.integers(-3000, 3000, (40, N)),
+    ]).astype(np.int32)
+    x_scale, y_scale = np.float32(0.0137), np.float32(0.0911)
+    w_scale = rng.uniform(1e-3, 3e-2, N).astype(np.float32)
+    bias = rng.normal(0, 0.7, N).astype(np.float32)
+    # the factors, each operation rounded to fp32 (the oracle's stated association)
+    sxw = (x_scale * w_scale).astype(np.float32)
+    alpha = (sxw / y_scale).astype(np.float32)
+    beta = (bias / y_scale).astype(np.float32)
+    got8 = oracle.epilogue_i8(acc, float(x_scale), w_scale, bias, float(y_scale))
+    got32 = oracle.epilogue_f32(acc, float(x_scale), w_scale, bias)
+    n_double_rounding_differs = 0
+    for m in range(acc.shape[0]):
+        for n in range(N):
+            a = Fraction(float(np.float32(acc[m, n])))  # int -> fp32, nearest even (numpy's conversion)
+            y32 = _round_to_f32(a * Fraction(float(sxw[n])) + Fraction(float(bias[n])))
+            assert got32[m, n] == y32, (m, n)
+            y = _round_to_f32(a * Fraction(float(alpha[n])) + Fraction(float(beta[n])))
+            want = min(127, max(-128, round(Fraction(float(y)))))  # round(): half to even on exact rationals
+            assert int(got8[m, n]) == want, (m, n)
+            two = np.float32(np.float32(np.float32(acc[m, n]) * sxw[n]) + bias[n])
+            n_double_rounding_differs += int(two != y32)
+    assert n_double_rounding_differs > 20  # the case set tells one rounding from two
+
+
+def test_epilogue_int8_decisions_next_to_ties():
+    """The int8 output at accumulators chosen (by a scan in float64) so that y lies within a few fp32 ulps of a
+    half-integer: there a product rounded before the addition, or alpha built as x_scale * (w_scale / y_scale),
+    decides differently from the single fused rounding of the stated factors.  Expectations in exact rationals."""
+    from fractions import Fraction
+    rng = np.random.default_rng(81)
+    N = 512
+    x_scale, y_scale = np.float32(0.0137), np.float32(0.0911)
+    w_scale = rng.uniform(1e-3, 3e-2, N).astype(np.float32)
+    bias = rng.normal(0, 0.7, N).astype(np.float32)
+    alpha = ((x_scale * w_scale).astype(np.float32) / y_scale).astype(np.float32)
+    alpha_alt = (x_scale * (w_scale / y_scale).astype(np.float32)).astype(np.float32)
+    beta = (bias / y_scale).astype(np.float32)
+    cases = []  # (n, acc)
+    n_two, n_alt = 0, 0
+    for n in range(N):
+        lim = int(120.0 / float(alpha[n]))
+        a = np.arange(-lim, lim + 1, dtype=np.int64)
+        a32 = a.astype(np.float32)
+        fused = (a32.astype(np.float64) * np.float64(alpha[n]) + np.float64(beta[n])).astype(np.float32)
+        two = ((a32 * alpha[n]).astype(np.float32) + beta[n]).astype(np.float32)
+        alt = (a32.astype(np.float64) * np.float64(alpha_alt[n]) + np.float64(beta[n])).astype(np.float32)
+        pick_two = np.nonzero(np.rint(fused) != np.rint(two))[0]
+        pick_alt = np.nonzero(np.rint(fused) != np.rint(alt))[0]
+        n_two += pick_two.size
+        n_alt += pick_alt.size
+        for i in np.concatenate([pick_two[:2], pick_alt[:2]]):
+            cases.append((n, int(a[i])))
+    assert n_two >= 8 and n_alt >= 4, (n_two, n_alt)  # the scan found cases that tell the readings apart
+    acc = np.zeros((len(cases), N), np.int32)
+    for r, (n, v) in enumerate(cases):
+        acc[r, n] = v
+    got = oracle.epilogue_i8(acc, float(x_scale), w_scale, bias, float(y_scale))
+    for r, (n, v) in enumerate(cases):
+        y = _round_to_f32(Fraction(v) * Fraction(float(alpha[n])) + Fraction(float(beta[n])))
+        assert int(got[r, n]) == min(127, max(-128, round(Fraction(float(y))))), (n, v)
