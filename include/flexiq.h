@@ -14,6 +14,10 @@
  *     steady-state calls allocate nothing.
  *   - There is no CPU fallback: on a device that is not sm_100 the calls return
  *     FLEXIQ_ERR_UNSUPPORTED.
+ *   - A layer handle belongs to the device that was current when it was created.  Every call
+ *     that enqueues work for a handle returns FLEXIQ_ERR_INVALID_ARG when another device is
+ *     current (its pointers would not be valid there).  One handle is used from one stream at a
+ *     time; different handles may run on different streams concurrently.
  *   - Every device-side wait is bounded.  If one expires the kernel raises a status
  *     word that flexiq_check_status() reports as FLEXIQ_ERR_TIMEOUT; the context
  *     stays usable.
@@ -62,8 +66,10 @@ extern "C" {
  * MASKED : one int8 per value holding the 4-bit value already shifted back to its
  *          extraction position (x4 << sx), in ONE slab [M][K] together with the 8-bit groups
  *          (low groups first); the mainloop is a plain 8-bit integer GEMM over whole K blocks
- *          against one weight operand that follows the ratio (only the channel groups that
- *          changed sides are copied, on the stream of the next mixed_* call).
+ *          (128 channels; 64 for layers of fewer than 128): blocks below max_4bit_ch read the
+ *          4-bit weights at their positions, blocks above it the 8-bit weights, and only the
+ *          one block per filter tap that max_4bit_ch falls into (none when it is a multiple of
+ *          the block) depends on the ratio; see flexiq_set_lowbit_ratio.
  * Both give bit-identical accumulators. */
 #define FLEXIQ_LOWBIT_MASKED_I8 0
 #define FLEXIQ_LOWBIT_PACKED_U4 1
@@ -113,28 +119,38 @@ int flexiq_layer_set_group_perm(flexiq_layer_t layer, const int8_t *Wq_dev, cons
  * its slabs. */
 int flexiq_layer_set_lowbit_path(flexiq_layer_t layer, int lowbit_path);
 
-/* Brings the layer's private weight operand to the ratio in force, in stream order (a copy of the
- * channel groups that changed sides since the last mixed_* call; nothing when none did).  The
- * mixed_* calls do this themselves; the explicit call is for CUDA graphs: a graph captured while
- * ratio r was in force holds no such copy, so before it is replayed after another ratio was used,
- * set r again (flexiq_set_lowbit_ratio) and call this on the replaying stream.  One graph per ratio
- * and problem size can then be kept and replayed in any order (Sec. 7: the ratio changes at run
- * time without re-packing the weights). */
+/* Writes, in stream order, the one weight K block per filter tap that max_4bit_ch falls into (see
+ * flexiq_set_lowbit_ratio) for the ratio in force, if the stream does not hold it already; nothing
+ * on the PACKED path or when max_4bit_ch is a multiple of the block.  flexiq_quantize_lower and the
+ * mixed_* calls do this themselves, also inside a stream capture, where the write always becomes
+ * part of the graph: every captured graph is complete in itself, and one graph per ratio and problem
+ * size can be kept and replayed in any order (Sec. 7: the ratio changes at run time without
+ * re-packing the weights) with no call in between.  Kept for callers that want the write off their
+ * critical path. */
 int flexiq_layer_sync_ratio(flexiq_layer_t layer, void *stream);
 
 /* Run-time ratio switch (Sec. 7, "Low-bitwidth Ratio Adjustment"): sets
- * max_4bit_ch = K_lo = ceil(ratio * n_g - 1e-4) * G, clamped to [0, K].  Host-only, one
- * integer, no data movement.  Takes effect for calls enqueued afterwards.
+ * max_4bit_ch = K_lo = ceil(ratio * n_g - 1e-4) * G, clamped to [0, K].  The call itself is
+ * host-only: one integer.  Takes effect for calls enqueued afterwards.
+ * What the switch costs on the device: PACKED path nothing.  MASKED path nothing when K_lo is a
+ * multiple of the K block (128 channels; 64 for layers of fewer than 128 channels); otherwise the
+ * next flexiq_quantize_lower (extra thread blocks of its launch) or mixed_* call (a small kernel
+ * in front of it) writes the one K block per filter tap that K_lo falls into: N * taps * block
+ * bytes, e.g. 393 KB for a 768 x 3072 linear layer.  The weights themselves are never re-packed.
  * The slabs a flexiq_quantize_lower call writes belong to the ratio in force when it was enqueued,
- * and the mixed_* call that reads them must be enqueued at the same ratio: the library does not
- * record which ratio a caller's buffer was written at (slabs of several ratios may be prepared ahead
- * and used later), so a mismatch is not detected and gives wrong values.  On the PACKED path the
- * mixed_* call addresses X4_dev / X8_dev with the row pitches of the ratio in force when IT is
- * enqueued: buffers sized for a smaller low-bit slice would then be read past their end, so size
- * them for the largest ratio used (the MASKED slab is [M][K] at every ratio).
+ * and the mixed_* call that reads them must be enqueued at the same ratio.  The handle remembers
+ * at which max_4bit_ch it last saw each of the caller's slab buffers written (the eight most recent
+ * buffers, by address: slabs of several ratios may be prepared ahead in buffers of their own), and a
+ * mixed_* call that passes a remembered buffer at another ratio returns FLEXIQ_ERR_INVALID_ARG
+ * instead of computing wrong values or, on the PACKED path where the row pitch depends on the ratio,
+ * reading past the end of a buffer.  Buffers the handle has not seen written are taken on trust;
+ * flexiq_layer_set_slab_check(layer, 0) turns the check off for callers that fill slabs themselves.
  * ratio outside [0, 1] or NaN: FLEXIQ_ERR_INVALID_ARG. */
 int flexiq_set_lowbit_ratio(flexiq_layer_t layer, float ratio);
 int flexiq_get_max_4bit_ch(flexiq_layer_t layer, int *K_lo);
+/* enabled = 0: mixed_* calls no longer compare the ratio with the one a slab buffer was written at
+ * (see flexiq_set_lowbit_ratio); any other value turns the check back on (the default). */
+int flexiq_layer_set_slab_check(flexiq_layer_t layer, int enabled);
 
 /* Row pitch in bytes of the X4_dev slab for a given K_lo under the layer's path:
  * PACKED: K_lo / 2 rounded up to a multiple of 16;  MASKED: K (the slab holds every group). */

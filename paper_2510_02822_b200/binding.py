@@ -23,7 +23,7 @@ REORDER_TO_SLAB, REORDER_FROM_SLAB = 0, 1
 
 EXPORTS = [
     "flexiq_layer_create_linear", "flexiq_layer_create_conv", "flexiq_layer_destroy",
-    "flexiq_layer_set_group_perm", "flexiq_layer_set_lowbit_path", "flexiq_layer_sync_ratio", "flexiq_set_lowbit_ratio", "flexiq_get_max_4bit_ch",
+    "flexiq_layer_set_group_perm", "flexiq_layer_set_lowbit_path", "flexiq_layer_sync_ratio", "flexiq_layer_set_slab_check", "flexiq_set_lowbit_ratio", "flexiq_get_max_4bit_ch",
     "flexiq_x4_pitch", "flexiq_quantize_lower", "flexiq_quantize_lower_dynamic_noalloc", "flexiq_mixed_gemm", "flexiq_mixed_conv",
     "flexiq_mixed_gemm_to_slab", "flexiq_mixed_conv_to_slab", "flexiq_reorder_channels",
     "flexiq_calib_channel_ranges", "flexiq_calib_channel_histogram", "flexiq_calib_ranges_from_histogram",
@@ -58,6 +58,7 @@ def lib():
         L.flexiq_layer_destroy.argtypes = [vp]
         L.flexiq_layer_set_lowbit_path.argtypes = [vp, i32]
         L.flexiq_layer_sync_ratio.argtypes = [vp, vp]
+        L.flexiq_layer_set_slab_check.argtypes = [vp, i32]
         L.flexiq_layer_set_group_perm.argtypes = [vp, vp, vp, vp, vp]
         L.flexiq_set_lowbit_ratio.argtypes = [vp, f32]
         L.flexiq_get_max_4bit_ch.argtypes = [vp, C.POINTER(i32)]
@@ -144,6 +145,10 @@ def flexiq_layer_destroy(h):
 
 def flexiq_layer_set_lowbit_path(h, path):
     _check(lib().flexiq_layer_set_lowbit_path(h, path))
+
+
+def flexiq_layer_set_slab_check(h, enabled):
+    _check(lib().flexiq_layer_set_slab_check(h, int(bool(enabled))))
 
 
 def flexiq_set_lowbit_ratio(h, ratio):
@@ -301,7 +306,7 @@ class Layer:
         _check(lib().flexiq_layer_set_group_perm(self.h, _ptr(Wq), _np_ptr(perm), None if xs is None else _np_ptr(xs), _stream()))
 
     def sync_ratio(self):
-        """Weight operand to the ratio in force, on the current stream (needed only before a CUDA-graph replay)."""
+        """Writes the ratio-dependent weight K block for the ratio in force on the current stream, if it is not there yet."""
         _check(lib().flexiq_layer_sync_ratio(self.h, _stream()))
 
     @property

@@ -16,11 +16,16 @@ namespace flexiq {
 // With r correctly rounded and the first corrected t faithful, the last step yields the
 // correctly rounded quotient RN(x/S) (Markstein's theorem), i.e. the IEEE division result,
 // at five instructions per element.  (Only the final integer matters here: results in the
-// subnormal range may differ but round to 0 either way; inf / NaN inputs are excluded.)
+// subnormal range may differ but round to 0 either way.)  Infinite inputs, or inputs whose product with
+// r overflows, turn the corrections into NaN (inf - inf); the caller's clip fmaxf(NaN, lo) then yields lo,
+// which is right for the negative side only.  So x is first capped at 256 S from above -- every value
+// beyond it quantizes to 127 anyway -- and both infinities saturate as Eq. 1's clip says.  NaN inputs
+// are excluded.
 struct Divider {
-    float S, r;
+    float S, r, lim;
     __device__ __forceinline__ float operator()(float x) const
     {
+        x = fminf(x, lim);
         float t = __fmul_rn(x, r);
         t = __fmaf_rn(__fmaf_rn(-S, t, x), r, t);
         t = __fmaf_rn(__fmaf_rn(-S, t, x), r, t);
@@ -32,6 +37,7 @@ __device__ __forceinline__ Divider make_divider(float scale)
     Divider d;
     d.S = scale;
     d.r = __frcp_rn(scale);
+    d.lim = __fmul_rn(256.0f, scale);
     return d;
 }
 

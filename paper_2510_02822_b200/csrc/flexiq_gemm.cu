@@ -23,26 +23,13 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include "sm100_ptx.cuh"
-
-#include <stdlib.h>
+#include "straddle.cuh"
 
 namespace flexiq {
 
 __device__ unsigned int g_status_word = 0;
 
-// Optional role timers (build with -DFLEXIQ_PROFILE): cycles CTA 0 spends waiting per role.
-#ifdef FLEXIQ_PROFILE
-__device__ long long g_prof[16];
-#define PROF_DECL(name) long long name = 0
-#define PROF_T0(t) const long long t = clock64()
-#define PROF_ADD(name, t) name += clock64() - t
-#define PROF_STORE(i, v) do { if (blockIdx.x == 0) g_prof[i] = (v); } while (0)
-#else
-#define PROF_DECL(name)
-#define PROF_T0(t)
-#define PROF_ADD(name, t)
-#define PROF_STORE(i, v)
-#endif
+#include "role_timers.cuh"   // PROF_* expand to nothing in the product build
 
 constexpr int BM = 128;
 constexpr int kNumWorkWarps = 16;                     // epilogue warps (+ expander warps on the packed path)
@@ -69,12 +56,18 @@ struct GemmParams {
     int BN;              // tile width: 64, 128, 192 or 256
     int stages;          // depth of the operand ring
     int tps;             // filter taps per ring stage (> 1 only for masked convolutions whose C fits one K block)
-    int nb_lo, nb_hi;    // k-blocks per tap in the low / high slab
+    int nb_lo, nb_hi;    // K blocks per tap of the first / second run of blocks (packed path: low slab / 8-bit slab;
+                         // masked path: blocks read from w8m plus the straddle block / blocks read from w8)
+    int ks_last_lo, ks_last_hi;  // 32-byte K steps of the last block of each run (the others have BK / 32)
+    int xa_hi0, xb_hi0;  // first A / B column of the second run within a tap
+    int st_cb;           // masked path: block of the first run that is read from the straddle buffer (its last), or -1
+    int b_tap_step;      // multi-tap stages: columns from one tap to the next in the weight operand
     int im2col;          // A operand through im2col-mode TMA
     int P, Q, stride, pad;
     int out_mode;
-    const float *alpha;  // [N] per-output-channel multiplier of this call
-    const float *beta;   // [N] per-output-channel addend of this call
+    const float *w_scale;  // [N] per-output-channel weight scales
+    const float *bias;     // [N] or nullptr
+    float x_scale, y_scale;
     void *Y;
     int m_tiles, n_tiles;
     // fused layer boundary only: where each 16-channel chunk of the output lands in the next layer's slab
@@ -324,8 +317,14 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
     const int cols = BN >= 192 ? 64 : 32;
     const bool y32 = (reinterpret_cast<uintptr_t>(p.Y) & 31) == 0;
     const bool wide = y32 && (p.N & 31) == 0;    // int8 rows are 32-byte aligned: 256-bit stores
-    // lane l keeps factors 4l..4l+3 of the table alpha[64] | beta[64]
-    const float *fsrc = (lane < 16 ? p.alpha : p.beta) + 4 * (lane & 15);
+    // Per-output-channel factors, computed here from the layer's scales (each operation rounds once, in fp32):
+    //   re-quantizing modes  alpha = (S_x * S_w[n]) / S_y,  beta = bias[n] / S_y
+    //   floating-point modes alpha = S_x * S_w[n],          beta = bias[n]
+    // Lanes 0-15 build alpha, lanes 16-31 beta; lane l keeps factors 4l..4l+3 of the table alpha[64] | beta[64].
+    constexpr bool kRequant = MODE == FLEXIQ_OUT_REQUANT_I8 || MODE == kOutNextSlab;
+    const float *fsrc = (lane < 16 ? p.w_scale : p.bias);
+    if (fsrc) fsrc += 4 * (lane & 15);
+    const float fmul = lane < 16 ? p.x_scale : 1.0f;   // multiplying by 1 is exact
     int buf = 0;
     uint32_t buf_phase = 0;
     PROF_DECL(prof_wait);
@@ -356,7 +355,14 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                 continue;
             }
             float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (kScaled && nw + 4 * (lane & 15) < p.N) f = __ldg(reinterpret_cast<const float4 *>(fsrc + nw));
+            if (kScaled && fsrc && nw + 4 * (lane & 15) < p.N) {
+                f = __ldg(reinterpret_cast<const float4 *>(fsrc + nw));
+                f.x = __fmul_rn(fmul, f.x); f.y = __fmul_rn(fmul, f.y); f.z = __fmul_rn(fmul, f.z); f.w = __fmul_rn(fmul, f.w);
+                if (kRequant) {
+                    f.x = __fdiv_rn(f.x, p.y_scale); f.y = __fdiv_rn(f.y, p.y_scale);
+                    f.z = __fdiv_rn(f.z, p.y_scale); f.w = __fdiv_rn(f.w, p.y_scale);
+                }
+            }
             int ent = 0;                                     // fused boundary: lane g fetches chunk g's slab entry
             if (MODE == kOutNextSlab && lane < 4 && nw + 16 * lane < p.N) ent = __ldg(p.next_ent + (nw >> 4) + lane);
             if (!waited) {
@@ -598,7 +604,7 @@ template <int CG, int PK, int KIND, bool SPLIT>
 __global__ void __launch_bounds__(kThreads, 1)
 mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_constant__ CUtensorMap mapA_hi,
                   const __grid_constant__ CUtensorMap mapB_lo, const __grid_constant__ CUtensorMap mapB_hi,
-                  const __grid_constant__ CUtensorMap mapY, const __grid_constant__ CUtensorMap mapY16,
+                  const __grid_constant__ CUtensorMap mapB_st, const __grid_constant__ CUtensorMap mapY, const __grid_constant__ CUtensorMap mapY16,
                   const GemmParams p)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -680,6 +686,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             ptx::prefetch_tmap(&mapA_hi);
             ptx::prefetch_tmap(&mapB_lo);
             ptx::prefetch_tmap(&mapB_hi);
+            if (!PK && p.st_cb >= 0) ptx::prefetch_tmap(&mapB_st);
         }
         const uint32_t tx_bytes = (uint32_t)(CG * (BM * p.BK + b_rows * p.BK));  // both CTAs' loads
         const uint32_t stage0 = ptx::smem_u32(stage_base) + (uint32_t)ring_off;
@@ -702,7 +709,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             if (leader) ptx::mbar_expect_tx_s(bar, (uint32_t)(CG * p.T * b_sub));
             const uint32_t bar_lead = CG == 2 ? ptx::mapa(bar, 0) : bar;
             for (int t = 0; t < p.T; ++t)
-                ptx::tma_load_2d_s<CG>(ptx::smem_u32(stage_base) + t * b_sub, &mapB_hi, bar_lead, t * p.C, (int)cta_rank * b_rows);
+                ptx::tma_load_2d_s<CG>(ptx::smem_u32(stage_base) + t * b_sub, &mapB_hi, bar_lead, t * p.b_tap_step, (int)cta_rank * b_rows);
         }
         __syncwarp();
         // Output pixel (image, row, column) of this CTA's first row in the current tile, kept up to date by
@@ -736,12 +743,12 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                         for (int i = 0; i < nt; ++i) {
                             ptx::tma_load_im2col_4d_s<CG>(sa + i * a_sub, &mapA_hi, bar, 0, pix_w, pix_h, pix_n, (uint16_t)ts, (uint16_t)tr);
                             if (!k_bres) ptx::tma_load_2d_s<CG>(sa + b_off + i * b_sub, &mapB_hi, bar, tk, n0);
-                            tk += p.C;
+                            tk += p.b_tap_step;
                             if (++ts == p.S) { ts = 0; ++tr; }
                         }
                     }
                     for (int i = 0; i < nt; ++i) {
-                        tap_k += p.C;
+                        tap_k += p.b_tap_step;
                         if (++tap_s == p.S) { tap_s = 0; ++tap_r; }
                     }
                     __syncwarp();
@@ -755,12 +762,11 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                 if (nb == 0) continue;
                 const CUtensorMap *ma = part ? &mapA_hi : &mapA_lo;
                 const CUtensorMap *mb = part ? &mapB_hi : &mapB_lo;
-                // weights: slab-order [N][T*C]; the low forms start each tap at channel 0, the
-                // 8-bit form of the high groups at channel C_lo
-                int xb_tap = part ? p.C_lo : 0;
+                // weights: slab-order [N][T*C]; the first run starts each tap at channel 0, the second at xb_hi0
+                int xb_tap = part ? p.xb_hi0 : 0;
                 int tap_r = 0, tap_s = 0;
                 for (int tap = 0; tap < p.T && ok; ++tap) {
-                    int xa = 0, xb = xb_tap;
+                    int xa = part ? p.xa_hi0 : 0, xb = xb_tap;
                     for (int cb = 0; cb < nb; ++cb) {
                         if (PK && part == 0) {
                             // packed low block: half-size raw tiles for the expander warps; the operand-ring
@@ -796,7 +802,9 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                                 ptx::tma_load_im2col_4d_s<CG>(sa, ma, bar, xa, pix_w, pix_h, pix_n, (uint16_t)tap_s, (uint16_t)tap_r);
                             else
                                 ptx::tma_load_2d_s<CG>(sa, ma, bar, xa, (int)m0);
-                            ptx::tma_load_2d_s<CG>(sa + b_off, mb, bar, xb, n0);
+                            // the block that max_4bit_ch falls into comes from the straddle buffer [N][T][BK]
+                            if (!PK && part == 0 && cb == p.st_cb) ptx::tma_load_2d_s<CG>(sa + b_off, &mapB_st, bar, tap * p.BK, n0);
+                            else ptx::tma_load_2d_s<CG>(sa + b_off, mb, bar, xb, n0);
                         }
                         __syncwarp();
                         xa += p.BK;
@@ -919,7 +927,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                 for (int part = 0; part < 2 && ok && k_tps == 1; ++part) {
                     const int nb = part ? p.nb_hi : p.nb_lo;
                     if (nb == 0) continue;
-                    const int ks_last = ((part ? p.C_hi : p.C_lo) - (nb - 1) * p.BK + 31) >> 5;
+                    const int ks_last = part ? p.ks_last_hi : p.ks_last_lo;
                     for (int tap = 0; tap < p.T && ok; ++tap) {
                         for (int cb = 0; cb < nb; ++cb) {
                             if (SPLIT) {
@@ -1126,34 +1134,12 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
     }
 }
 
-// Brings the masked path's weight operand up to date with max_4bit_ch: the channel range
-// [k_from, k_to) of every tap and output channel is copied from `src` (w8m when the range became
-// low-bit, w8 when it returned to 8 bits), 16 bytes per thread.
-__global__ void patch_weights_kernel(int8_t *__restrict__ wf, const int8_t *__restrict__ src, int N, int T, int C,
-                                     int k_from, int k_to)
+// The straddle block of the masked path (straddle.cuh) for a GEMM that no prologue launch precedes.
+__global__ void straddle_kernel(const StraddleJob job)
 {
-    const int upt = (k_to - k_from) >> 4;  // 16-byte units per (n, tap)
-    const long long total = (long long)N * T * upt;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    ptx::pdl_wait();  // the previous kernel of the stream may still read wf
-    if (idx >= total) return;
-    const int u = (int)(idx % upt);
-    const long long nt = idx / upt;  // n * T + tap
-    const size_t off = (size_t)nt * C + k_from + 16 * u;
-    *reinterpret_cast<uint4 *>(wf + off) = *reinterpret_cast<const uint4 *>(src + off);
-}
-
-// Per-output-channel factors of a call: REQUANT alpha = (S_x * S_w[n]) / S_y, beta = bias[n] / S_y;
-// DEQUANT alpha = S_x * S_w[n], beta = bias[n].  Each operation rounds once, in fp32.
-__global__ void scale_vectors_kernel(int N, float x_scale, float y_scale, int requant, const float *__restrict__ w_scale,
-                                     const float *__restrict__ bias, float *__restrict__ alpha, float *__restrict__ beta)
-{
-    const int n = blockIdx.x * blockDim.x + threadIdx.x;
-    if (n >= N) return;
-    const float sxw = __fmul_rn(x_scale, w_scale[n]);
-    const float bv = bias ? bias[n] : 0.f;
-    alpha[n] = requant ? __fdiv_rn(sxw, y_scale) : sxw;
-    beta[n] = requant ? __fdiv_rn(bv, y_scale) : bv;
+    ptx::pdl_wait();  // the previous kernel of the stream may still read the block
+    if (idx < (long long)job.rows * (job.BK >> 4)) straddle_write_unit(job, idx);
 }
 
 // ------------------------------------------------------------------------------------
@@ -1169,14 +1155,6 @@ __global__ void scale_vectors_kernel(int N, float x_scale, float y_scale, int re
 //                (cluster launch and barriers), which pays off once the machine is full.
 struct TileChoice { int cg, bn; };
 static TileChoice g_forced_tile{0, 0};  // test hook: 0 = choose automatically
-static bool direct_stores_only()
-{
-#ifdef FLEXIQ_PROFILE
-    return getenv("FLEXIQ_DIRECT_STORES") != nullptr;  // A/B timing in the profiling build
-#else
-    return false;
-#endif
-}
 static TileChoice choose_tile(long long M, int N, int k_blocks, int bk, int sms)
 {
     const int bns[4] = {256, 192, 128, 64};
@@ -1230,7 +1208,7 @@ static int make_map_im2col(CUtensorMap *map, const void *base, int Cpart, long l
 
 template <int CG, int PK, int KIND, bool SPLIT>
 static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const CUtensorMap &b_lo, const CUtensorMap &b_hi,
-                         const CUtensorMap &y_map, const CUtensorMap &y_map16, const GemmParams &p, int sms, cudaStream_t st)
+                         const CUtensorMap &b_st, const CUtensorMap &y_map, const CUtensorMap &y_map16, const GemmParams &p, int sms, cudaStream_t st)
 {
     static bool attr_set[64] = {};   // per instantiation
     int dev = 0;
@@ -1256,23 +1234,26 @@ static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    FLEXIQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, mixed_gemm_kernel<CG, PK, KIND, SPLIT>, a_lo, a_hi, b_lo, b_hi, y_map, y_map16, p));
+    FLEXIQ_CUDA_TRY(cudaLaunchKernelEx(&cfg, mixed_gemm_kernel<CG, PK, KIND, SPLIT>, a_lo, a_hi, b_lo, b_hi, b_st, y_map, y_map16, p));
     return FLEXIQ_OK;
 }
 
-// Masked path: the weight operand wf follows the ratio lazily.  Only the channel groups that changed
-// sides since the last update are copied (from w8m when they became low-bit, from w8 when they
-// returned to 8 bits), in stream order.
-static int sync_weight_operand(Layer *L, cudaStream_t st)
+// Masked path: writes the straddle block for the current max_4bit_ch when the stream does not hold it yet
+// (a prologue launch at this ratio normally has written it already).
+static int sync_straddle(Layer *L, cudaStream_t st)
 {
-    const int C_lo = L->K_lo;
-    if (L->wf_K_lo == C_lo) return FLEXIQ_OK;
-    const int k_from = C_lo < L->wf_K_lo ? C_lo : L->wf_K_lo, k_to = C_lo < L->wf_K_lo ? L->wf_K_lo : C_lo;
-    const long long total = (long long)L->N * L->R * L->S * ((k_to - k_from) >> 4);
-    patch_weights_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(L->wf, C_lo > L->wf_K_lo ? L->w8m : L->w8, L->N,
-                                                                          L->R * L->S, L->C, k_from, k_to);
+    if (!straddle_in_use(L) || !straddle_stale(L, st)) return FLEXIQ_OK;
+    StraddleJob job{};
+    job.wst = L->wst; job.w8m = L->w8m; job.w8 = L->w8;
+    job.rows = L->N * L->R * L->S;
+    job.C = L->C;
+    job.BK = choose_bk(L);
+    job.blk0 = (L->K_lo / job.BK) * job.BK;
+    job.K_lo = L->K_lo;
+    const long long total = (long long)job.rows * (job.BK >> 4);
+    straddle_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(job);
     FLEXIQ_CUDA_TRY(cudaGetLastError());
-    L->wf_K_lo = C_lo;
+    straddle_written(L, st);
     return FLEXIQ_OK;
 }
 
@@ -1309,21 +1290,45 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
         return set_error(FLEXIQ_ERR_UNSUPPORTED, "packed low-bit convolution needs Cin %% 32 == 0 (TMA start alignment of the 4-bit weight taps)");
     int rc = check_device_sm100();
     if (rc) return rc;
+    if ((rc = check_layer_device(L))) return rc;
+    // the slabs must have been written at the ratio now in force (known buffers only)
+    if (packed_path) {
+        if (C_lo > 0 && (rc = check_slab(L, X4, "X4_dev"))) return rc;
+        if (C_hi > 0 && (rc = check_slab(L, X8, "X8_dev"))) return rc;
+    } else if ((rc = check_slab(L, X4, "X4_dev"))) return rc;
     const int sms = device_sm_count(L->device);
 
-    if (!packed) {
-        // Masked path: activations are one slab [rows][C] and the weights one operand wf, so the
-        // mainloop is a plain 8-bit GEMM over whole K blocks whatever the ratio.  wf follows the
-        // ratio lazily: only the channel groups that changed sides are copied, in stream order.
-        int rcw = sync_weight_operand(L, st);
-        if (rcw) return rcw;
-    }
     GemmParams p{};
     p.M = M; p.N = L->N; p.C = L->C; p.C_lo = packed ? C_lo : 0; p.C_hi = packed ? C_hi : L->C;
     p.T = L->R * L->S; p.S = L->S;
     p.BK = choose_bk(L);
-    p.nb_lo = (p.C_lo + p.BK - 1) / p.BK;
-    p.nb_hi = (p.C_hi + p.BK - 1) / p.BK;
+    p.st_cb = -1;
+    p.b_tap_step = L->C;
+    int b_whole = 0;   // masked multi-tap stages: 0 = w8, 1 = w8m, 2 = straddle buffer
+    if (packed) {
+        p.nb_lo = (p.C_lo + p.BK - 1) / p.BK;
+        p.nb_hi = (p.C_hi + p.BK - 1) / p.BK;
+        p.ks_last_lo = (p.C_lo - (p.nb_lo - 1) * p.BK + 31) >> 5;
+        p.ks_last_hi = (p.C_hi - (p.nb_hi - 1) * p.BK + 31) >> 5;
+        p.xa_hi0 = 0;          // the 8-bit groups have a slab of their own
+        p.xb_hi0 = C_lo;
+    } else {
+        // Masked path: activations are one slab [rows][C], and the mainloop is a plain 8-bit GEMM over whole
+        // K blocks whatever the ratio: blocks below max_4bit_ch read w8m, blocks above it w8, and the block
+        // the boundary falls into (if any) the straddle buffer.  Nothing else depends on the ratio.
+        const int nbt = (L->C + p.BK - 1) / p.BK;
+        const bool st_blk = straddle_in_use(L);
+        if ((rc = sync_straddle(L, st))) return rc;
+        p.nb_lo = C_lo / p.BK + (st_blk ? 1 : 0);
+        if (C_lo == L->C) p.nb_lo = nbt;
+        p.nb_hi = nbt - p.nb_lo;
+        if (st_blk) p.st_cb = p.nb_lo - 1;
+        const int ks_end = (L->C - (nbt - 1) * p.BK + 31) >> 5;   // the last block of a tap may be partial
+        p.ks_last_lo = p.nb_hi == 0 ? ks_end : p.BK >> 5;
+        p.ks_last_hi = ks_end;
+        p.xa_hi0 = p.xb_hi0 = p.nb_lo * p.BK;
+        b_whole = C_lo == 0 ? 0 : (C_lo == L->C ? 1 : 2);   // when one K block holds all channels
+    }
     p.im2col = L->is_conv && (L->R != 1 || L->S != 1 || L->stride != 1 || L->pad != 0);
     p.stride = L->stride; p.pad = L->pad;
     if (L->is_conv) {
@@ -1332,7 +1337,7 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     }
     p.out_mode = out_mode; p.Y = Y;
     if (next) { p.next_ent = out_order == FLEXIQ_ORDER_NEXT_SLAB ? next->chunk_ent_slab : next->chunk_ent; p.next_K_lo = next->K_lo; p.relu = relu != 0; }
-    p.alpha = L->alpha; p.beta = L->beta;
+    p.w_scale = L->w_scale; p.bias = L->bias; p.x_scale = x_scale; p.y_scale = y_scale;
     TileChoice tc = g_forced_tile.cg ? g_forced_tile : choose_tile(M, L->N, p.T * (p.nb_lo + p.nb_hi), p.BK, sms);
     if (packed && tc.cg == 2) {  // the packed path runs single CTAs: re-choose among those
         tc.cg = 1;
@@ -1376,26 +1381,13 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
         p.stages = (kStageRegion - raw) / ((BM + bn) * p.BK);
         if (p.stages > kMaxStages) p.stages = kMaxStages;
     }
-    // the per-output-channel factors depend on the call's scales: recomputed (one tiny launch,
-    // stream-ordered before the GEMM) only when they differ from the previous call's
-    // the fused boundary re-quantizes with the REQUANT factors; the three floating-point outputs share theirs
-    const int fmode = next ? FLEXIQ_OUT_REQUANT_I8
-                           : ((out_mode == FLEXIQ_OUT_DEQUANT_F16 || out_mode == FLEXIQ_OUT_DEQUANT_BF16) ? FLEXIQ_OUT_DEQUANT_F32 : out_mode);
-    if (fmode != FLEXIQ_OUT_ACC_I32 &&
-        !(L->cache_mode == fmode && L->cache_xs == x_scale && (fmode == FLEXIQ_OUT_DEQUANT_F32 || L->cache_ys == y_scale))) {
-        scale_vectors_kernel<<<(L->N + 255) / 256, 256, 0, st>>>(L->N, x_scale, y_scale, fmode == FLEXIQ_OUT_REQUANT_I8,
-                                                                 L->w_scale, L->bias, L->alpha, L->beta);
-        FLEXIQ_CUDA_TRY(cudaGetLastError());
-        L->cache_mode = fmode; L->cache_xs = x_scale; L->cache_ys = y_scale;
-    }
-
     // activation maps (per call: they depend on the caller's buffers, M and the ratio);
     // an empty slab borrows the other one's map and is never addressed
     CUtensorMap a_lo, a_hi;
     const bool half_out = out_mode == FLEXIQ_OUT_DEQUANT_F16 || out_mode == FLEXIQ_OUT_DEQUANT_BF16;
     const bool word_out = out_mode == FLEXIQ_OUT_DEQUANT_F32 || out_mode == FLEXIQ_OUT_ACC_I32;
     const int y_elem = half_out ? 2 : (word_out ? 4 : 1);
-    const bool staged = (!next || out_order == FLEXIQ_ORDER_NEXT_SLAB) && !direct_stores_only();
+    const bool staged = !next || out_order == FLEXIQ_ORDER_NEXT_SLAB;
     const void *slab = packed_path ? static_cast<const void *>(X8) : static_cast<const void *>(X4);
     Layer::CallMaps &cm = L->call_maps;
     const bool cached = !packed && cm.slab == slab && cm.M == M && cm.Nb == Nb && cm.H == H && cm.W == W && cm.bk == p.BK &&
@@ -1451,8 +1443,12 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     // second accumulator's extra read in the epilogue would only cost (measured: +4 to +6 % on short-K shapes).
     const bool split = !packed && bn <= 128 && p.tps == 1 && p.T * (p.nb_lo + p.nb_hi) >= 8 &&
                        (long long)p.m_tiles * p.n_tiles <= sms / cg;
-    if (packed) return launch_kernel<1, 1, 1, false>(a_lo, a_hi, L->map_w4[bi], L->map_w8[bi], y_map, y_map16, p, sms, st);
-#define FLEXIQ_LAUNCH(CG_, KIND_, SPLIT_) launch_kernel<CG_, 0, KIND_, SPLIT_>(a_lo, a_hi, L->map_wf[bi], L->map_wf[bi], y_map, y_map16, p, sms, st)
+    if (next) record_slab(const_cast<Layer *>(next), Y, next->K_lo);   // the fused boundary writes the next layer's slab at its current ratio
+    if (packed) return launch_kernel<1, 1, 1, false>(a_lo, a_hi, L->map_w4[bi], L->map_w8[bi], L->map_w8[bi], y_map, y_map16, p, sms, st);
+    // multi-tap stages hold every channel in one K block: the whole weight operand is one of the three forms
+    const CUtensorMap &b_hi_map = p.tps > 1 ? (b_whole == 0 ? L->map_w8[bi] : (b_whole == 1 ? L->map_w8m[bi] : L->map_wst[bi])) : L->map_w8[bi];
+    if (p.tps > 1 && b_whole == 2) p.b_tap_step = p.BK;
+#define FLEXIQ_LAUNCH(CG_, KIND_, SPLIT_) launch_kernel<CG_, 0, KIND_, SPLIT_>(a_lo, a_hi, L->map_w8m[bi], b_hi_map, L->map_wst[bi], y_map, y_map16, p, sms, st)
     if (cg == 2) {
         if (conv_kind) return split ? FLEXIQ_LAUNCH(2, 1, true) : FLEXIQ_LAUNCH(2, 1, false);
         return split ? FLEXIQ_LAUNCH(2, 0, true) : FLEXIQ_LAUNCH(2, 0, false);
@@ -1521,15 +1517,6 @@ extern "C" int flexiq_mixed_conv_to_slab(flexiq_layer_t layer, const uint8_t *X4
                      reinterpret_cast<cudaStream_t>(stream), Nx, relu, out_order);
 }
 
-#ifdef FLEXIQ_PROFILE
-extern "C" int flexiq_profile_counters(long long *out16)
-{
-    FLEXIQ_CUDA_TRY(cudaDeviceSynchronize());
-    FLEXIQ_CUDA_TRY(cudaMemcpyFromSymbol(out16, g_prof, sizeof(long long) * 16));
-    return FLEXIQ_OK;
-}
-#endif
-
 extern "C" int flexiq_choose_tile(int64_t M, int N, int k_blocks, int block_k, int sm_count, int *cta_group_out, int *tile_n_out)
 {
     if (M <= 0 || N <= 0 || k_blocks <= 0 || sm_count <= 0 || (block_k != 128 && block_k != 64) || !cta_group_out || !tile_n_out)
@@ -1567,8 +1554,8 @@ extern "C" int flexiq_layer_sync_ratio(flexiq_layer_t layer, void *stream)
 {
     Layer *L = as_layer(layer);
     if (!L) return set_error(FLEXIQ_ERR_INVALID_ARG, "not a live flexiq layer handle");
-    if (L->lowbit_path == FLEXIQ_LOWBIT_PACKED_U4 && L->K_lo > 0) return FLEXIQ_OK;  // that path reads w4 and w8 as they are
     int rc = check_device_sm100();
     if (rc) return rc;
-    return sync_weight_operand(L, reinterpret_cast<cudaStream_t>(stream));
+    if ((rc = check_layer_device(L))) return rc;
+    return sync_straddle(L, reinterpret_cast<cudaStream_t>(stream));
 }

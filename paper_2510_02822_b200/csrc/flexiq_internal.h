@@ -38,8 +38,15 @@ struct Layer {
     int8_t *w8;      // [N][Kw] slab-order int8 weights
     int8_t *w8m;     // [N][Kw] (w >> sw) << sw : 4-bit weights at their extraction position
     uint8_t *w4;     // [N][Kw/2] packed 4-bit weights (w >> sw)
-    int8_t *wf;      // [N][Kw] masked path's operand: w8m for the groups below wf_K_lo, w8 for the rest
-    int wf_K_lo;     // the max_4bit_ch that wf currently reflects (patched lazily, in stream order)
+    // Masked path: K blocks wholly below max_4bit_ch are read from w8m, K blocks wholly above it from w8.
+    // Only the one block that contains the boundary (when max_4bit_ch is not a multiple of the block) needs
+    // both: it lives in wst, [N][taps][BK] bytes, rewritten when the ratio changes (see straddle.cuh).
+    int8_t *wst;
+    int st_K_lo;                   // the max_4bit_ch wst holds as far as eager calls know; -1 = unknown
+    int st_graph_seen;             // a write of wst was captured into a CUDA graph: replays rewrite wst behind
+                                   // st_K_lo, so eager calls no longer trust it
+    unsigned long long st_cap_id;  // capture sequence that last wrote wst, and for which max_4bit_ch
+    int st_cap_K_lo;
     uint8_t *sw;     // [n_g][N] weight extraction positions
     uint8_t *sx;     // [n_g] static activation positions, slab order
     int32_t *perm;   // [n_g]
@@ -61,11 +68,7 @@ struct Layer {
     int32_t *perm_host;
     uint8_t *sx_host;
     // tensor maps over the weights (encoded once)
-    CUtensorMap map_w8[kNumWeightMaps], map_w4[kNumWeightMaps], map_wf[kNumWeightMaps];  // one per box height
-    // per-output-channel epilogue factors of the most recent call and what they were computed for
-    float *alpha, *beta;
-    float cache_xs, cache_ys;
-    int cache_mode;
+    CUtensorMap map_w8[kNumWeightMaps], map_w4[kNumWeightMaps], map_w8m[kNumWeightMaps], map_wst[kNumWeightMaps];  // one per box height
     int w4_pitch;    // row pitch of w4 in bytes: Kw/2 rounded up to 16
     // tensor maps of the most recent masked-path call, reused while the caller passes the same buffers
     // and shapes (encoding three maps costs more host time than the rest of a small call)
@@ -75,7 +78,24 @@ struct Layer {
         int Nb, H, W, bk, im2col, staged, y_elem;
         CUtensorMap a, y, y16;
     } call_maps;
+    // Which max_4bit_ch the caller's slab buffers were last written at (by flexiq_quantize_lower or by a
+    // fused-boundary producer): a mixed_* call on a known buffer at another ratio is refused.
+    struct SlabRecord { const void *ptr; int K_lo; } slab_seen[8];
+    int slab_next;
+    int slab_check;  // 0 = the caller opted out
 };
+
+// the slab bookkeeping above
+void record_slab(Layer *L, const void *ptr, int K_lo);
+int check_slab(const Layer *L, const void *ptr, const char *what);
+// FLEXIQ_ERR_INVALID_ARG unless the current device is the one the handle was created on
+int check_layer_device(const Layer *L);
+// 0 when the stream is not being captured, else the id of the capture sequence
+unsigned long long stream_capture_id(cudaStream_t st);
+// masked path: does a GEMM at the layer's current max_4bit_ch read the straddle block, and must it be written first?
+bool straddle_in_use(const Layer *L);
+bool straddle_stale(const Layer *L, cudaStream_t st);
+void straddle_written(Layer *L, cudaStream_t st);
 
 constexpr uint32_t kLayerMagic = 0x464c5851u;  // "FLXQ"
 

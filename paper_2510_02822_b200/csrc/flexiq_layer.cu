@@ -58,6 +58,67 @@ Layer *as_layer(flexiq_layer_t h)
     return L;
 }
 
+int check_layer_device(const Layer *L)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return set_error(FLEXIQ_ERR_CUDA, "cudaGetDevice failed: %s", cudaGetErrorString(e));
+    if (dev != L->device)
+        return set_error(FLEXIQ_ERR_INVALID_ARG, "the layer lives on device %d but device %d is current: its pointers are not valid there",
+                         L->device, dev);
+    return FLEXIQ_OK;
+}
+
+unsigned long long stream_capture_id(cudaStream_t st)
+{
+    cudaStreamCaptureStatus status = cudaStreamCaptureStatusNone;
+    unsigned long long id = 0;
+    if (cudaStreamGetCaptureInfo(st, &status, &id) != cudaSuccess) { cudaGetLastError(); return 0; }
+    return status == cudaStreamCaptureStatusActive ? (id ? id : 1ull) : 0ull;
+}
+
+void record_slab(Layer *L, const void *ptr, int K_lo)
+{
+    if (!ptr) return;
+    for (int i = 0; i < 8; ++i)
+        if (L->slab_seen[i].ptr == ptr) { L->slab_seen[i].K_lo = K_lo; return; }
+    L->slab_seen[L->slab_next] = Layer::SlabRecord{ptr, K_lo};
+    L->slab_next = (L->slab_next + 1) & 7;
+}
+
+int check_slab(const Layer *L, const void *ptr, const char *what)
+{
+    if (!L->slab_check || !ptr) return FLEXIQ_OK;
+    for (int i = 0; i < 8; ++i)
+        if (L->slab_seen[i].ptr == ptr && L->slab_seen[i].K_lo != L->K_lo)
+            return set_error(FLEXIQ_ERR_INVALID_ARG,
+                             "%s was last written at max_4bit_ch = %d but the layer is now at %d: run flexiq_quantize_lower "
+                             "again, or set the ratio the slab was written at", what, L->slab_seen[i].K_lo, L->K_lo);
+    return FLEXIQ_OK;
+}
+
+// Masked path: the straddle block is read when max_4bit_ch falls inside a K block.
+bool straddle_in_use(const Layer *L)
+{
+    return L->lowbit_path == FLEXIQ_LOWBIT_MASKED_I8 && L->K_lo < L->C && (L->K_lo % choose_bk(L)) != 0;
+}
+// Does wst hold the block for the current max_4bit_ch at this point of the stream?  Outside a capture the
+// host's record decides, unless a captured graph may have rewritten wst since.  Inside a capture only a write
+// earlier in the same capture counts, so that every graph is complete in itself and graphs of different
+// ratios replay in any order.
+bool straddle_stale(const Layer *L, cudaStream_t st)
+{
+    const unsigned long long cap = stream_capture_id(st);
+    if (cap) return !(L->st_cap_id == cap && L->st_cap_K_lo == L->K_lo);
+    return L->st_graph_seen || L->st_K_lo != L->K_lo;
+}
+void straddle_written(Layer *L, cudaStream_t st)
+{
+    const unsigned long long cap = stream_capture_id(st);
+    if (cap) { L->st_cap_id = cap; L->st_cap_K_lo = L->K_lo; L->st_graph_seen = 1; L->st_K_lo = -1; }
+    else L->st_K_lo = L->K_lo;
+}
+
 static void *driver_entry(const char *name)
 {
     void *fn = nullptr;
@@ -189,8 +250,8 @@ static void free_layer(Layer *L)
 {
     if (!L) return;
     if (L->tables_in_flight) cudaEventSynchronize(L->tables_event);
-    cudaFree(L->w8); cudaFree(L->w8m); cudaFree(L->w4); cudaFree(L->wf); cudaFree(L->sw);
-    cudaFree(L->tables); cudaFree(L->w_scale); cudaFree(L->bias); cudaFree(L->alpha); cudaFree(L->beta);
+    cudaFree(L->w8); cudaFree(L->w8m); cudaFree(L->w4); cudaFree(L->wst); cudaFree(L->sw);
+    cudaFree(L->tables); cudaFree(L->w_scale); cudaFree(L->bias);
     if (L->tables_host) cudaFreeHost(L->tables_host);
     if (L->tables_event) cudaEventDestroy(L->tables_event);
     free(L->perm_host); free(L->sx_host);
@@ -205,7 +266,10 @@ int encode_weight_maps(Layer *L)
     for (int i = 0; i < kNumWeightMaps; ++i) {
         int rc = make_map_2d(&L->map_w8[i], L->w8, (uint64_t)L->Kw, (uint64_t)L->N, (uint64_t)L->Kw, bk, bns[i], bk);
         if (rc) return rc;
-        rc = make_map_2d(&L->map_wf[i], L->wf, (uint64_t)L->Kw, (uint64_t)L->N, (uint64_t)L->Kw, bk, bns[i], bk);
+        rc = make_map_2d(&L->map_w8m[i], L->w8m, (uint64_t)L->Kw, (uint64_t)L->N, (uint64_t)L->Kw, bk, bns[i], bk);
+        if (rc) return rc;
+        const uint64_t st_row = (uint64_t)L->R * L->S * bk;   // the straddle block of every tap
+        rc = make_map_2d(&L->map_wst[i], L->wst, st_row, (uint64_t)L->N, st_row, bk, bns[i], bk);
         if (rc) return rc;
         rc = make_map_2d(&L->map_w4[i], L->w4, (uint64_t)L->Kw / 2, (uint64_t)L->N, (uint64_t)L->w4_pitch, bk / 2, bns[i],
                          bk / 2 == 64 ? 64 : 0);  // raw 4-bit tiles: 64-byte rows are read row-per-thread, so they are swizzled
@@ -241,14 +305,15 @@ static int layout_layer(Layer *L, const int8_t *Wq, const int32_t *perm, const u
     FLEXIQ_CUDA_TRY(cudaMemcpyAsync(L->tables, L->tables_host, L->tables_bytes, cudaMemcpyHostToDevice, stream));
     FLEXIQ_CUDA_TRY(cudaEventRecord(L->tables_event, stream));
     L->tables_in_flight = 1;
-    const size_t wbytes = (size_t)N * L->Kw;
     const long long total = (long long)n_g * N;
     const int threads = 128;
     prep_weights_kernel<<<(unsigned)((total + threads - 1) / threads), threads, 0, stream>>>(
         Wq, L->is_conv, C, N, G, L->R * L->S, L->perm, L->w8, L->w8m, L->w4, L->w4_pitch, L->sw);
     FLEXIQ_CUDA_TRY(cudaGetLastError());
-    FLEXIQ_CUDA_TRY(cudaMemcpyAsync(L->wf, L->w8, wbytes, cudaMemcpyDeviceToDevice, stream));  // all groups at 8 bits;
-    L->wf_K_lo = 0;                                                                             // the next mixed call brings the low groups along
+    L->st_K_lo = -1;   // the straddle block was cut from the previous order's weights
+    L->st_cap_id = 0;
+    L->slab_next = 0;  // slabs written for the previous order are no longer this layer's
+    memset(L->slab_seen, 0, sizeof(L->slab_seen));
     return FLEXIQ_OK;
 }
 
@@ -288,7 +353,7 @@ static int create_common(flexiq_layer_t *out, int is_conv, int C, int N, int R, 
     } while (0)
     TRY_OR_FREE(cudaMalloc(&L->w8, wbytes));
     TRY_OR_FREE(cudaMalloc(&L->w8m, wbytes));
-    TRY_OR_FREE(cudaMalloc(&L->wf, wbytes));
+    TRY_OR_FREE(cudaMalloc(&L->wst, (size_t)N * R * S * choose_bk(L)));
     TRY_OR_FREE(cudaMalloc(&L->w4, (size_t)N * L->w4_pitch));
     TRY_OR_FREE(cudaMemsetAsync(L->w4, 0, (size_t)N * L->w4_pitch, stream));
     TRY_OR_FREE(cudaMalloc(&L->sw, (size_t)n_g * N));
@@ -307,9 +372,8 @@ static int create_common(flexiq_layer_t *out, int is_conv, int C, int N, int R, 
     }
     TRY_OR_FREE(cudaMalloc(&L->w_scale, sizeof(float) * N));
     if (bias) TRY_OR_FREE(cudaMalloc(&L->bias, sizeof(float) * N));
-    TRY_OR_FREE(cudaMalloc(&L->alpha, sizeof(float) * N));
-    TRY_OR_FREE(cudaMalloc(&L->beta, sizeof(float) * N));
-    L->cache_mode = -1;
+    L->st_K_lo = -1;
+    L->slab_check = 1;
     TRY_OR_FREE(cudaMemcpyAsync(L->w_scale, w_scale, sizeof(float) * N, cudaMemcpyDeviceToDevice, stream));
     if (bias) TRY_OR_FREE(cudaMemcpyAsync(L->bias, bias, sizeof(float) * N, cudaMemcpyDeviceToDevice, stream));
     rc = layout_layer(L, Wq, perm, x_shift, stream);
@@ -358,7 +422,7 @@ int flexiq_layer_set_group_perm(flexiq_layer_t layer, const int8_t *Wq_dev, cons
     if (x_shift_host)
         for (int g = 0; g < L->n_g; ++g)
             if (x_shift_host[g] > 4) return set_error(FLEXIQ_ERR_INVALID_ARG, "x_shift_host[%d] = %d exceeds 4", g, x_shift_host[g]);
-    rc = check_device_sm100();
+    rc = check_layer_device(L);
     if (rc) return rc;
     return layout_layer(L, Wq_dev, group_perm_host, x_shift_host, reinterpret_cast<cudaStream_t>(stream));
 }
@@ -391,6 +455,14 @@ int flexiq_set_lowbit_ratio(flexiq_layer_t layer, float ratio)
     if (n_low < 0) n_low = 0;
     if (n_low > L->n_g) n_low = L->n_g;
     L->K_lo = n_low * L->G;
+    return FLEXIQ_OK;
+}
+
+int flexiq_layer_set_slab_check(flexiq_layer_t layer, int enabled)
+{
+    Layer *L = as_layer(layer);
+    if (!L) return set_error(FLEXIQ_ERR_INVALID_ARG, "not a live flexiq layer handle");
+    L->slab_check = enabled != 0;
     return FLEXIQ_OK;
 }
 

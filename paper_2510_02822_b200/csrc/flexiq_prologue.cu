@@ -9,6 +9,7 @@
 
 #include "sm100_ptx.cuh"
 #include "eq1_quantize.cuh"
+#include "straddle.cuh"
 
 #include <stdlib.h>
 
@@ -63,15 +64,6 @@ __global__ void group_or_kernel(const void *__restrict__ X, long long M, int K, 
         if (or_s[i]) atomicOr(&or_words[i], or_s[i]);
 }
 
-// Piggy-backed update of the masked path's weight operand: blocks from first_block on copy the
-// channel range [k_from, k_to) of each of `rows` = N * taps weight rows (row length C) from src.
-struct WeightPatch {
-    int8_t *wf;
-    const int8_t *src;
-    int rows, C, k_from, k_to;
-    unsigned first_block;  // = number of quantizing blocks; the grid is larger only when there is work
-};
-
 // Quantize + lower + gather.  Thread <-> (row m, 16-channel slab chunk c16).
 //   sx != nullptr : static positions (slab order);  else positions from or_words.
 // Lowering works on the packed int8 words: q is first clipped to the range the 4-bit value
@@ -83,7 +75,7 @@ __global__ void quantize_lower_kernel(const void *__restrict__ X, long long M, i
                                       const int32_t *__restrict__ perm, const uint8_t *__restrict__ sx,
                                       const unsigned *__restrict__ or_words, uint8_t *__restrict__ X4,
                                       long long x4_pitch, int8_t *__restrict__ X8, long long x8_pitch, uint8_t *__restrict__ sx_out,
-                                      WeightPatch wp)
+                                      StraddleJob wp)
 {
     const int n_c16 = K / 16, c_per_g = G / 16, lo_c16 = K_lo / 16;
     const long long total = M * n_c16;
@@ -91,14 +83,10 @@ __global__ void quantize_lower_kernel(const void *__restrict__ X, long long M, i
     ptx::pdl_launch_dependents();
     ptx::pdl_wait();  // the previous kernel may still read the slabs this one overwrites, or write X
     if (blockIdx.x >= wp.first_block) {
-        // Extra blocks behind the quantizing ones: bring the masked path's weight operand up to date
-        // with the ratio (only the channel groups that changed sides), 16 bytes per thread.
-        const int upt = (wp.k_to - wp.k_from) >> 4;
+        // Extra blocks behind the quantizing ones: the weight K block that max_4bit_ch falls into, for the
+        // GEMM that consumes these slabs (the only weight data that depends on the ratio), 16 bytes per thread.
         const long long idx = (long long)(blockIdx.x - wp.first_block) * blockDim.x + threadIdx.x;
-        if (idx < (long long)wp.rows * upt) {
-            const size_t off = (size_t)(idx / upt) * wp.C + wp.k_from + 16 * (int)(idx % upt);
-            *reinterpret_cast<uint4 *>(wp.wf + off) = *reinterpret_cast<const uint4 *>(wp.src + off);
-        }
+        if (idx < (long long)wp.rows * (wp.BK >> 4)) straddle_write_unit(wp, idx);
         return;
     }
     if (sx_out != nullptr && blockIdx.x == 0)
@@ -150,7 +138,7 @@ static int static_scratch_address(unsigned **out)
 {
     static unsigned *cached[64] = {};
     int dev = 0;
-    FLEXIQ_CUDA_TRY(cudaGetDevice(&dev));
+    FLEXIQ_CUDA_TRY(cudaGetDevice(&dev));   // the caller has checked that this is the layer's device
     if (dev < 0 || dev >= 64) return set_error(FLEXIQ_ERR_UNSUPPORTED, "device ordinal %d is beyond the 64 this entry point tracks", dev);
     if (cached[dev] == nullptr) {
         void *p = nullptr;
@@ -198,26 +186,29 @@ static int launch_prologue(Layer *L, const void *X, long long M, float S, int dy
     long long want = (M * n_c16 + threads - 1) / threads;
     long long blocks = want < (long long)sms * 16 ? want : (long long)sms * 16;
     const uint8_t *sx = dynamic ? nullptr : L->sx;
-    WeightPatch wp{};
+    StraddleJob wp{};
     wp.first_block = (unsigned)blocks;
     long long extra = 0;
     const bool masked = L->lowbit_path == FLEXIQ_LOWBIT_MASKED_I8;
-    if (masked && L->wf_K_lo != L->K_lo) {
-        // the GEMM that consumes these slabs needs the weight operand at the same ratio
-        wp.wf = L->wf;
-        wp.src = L->K_lo > L->wf_K_lo ? L->w8m : L->w8;
+    if (straddle_in_use(L) && straddle_stale(L, st)) {
+        // the GEMM that consumes these slabs reads the straddle block of the same max_4bit_ch
+        wp.wst = L->wst; wp.w8m = L->w8m; wp.w8 = L->w8;
         wp.rows = L->N * L->R * L->S;
         wp.C = L->C;
-        wp.k_from = L->K_lo < L->wf_K_lo ? L->K_lo : L->wf_K_lo;
-        wp.k_to = L->K_lo < L->wf_K_lo ? L->wf_K_lo : L->K_lo;
-        extra = ((long long)wp.rows * ((wp.k_to - wp.k_from) >> 4) + threads - 1) / threads;
+        wp.BK = choose_bk(L);
+        wp.blk0 = (L->K_lo / wp.BK) * wp.BK;
+        wp.K_lo = L->K_lo;
+        extra = ((long long)wp.rows * (wp.BK >> 4) + threads - 1) / threads;
     }
     const unsigned grid = (unsigned)(blocks + extra);
     if (!masked)
         FLEXIQ_CUDA_TRY(launch_pdl(quantize_lower_kernel<DTYPE, 1>, grid, threads, 0, st, X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, pitch8, dynamic ? sx_out : nullptr, wp));
     else
         FLEXIQ_CUDA_TRY(launch_pdl(quantize_lower_kernel<DTYPE, 0>, grid, threads, 0, st, X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, pitch8, dynamic ? sx_out : nullptr, wp));
-    if (extra) L->wf_K_lo = L->K_lo;
+    if (extra) straddle_written(L, st);
+    // remember at which max_4bit_ch these buffers were written (the mixed_* calls check it)
+    if (masked || L->K_lo > 0) record_slab(L, X4, L->K_lo);
+    if (!masked && L->K_lo < L->C) record_slab(L, X8, L->K_lo);
     return FLEXIQ_OK;
 }
 
@@ -249,6 +240,7 @@ extern "C" int flexiq_quantize_lower(flexiq_layer_t layer, const void *X_dev, in
         return set_error(FLEXIQ_ERR_INVALID_ARG, "X_dev, X4_dev and X8_dev must be 16-byte aligned");
     int rc = check_device_sm100();
     if (rc) return rc;
+    if ((rc = check_layer_device(L))) return rc;
     int64_t pitch = 0;
     flexiq_x4_pitch(layer, K_lo, &pitch);
     // masked path: one slab, low groups first, the 8-bit groups behind them in the same rows
@@ -273,8 +265,9 @@ extern "C" int flexiq_quantize_lower_dynamic_noalloc(flexiq_layer_t layer, const
         return set_error(FLEXIQ_ERR_INVALID_ARG,
                          "layer has %d channel groups; the built-in scratch of this entry point holds at most %d "
                          "(use flexiq_quantize_lower with caller-provided scratch instead)", L->n_g, kStaticScratchGroups);
-    unsigned *scratch = nullptr;
-    const int rc = static_scratch_address(&scratch);
+    int rc = check_layer_device(L);   // the array's address is per device: look it up on the layer's
     if (rc) return rc;
+    unsigned *scratch = nullptr;
+    if ((rc = static_scratch_address(&scratch))) return rc;
     return flexiq_quantize_lower(layer, X_dev, x_dtype, M, x_scale, 1, X4_dev, X8_dev, x_shift_out_dev, scratch, stream);
 }

@@ -59,6 +59,7 @@ extern "C" int flexiq_reorder_channels(flexiq_layer_t layer, const void *X_dev, 
         return set_error(FLEXIQ_ERR_INVALID_ARG, "X_dev and Y_dev must be 16-byte aligned");
     int rc = check_device_sm100();
     if (rc) return rc;
+    if ((rc = check_layer_device(L))) return rc;
     const int sms = device_sm_count(L->device);
     const int upr = L->C * elem_bytes / 16, upg = L->G * elem_bytes / 16;
     const long long total = (long long)M * upr;

@@ -150,7 +150,9 @@ def test_quantization_matches_ieee_division_near_ties(dev, S):
         lo = np.nextafter(lo, np.float32(-np.inf))
         vals.append(lo)
     rng = np.random.default_rng(7)
-    x = np.concatenate(vals + [rng.uniform(-140 * S, 140 * S, 4096).astype(np.float32)])
+    # ... and inputs beyond every finite quotient: Eq. 1's clip saturates them with their sign
+    huge = np.array([np.inf, -np.inf, 3.0e38, -3.0e38, 1e30, -1e30], np.float32)
+    x = np.concatenate(vals + [huge, rng.uniform(-140 * S, 140 * S, 4096).astype(np.float32)])
     K, G = 64, 16
     M = (x.size + K - 1) // K
     X = np.zeros((M, K), np.float32)
@@ -452,6 +454,102 @@ def test_cuda_graph_replay_matches_oracle(dev):
         assert np.array_equal(Y.cpu().numpy(), oracle.epilogue_i8(acc, case.x_scale, case.w_scale, case.bias, case.y_scale))
     fx.flexiq_check_status()
     L.close()
+
+
+def test_graph_captured_cold_then_eager_calls_then_replays(dev):
+    """Graphs captured with nothing warmed up (no earlier call at their ratio or scales), eager calls at other
+    ratios and scales in between, replays in scrambled order: every graph carries the ratio-dependent weight
+    block it needs, and eager calls never trust state that a replay may have rewritten."""
+    case = inputs.ranged_linear("gc", 300, 384, 272, 16, seed=27, group_structured=True)
+    perm, sxg, sxs, sw = helpers.prepare_linear(case)
+    L = _layer(case, dev, perm, sxg)
+    X = torch.from_numpy(case.X).to(dev)
+    q = oracle.quantize(case.X, case.x_scale)
+
+    def want(r, y_scale):
+        acc = oracle.mixed_gemm_acc(q, case.Wq, case.G, perm, sxs, sw, oracle.n_low(r, case.K // case.G))
+        return oracle.epilogue_i8(acc, case.x_scale, case.w_scale, case.bias, y_scale)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graphs = {}
+    with torch.cuda.stream(side):
+        for r in (0.25, 0.75, 1.0 / 3.0):   # max_4bit_ch 96, 288, 128: two fall inside a K block of 128, one on its edge
+            L.set_lowbit_ratio(r)
+            x4 = torch.empty(case.M * case.K + 16, dtype=torch.uint8, device=dev)
+            Y = torch.empty((case.M, case.N), dtype=torch.int8, device=dev)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                fx.flexiq_quantize_lower(L.h, X, fx.DTYPE_F32, case.M, case.x_scale, 0, x4, None)
+                fx.flexiq_mixed_gemm(L.h, x4, None, None, case.M, case.x_scale, case.y_scale, fx.OUT_REQUANT_I8, Y)
+            graphs[r] = (g, Y, x4)
+        # a graph that holds only the GEMM, on a slab written eagerly beforehand
+        L.set_lowbit_ratio(0.5)
+        x4e = torch.empty(case.M * case.K + 16, dtype=torch.uint8, device=dev)
+        Ye = torch.empty((case.M, case.N), dtype=torch.int8, device=dev)
+        fx.flexiq_quantize_lower(L.h, X, fx.DTYPE_F32, case.M, case.x_scale, 0, x4e, None)
+        side.synchronize()
+        ge = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(ge, stream=side):
+            fx.flexiq_mixed_gemm(L.h, x4e, None, None, case.M, case.x_scale, case.y_scale, fx.OUT_REQUANT_I8, Ye)
+        graphs[0.5] = (ge, Ye, x4e)
+    torch.cuda.synchronize()
+    ys2 = float(np.float32(case.y_scale * 1.7))
+    for r in (0.75, 0.25, 0.5, 1.0 / 3.0, 0.25, 0.5, 0.75):
+        # an eager call at another ratio and another output scale first
+        r_e = 0.625 if r != 0.5 else 0.125
+        L.set_lowbit_ratio(r_e)
+        x4, x8, _ = L.quantize_lower(X, case.x_scale)
+        y = L.mixed_gemm(x4, x8, case.M, case.x_scale, ys2, fx.OUT_REQUANT_I8)
+        torch.cuda.synchronize()
+        assert np.array_equal(y.cpu().numpy(), want(r_e, ys2)), f"eager call at {r_e}"
+        g, Y, _ = graphs[r]
+        Y.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(Y.cpu().numpy(), want(r, case.y_scale)), f"replay at {r}"
+        # and an eager GEMM on the slab the eager prologue wrote before the replay
+        y = L.mixed_gemm(x4, x8, case.M, case.x_scale, ys2, fx.OUT_REQUANT_I8)
+        torch.cuda.synchronize()
+        assert np.array_equal(y.cpu().numpy(), want(r_e, ys2)), f"eager GEMM after the replay at {r}"
+    fx.flexiq_check_status()
+    L.close()
+
+
+def test_slab_written_at_another_ratio_is_refused(dev):
+    """A mixed_* call on a slab buffer that the handle saw written at another max_4bit_ch returns an error instead
+    of wrong values (masked path) or a read past the end of the buffer (packed path); slabs of several ratios
+    prepared ahead in buffers of their own are fine; the check can be switched off."""
+    case = inputs.ranged_linear("sr", 200, 256, 64, 16, seed=28, group_structured=True)
+    perm, sxg, sxs, sw = helpers.prepare_linear(case)
+    q = oracle.quantize(case.X, case.x_scale)
+    for path in (fx.LOWBIT_MASKED_I8, fx.LOWBIT_PACKED_U4):
+        L = _layer(case, dev, perm, sxg, path=path)
+        X = torch.from_numpy(case.X).to(dev)
+        slabs = {}
+        for r in (0.25, 0.75):
+            L.set_lowbit_ratio(r)
+            bufs = (torch.empty(case.M * case.K + 16, dtype=torch.uint8, device=dev), torch.empty(case.M * case.K + 16, dtype=torch.int8, device=dev))
+            L.quantize_lower(X, case.x_scale, slabs=bufs)
+            slabs[r] = bufs
+        for r_set, r_slab in ((0.25, 0.75), (0.75, 0.25), (1.0, 0.25), (0.0, 0.75)):
+            L.set_lowbit_ratio(r_set)
+            with pytest.raises(fx.FlexiqError) as e:
+                L.mixed_gemm(*slabs[r_slab], case.M, case.x_scale, case.y_scale, fx.OUT_ACC_I32)
+            assert e.value.code == fx.ERR_INVALID_ARG and "max_4bit_ch" in str(e.value)
+        for r in (0.75, 0.25):   # each buffer at its own ratio, in any order
+            L.set_lowbit_ratio(r)
+            acc = L.mixed_gemm(*slabs[r], case.M, case.x_scale, case.y_scale, fx.OUT_ACC_I32)
+            torch.cuda.synchronize()
+            assert np.array_equal(acc.cpu().numpy(), oracle.mixed_gemm_acc(q, case.Wq, case.G, perm, sxs, sw, oracle.n_low(r, case.K // case.G)))
+        if path == fx.LOWBIT_MASKED_I8:   # opt-out (masked slabs have the same shape at every ratio: no overrun)
+            fx.flexiq_layer_set_slab_check(L.h, False)
+            L.set_lowbit_ratio(0.25)
+            L.mixed_gemm(*slabs[0.75], case.M, case.x_scale, case.y_scale, fx.OUT_ACC_I32)
+            fx.flexiq_layer_set_slab_check(L.h, True)
+        torch.cuda.synchronize()
+        fx.flexiq_check_status()
+        L.close()
 
 
 def test_two_layers_on_two_streams(dev):

@@ -4,7 +4,7 @@ Some callers cannot call cudaMalloc where they run the prologue (a stream being 
 a CUDA graph, an allocator hook, a serving loop that owns no spare device memory), so they
 cannot provide the scratch words the regular dynamic-position call needs.  The entry point
 tested here uses a fixed array inside the library instead.  It must give exactly the slabs and
-positions of the regular entry point, on two calls in a row (the array keeps the previous
+positions of the regular entry point -- and of the CPU oracle -- on two calls in a row (the array keeps the previous
 call's contents, so the second call proves that it is cleared), and it must refuse layers
 with more channel groups than the array holds.
 
@@ -14,16 +14,21 @@ import numpy as np
 import pytest
 import torch
 
+import helpers
+import oracle
 from paper_2510_02822_b200 import binding as fx
 from paper_2510_02822_b200 import inputs
 
 pytestmark = pytest.mark.gpu
 
 
+def _perm(case, G):
+    return np.random.default_rng(case.K).permutation(case.K // G).astype(np.int32)
+
+
 def _layer(case, dev, G):
     n_g = case.K // G
-    rng = np.random.default_rng(case.K)
-    perm = rng.permutation(n_g).astype(np.int32)
+    perm = _perm(case, G)
     return fx.Layer(torch.from_numpy(case.Wq).to(dev), torch.from_numpy(case.w_scale).to(dev), None, perm,
                     np.zeros(n_g, np.uint8), G)
 
@@ -58,6 +63,22 @@ def test_noalloc_entry_point_matches_regular_entry_point_twice(path):
         got = _run(L, case, X, "noalloc", dev)
         for r, g in zip(ref, got):
             assert np.array_equal(r, g)
+        # and against the oracle: positions from the OR over the call's own values, slabs lowered with them
+        M, K, G = case.M, case.K, 16
+        perm = _perm(big, G)
+        q = oracle.quantize(case.X, case.x_scale)
+        sx = oracle.dynamic_positions(q, G, perm)
+        assert np.array_equal(got[2], sx)
+        nl = oracle.n_low(0.75, K // G)
+        e4, e8 = oracle.make_slabs(q, G, perm, sx, nl)
+        if path == fx.LOWBIT_MASKED_I8:
+            slab = got[0][:M * K].reshape(M, K).view(np.int8)
+            assert np.array_equal(slab[:, :nl * G], helpers.masked_slab(e4, G, sx, nl))
+            assert np.array_equal(slab[:, nl * G:], e8)
+        else:
+            pitch = fx.flexiq_x4_pitch(L.h, nl * G)
+            assert np.array_equal(got[0][:M * pitch].reshape(M, pitch)[:, :nl * G // 2], e4[:, :nl * G // 2])
+            assert np.array_equal(got[1][:M * (K - nl * G)].reshape(M, K - nl * G), e8)
     # the second input is much smaller, so its positions must be smaller too (nothing left over)
     assert _run(L, small, torch.from_numpy(small.X).to(dev), "noalloc", dev)[2].max() <= 1
     L.close()
