@@ -65,9 +65,8 @@ struct GemmParams {
     int im2col;          // A operand through im2col-mode TMA
     int P, Q, stride, pad;
     int out_mode;
-    const float *w_scale;  // [N] per-output-channel weight scales
-    const float *bias;     // [N] or nullptr
-    float x_scale, y_scale;
+    const float *alpha;  // [N] per-output-channel multiplier of this call
+    const float *beta;   // [N] per-output-channel addend of this call
     void *Y;
     int m_tiles, n_tiles;
     // fused layer boundary only: where each 16-channel chunk of the output lands in the next layer's slab
@@ -317,14 +316,8 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
     const int cols = BN >= 192 ? 64 : 32;
     const bool y32 = (reinterpret_cast<uintptr_t>(p.Y) & 31) == 0;
     const bool wide = y32 && (p.N & 31) == 0;    // int8 rows are 32-byte aligned: 256-bit stores
-    // Per-output-channel factors, computed here from the layer's scales (each operation rounds once, in fp32):
-    //   re-quantizing modes  alpha = (S_x * S_w[n]) / S_y,  beta = bias[n] / S_y
-    //   floating-point modes alpha = S_x * S_w[n],          beta = bias[n]
-    // Lanes 0-15 build alpha, lanes 16-31 beta; lane l keeps factors 4l..4l+3 of the table alpha[64] | beta[64].
-    constexpr bool kRequant = MODE == FLEXIQ_OUT_REQUANT_I8 || MODE == kOutNextSlab;
-    const float *fsrc = (lane < 16 ? p.w_scale : p.bias);
-    if (fsrc) fsrc += 4 * (lane & 15);
-    const float fmul = lane < 16 ? p.x_scale : 1.0f;   // multiplying by 1 is exact
+    // lane l keeps factors 4l..4l+3 of the table alpha[64] | beta[64]
+    const float *fsrc = (lane < 16 ? p.alpha : p.beta) + 4 * (lane & 15);
     int buf = 0;
     uint32_t buf_phase = 0;
     PROF_DECL(prof_wait);
@@ -355,14 +348,7 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                 continue;
             }
             float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (kScaled && fsrc && nw + 4 * (lane & 15) < p.N) {
-                f = __ldg(reinterpret_cast<const float4 *>(fsrc + nw));
-                f.x = __fmul_rn(fmul, f.x); f.y = __fmul_rn(fmul, f.y); f.z = __fmul_rn(fmul, f.z); f.w = __fmul_rn(fmul, f.w);
-                if (kRequant) {
-                    f.x = __fdiv_rn(f.x, p.y_scale); f.y = __fdiv_rn(f.y, p.y_scale);
-                    f.z = __fdiv_rn(f.z, p.y_scale); f.w = __fdiv_rn(f.w, p.y_scale);
-                }
-            }
+            if (kScaled && nw + 4 * (lane & 15) < p.N) f = __ldg(reinterpret_cast<const float4 *>(fsrc + nw));
             int ent = 0;                                     // fused boundary: lane g fetches chunk g's slab entry
             if (MODE == kOutNextSlab && lane < 4 && nw + 16 * lane < p.N) ent = __ldg(p.next_ent + (nw >> 4) + lane);
             if (!waited) {
@@ -1134,6 +1120,20 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
     }
 }
 
+// Per-output-channel factors of a call: REQUANT alpha = (S_x * S_w[n]) / S_y, beta = bias[n] / S_y;
+// DEQUANT alpha = S_x * S_w[n], beta = bias[n].  Each operation rounds once, in fp32.
+__global__ void scale_vectors_kernel(int N, float x_scale, float y_scale, int requant, const float *__restrict__ w_scale,
+                                     const float *__restrict__ bias, float *__restrict__ alpha, float *__restrict__ beta)
+{
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    ptx::pdl_wait();  // the previous kernel of the stream may still read the table
+    if (n >= N) return;
+    const float sxw = __fmul_rn(x_scale, w_scale[n]);
+    const float bv = bias ? bias[n] : 0.f;
+    alpha[n] = requant ? __fdiv_rn(sxw, y_scale) : sxw;
+    beta[n] = requant ? __fdiv_rn(bv, y_scale) : bv;
+}
+
 // The straddle block of the masked path (straddle.cuh) for a GEMM that no prologue launch precedes.
 __global__ void straddle_kernel(const StraddleJob job)
 {
@@ -1337,7 +1337,42 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     }
     p.out_mode = out_mode; p.Y = Y;
     if (next) { p.next_ent = out_order == FLEXIQ_ORDER_NEXT_SLAB ? next->chunk_ent_slab : next->chunk_ent; p.next_K_lo = next->K_lo; p.relu = relu != 0; }
-    p.w_scale = L->w_scale; p.bias = L->bias; p.x_scale = x_scale; p.y_scale = y_scale;
+    // The per-output-channel factors depend on the call's scales.  The handle keeps a few factor tables, each
+    // written once for one (kind, S_x, S_y) and never changed while anything may still depend on it, so a
+    // table that a captured graph reads (or writes) stays what that graph expects whatever runs in between.
+    // The fused boundary re-quantizes with the REQUANT factors; the three floating-point outputs share theirs.
+    const int fmode = next ? FLEXIQ_OUT_REQUANT_I8
+                           : ((out_mode == FLEXIQ_OUT_DEQUANT_F16 || out_mode == FLEXIQ_OUT_DEQUANT_BF16) ? FLEXIQ_OUT_DEQUANT_F32 : out_mode);
+    if (fmode != FLEXIQ_OUT_ACC_I32) {
+        const unsigned long long cap = stream_capture_id(st);
+        const float ys_key = fmode == FLEXIQ_OUT_REQUANT_I8 ? y_scale : 0.0f;
+        Layer::FactorTable *ft = nullptr;
+        for (int i = 0; i < Layer::kFactorTables && !ft; ++i)
+            if (L->factors[i].keyed && L->factors[i].mode == fmode && L->factors[i].xs == x_scale && L->factors[i].ys == ys_key) ft = &L->factors[i];
+        if (!ft) {
+            // a table nothing captured depends on, taken in turn; failing that the scratch table, rewritten by every call
+            for (int k = 0; k < Layer::kFactorTables && !ft; ++k) {
+                Layer::FactorTable *c = &L->factors[(L->factor_next + k) % Layer::kFactorTables];
+                if (!c->pinned) { ft = c; L->factor_next = (int)(c - L->factors + 1) % Layer::kFactorTables; }
+            }
+            if (!ft) ft = &L->factors[Layer::kFactorTables];
+            ft->mode = fmode; ft->xs = x_scale; ft->ys = ys_key;
+            ft->keyed = ft != &L->factors[Layer::kFactorTables];   // the scratch table is never found again
+            ft->on_device = 0; ft->cap_id = 0;
+        }
+        // The values are on the device for this call when an eager call wrote them (they then stay: a keyed table is
+        // only ever rewritten with the same values) or when this very capture already holds the write.  A write that
+        // only another captured graph holds does not count: that graph may never have run.
+        if (!(ft->on_device || (cap && ft->cap_id == cap))) {
+            scale_vectors_kernel<<<(L->N + 255) / 256, 256, 0, st>>>(L->N, x_scale, y_scale, fmode == FLEXIQ_OUT_REQUANT_I8,
+                                                                     L->w_scale, L->bias, ft->alpha, ft->beta);
+            FLEXIQ_CUDA_TRY(cudaGetLastError());
+            if (cap) ft->cap_id = cap;
+            else ft->on_device = ft->keyed;
+        }
+        if (cap && ft->keyed) ft->pinned = 1;   // a graph now reads (or rewrites) this table with these values
+        p.alpha = ft->alpha; p.beta = ft->beta;
+    }
     TileChoice tc = g_forced_tile.cg ? g_forced_tile : choose_tile(M, L->N, p.T * (p.nb_lo + p.nb_hi), p.BK, sms);
     if (packed && tc.cg == 2) {  // the packed path runs single CTAs: re-choose among those
         tc.cg = 1;

@@ -69,6 +69,22 @@ struct Layer {
     uint8_t *sx_host;
     // tensor maps over the weights (encoded once)
     CUtensorMap map_w8[kNumWeightMaps], map_w4[kNumWeightMaps], map_w8m[kNumWeightMaps], map_wst[kNumWeightMaps];  // one per box height
+    // Per-output-channel epilogue factors.  Each table is written for one (kind of output, S_x, S_y) and
+    // then only read; a table that a captured CUDA graph reads or writes is pinned to its key for good, so
+    // graph replays and eager calls cannot invalidate each other's factors.  The last table is scratch:
+    // used (and rewritten by every call) only when all others are pinned to other keys.
+    static constexpr int kFactorTables = 4;
+    struct FactorTable {
+        float *alpha, *beta;
+        float xs, ys;
+        int mode;
+        int keyed;                  // the key above is in force (always 0 for the scratch table)
+        int on_device;              // an eager call has written the values
+        int pinned;                 // a captured graph depends on the table keeping this key
+        unsigned long long cap_id;  // capture sequence that holds a write of the values
+    } factors[kFactorTables + 1];
+    int factor_next;
+    float *factor_mem;   // one allocation behind all tables
     int w4_pitch;    // row pitch of w4 in bytes: Kw/2 rounded up to 16
     // tensor maps of the most recent masked-path call, reused while the caller passes the same buffers
     // and shapes (encoding three maps costs more host time than the rest of a small call)

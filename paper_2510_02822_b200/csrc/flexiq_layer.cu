@@ -251,7 +251,7 @@ static void free_layer(Layer *L)
     if (!L) return;
     if (L->tables_in_flight) cudaEventSynchronize(L->tables_event);
     cudaFree(L->w8); cudaFree(L->w8m); cudaFree(L->w4); cudaFree(L->wst); cudaFree(L->sw);
-    cudaFree(L->tables); cudaFree(L->w_scale); cudaFree(L->bias);
+    cudaFree(L->tables); cudaFree(L->w_scale); cudaFree(L->bias); cudaFree(L->factor_mem);
     if (L->tables_host) cudaFreeHost(L->tables_host);
     if (L->tables_event) cudaEventDestroy(L->tables_event);
     free(L->perm_host); free(L->sx_host);
@@ -374,6 +374,11 @@ static int create_common(flexiq_layer_t *out, int is_conv, int C, int N, int R, 
     if (bias) TRY_OR_FREE(cudaMalloc(&L->bias, sizeof(float) * N));
     L->st_K_lo = -1;
     L->slab_check = 1;
+    TRY_OR_FREE(cudaMalloc(&L->factor_mem, sizeof(float) * 2 * (size_t)N * (Layer::kFactorTables + 1)));
+    for (int i = 0; i <= Layer::kFactorTables; ++i) {
+        L->factors[i].alpha = L->factor_mem + (size_t)2 * N * i;
+        L->factors[i].beta = L->factors[i].alpha + N;
+    }
     TRY_OR_FREE(cudaMemcpyAsync(L->w_scale, w_scale, sizeof(float) * N, cudaMemcpyDeviceToDevice, stream));
     if (bias) TRY_OR_FREE(cudaMemcpyAsync(L->bias, bias, sizeof(float) * N, cudaMemcpyDeviceToDevice, stream));
     rc = layout_layer(L, Wq, perm, x_shift, stream);

@@ -82,24 +82,37 @@ __global__ void quantize_lower_kernel(const void *__restrict__ X, long long M, i
     const Divider div = make_divider(S);
     ptx::pdl_launch_dependents();
     ptx::pdl_wait();  // the previous kernel may still read the slabs this one overwrites, or write X
-    if (blockIdx.x >= wp.first_block) {
-        // Extra blocks behind the quantizing ones: the weight K block that max_4bit_ch falls into, for the
-        // GEMM that consumes these slabs (the only weight data that depends on the ratio), 16 bytes per thread.
-        const long long idx = (long long)(blockIdx.x - wp.first_block) * blockDim.x + threadIdx.x;
+    if (blockIdx.x < wp.first_block) {
+        // Extra blocks in front of the quantizing ones (so that they run beside the first wave, not behind the
+        // last): the weight K block that max_4bit_ch falls into, for the GEMM that consumes these slabs -- the
+        // only weight data that depends on the ratio -- 16 bytes per thread.
+        const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
         if (idx < (long long)wp.rows * (wp.BK >> 4)) straddle_write_unit(wp, idx);
         return;
     }
-    if (sx_out != nullptr && blockIdx.x == 0)
+    const unsigned qblock = blockIdx.x - wp.first_block, qblocks = gridDim.x - wp.first_block;
+    if (sx_out != nullptr && qblock == 0)
         for (int j = threadIdx.x; j < K / G; j += blockDim.x) sx_out[j] = (uint8_t)position_from_or(or_words[j]);
-    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-         idx += (long long)wp.first_block * blockDim.x) {
+    for (long long idx = (long long)qblock * blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)qblocks * blockDim.x) {
         const long long m = idx / n_c16;
         const int c16 = (int)(idx - m * n_c16);
         const int j = c16 / c_per_g;
         const int src_c = perm[j] * G + (c16 % c_per_g) * 16;
         const void *src = reinterpret_cast<const char *>(X) + ((size_t)m * K + src_c) * elem_bytes<DTYPE>();
         unsigned w[4];
-        if (c16 < lo_c16) {
+        if (!PACKED) {
+            // Masked path: one instruction stream for both kinds of group (a warp spans the boundary in most rows).
+            // A low group keeps bits s..s+3 of values clipped to what four bits hold at position s; an 8-bit group
+            // is the same with the full range and nothing cleared.  The slab is [M][K]: X8 is X4 + K_lo.
+            const bool low = c16 < lo_c16;
+            const int s = low ? (sx ? (int)sx[j] : position_from_or(or_words[j])) : 4;
+            const float bound = (float)(8 << s);
+            quantize16<DTYPE>(src, div, -bound, bound - 1.f, w);
+            const unsigned mask = low ? ((0xffu << s) & 0xffu) * 0x01010101u : 0xffffffffu;
+            *reinterpret_cast<uint4 *>(X4 + m * x4_pitch + (size_t)c16 * 16) =
+                make_uint4(w[0] & mask, w[1] & mask, w[2] & mask, w[3] & mask);
+        } else if (c16 < lo_c16) {
             const int s = sx ? (int)sx[j] : position_from_or(or_words[j]);
             const float bound = (float)(8 << s);
             quantize16<DTYPE>(src, div, -bound, bound - 1.f, w);
@@ -187,7 +200,6 @@ static int launch_prologue(Layer *L, const void *X, long long M, float S, int dy
     long long blocks = want < (long long)sms * 16 ? want : (long long)sms * 16;
     const uint8_t *sx = dynamic ? nullptr : L->sx;
     StraddleJob wp{};
-    wp.first_block = (unsigned)blocks;
     long long extra = 0;
     const bool masked = L->lowbit_path == FLEXIQ_LOWBIT_MASKED_I8;
     if (straddle_in_use(L) && straddle_stale(L, st)) {
@@ -200,6 +212,7 @@ static int launch_prologue(Layer *L, const void *X, long long M, float S, int dy
         wp.K_lo = L->K_lo;
         extra = ((long long)wp.rows * (wp.BK >> 4) + threads - 1) / threads;
     }
+    wp.first_block = (unsigned)extra;   // the straddle blocks come first
     const unsigned grid = (unsigned)(blocks + extra);
     if (!masked)
         FLEXIQ_CUDA_TRY(launch_pdl(quantize_lower_kernel<DTYPE, 1>, grid, threads, 0, st, X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, pitch8, dynamic ? sx_out : nullptr, wp));

@@ -19,7 +19,7 @@ struct StraddleJob {
     int C, BK;
     int blk0;              // first channel of the straddle block
     int K_lo;              // max_4bit_ch
-    unsigned first_block;  // prologue launches: number of quantizing blocks in front of the straddle blocks
+    unsigned first_block;  // prologue launches: number of straddle blocks, which come in front of the quantizing blocks
 };
 
 // one 16-byte unit of the straddle block; idx < rows * (BK / 16)

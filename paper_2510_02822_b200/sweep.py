@@ -46,12 +46,17 @@ def _alg_bytes(case, is_conv, ratio, Mout):
     return Min * K * (1 - rho / 2) + taps * K * N * (1 - rho / 2) + n_low * N + 8 * N + Mout * N
 
 
-def time_case(case, is_conv, dev, path, iters, cold, flush, graph=False):
+def _say(quiet, obj):
+    if not quiet:
+        print(json.dumps(obj), flush=True)
+
+
+def time_case(case, is_conv, dev, path, iters, cold, flush, graph=False, ratios=None, quiet=False):
     L = _layer_for(case, dev, is_conv, path)
     X = torch.from_numpy(case.X).to(dev)
     stream = torch.cuda.current_stream()
     rows = []
-    for r in RATIOS:
+    for r in (RATIOS if ratios is None else ratios):
         L.set_lowbit_ratio(r)
         x4, x8, _ = L.quantize_lower(X, case.x_scale)
 
@@ -118,17 +123,23 @@ def time_case(case, is_conv, dev, path, iters, cold, flush, graph=False):
             tp, tg = e[0].elapsed_time(e[1]) / iters, e[1].elapsed_time(e[2]) / iters
         rows.append({"layer": case.name, "ratio": r, "path": "packed" if path else "masked", "cold": bool(cold), "graph": bool(graph),
                      "prologue_us": round(tp * 1e3, 2), "mixed_us": round(tg * 1e3, 2),
-                     "mixed_tops": round(ops / tg / 1e9, 1), "mixed_alg_gbs": round(_alg_bytes(case, is_conv, r, Mout) / tg / 1e6, 1)})
-        print(json.dumps(rows[-1]), flush=True)
+                     "mixed_tops": round(ops / tg / 1e9, 1), "mixed_alg_gbs": round(_alg_bytes(case, is_conv, r, Mout) / tg / 1e6, 1),
+                     "ops": ops, "alg_bytes": _alg_bytes(case, is_conv, r, Mout)})
+        _say(quiet, rows[-1])
     fx.flexiq_check_status()
     L.close()
     return rows
 
 
-def run_stack(dev, batch, iters):
+def run_stack(dev, batch, iters, quiet=False):
     """ViT-L/16 stack of linears: every layer's prologue + mixed GEMM in sequence, the ratio switched
-    between passes with flexiq_set_lowbit_ratio (no re-packing, no re-allocation)."""
+    between passes with flexiq_set_lowbit_ratio (no re-packing, no re-allocation).  Also: the mixed GEMM
+    alone per layer shape (the 24 blocks' layers of that shape in turn, so that no weights stay in L2), and
+    the device time of a ratio switch.  The activations are a seeded block of M / 8 rows repeated eight times
+    (the time does not depend on the values; drawing 130 million numbers on the host would take longer than
+    the measurement).  Returns the rows it prints."""
     M = batch * 197
+    out = []
     layers, meta = [], []
     t0 = time.time()
     Xs = {}
@@ -140,11 +151,12 @@ def run_stack(dev, batch, iters):
             layers.append(L)
             meta.append((K, N, c.x_scale, c.y_scale))
             if K not in Xs:
-                big = inputs.vit_linear("x", M, K, 16, 16, seed=5900 + K)
-                Xs[K] = torch.from_numpy(big.X).to(dev)
+                rows_drawn = (M + 7) // 8
+                big = inputs.vit_linear("x", rows_drawn, K, 16, 16, seed=5900 + K)
+                Xs[K] = torch.from_numpy(big.X).to(dev).repeat(8, 1)[:M].contiguous()
     slabs = {K: (torch.empty(M * K + 16, dtype=torch.uint8, device=dev), torch.empty(M * K + 16, dtype=torch.int8, device=dev)) for K in Xs}
     Ys = {N: torch.empty((M, N), dtype=torch.int8, device=dev) for N in {n for _, n, _, _ in meta}}
-    print(json.dumps({"setup_s": round(time.time() - t0, 1), "layers": len(layers), "M": M}), flush=True)
+    _say(quiet, {"setup_s": round(time.time() - t0, 1), "layers": len(layers), "M": M})
     ops = sum(2.0 * M * K * N for K, N, _, _ in meta)
     stream = torch.cuda.current_stream()
 
@@ -174,13 +186,79 @@ def run_stack(dev, batch, iters):
     for ratio in (0.0, 0.5, 1.0):
         ms = sum(m for m, _ in acc[ratio]) / len(acc[ratio])
         switch_us = sum(u for _, u in acc[ratio]) / len(acc[ratio])
-        print(json.dumps({"config": 5, "ratio": ratio, "pass_ms": round(ms, 3), "pass_ms_up_down": [round(m, 3) for m, _ in acc[ratio]],
-                          "pass_tops_prologue_plus_gemm": round(ops / ms / 1e9, 1),
-                          "ratio_switch_us_all_96_layers": round(switch_us, 1)}), flush=True)
+        out.append({"config": 5, "ratio": ratio, "pass_ms": round(ms, 3), "pass_ms_up_down": [round(m, 3) for m, _ in acc[ratio]],
+                    "pass_tops_prologue_plus_gemm": round(ops / ms / 1e9, 1),
+                    "ratio_switch_host_us_all_96_layers": round(switch_us, 1)})
+        _say(quiet, out[-1])
+    # the mixed GEMM alone, per layer shape and ratio: slabs written once, then the 24 layers of the shape in turn
+    for si, (name, K, N) in enumerate(inputs.VIT_L_LAYERS):
+        same = [L for i, L in enumerate(layers) if i % 4 == si]
+        xs, ys = meta[si][2], meta[si][3]
+        for ratio in (0.0, 0.5, 1.0):
+            for L in same:
+                L.set_lowbit_ratio(ratio)
+            x4, x8 = slabs[K]
+            fx.flexiq_quantize_lower(same[0].h, Xs[K], fx.DTYPE_F32, M, xs, 0, x4, x8)
+            for L in same:
+                fx.flexiq_layer_set_slab_check(L.h, False)   # one slab (same group order is not required for timing) feeds all 24
+                fx.flexiq_mixed_gemm(L.h, x4, x8, None, M, xs, ys, fx.OUT_REQUANT_I8, Ys[N])
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(iters):
+                for L in same:
+                    fx.flexiq_mixed_gemm(L.h, x4, x8, None, M, xs, ys, fx.OUT_REQUANT_I8, Ys[N])
+            e1.record(stream)
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) / (iters * len(same)) * 1e3
+            out.append({"config": 5, "gemm_only": name, "K": K, "N": N, "ratio": ratio, "us": round(us, 2),
+                        "tops": round(2.0 * M * K * N / us / 1e6, 1)})
+            _say(quiet, out[-1])
+        for L in same:
+            fx.flexiq_layer_set_slab_check(L.h, True)
+    # Device time of a ratio switch: everything flexiq_layer_sync_ratio enqueues for the 96 layers, captured in one
+    # CUDA graph and replayed (launched from the host the 96 calls take longer than their kernels run).  At 0 / 50 /
+    # 100 % max_4bit_ch is a multiple of the K block in every layer, so nothing is enqueued at all; 30 % falls
+    # inside a block.  In a running model the write rides in the next prologue launch instead.
+    for frm, to in ((0.0, 0.5), (0.5, 1.0), (1.0, 0.3), (0.3, 0.0)):
+        t_sw = time.perf_counter()
+        for L in layers:
+            L.set_lowbit_ratio(to)
+        host_us = (time.perf_counter() - t_sw) * 1e6
+        moved = sum(N * 128 for K, N, _, _ in meta if (oracle_free_n_low(to, K // 16) * 16) % 128 != 0)
+        dev_us = 0.0
+        if moved:
+            g = torch.cuda.CUDAGraph()
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(g, stream=side):
+                    for L in layers:
+                        L.sync_ratio()
+            torch.cuda.synchronize()
+            g.replay()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(5):
+                g.replay()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            dev_us = e0.elapsed_time(e1) / 5 * 1e3
+        out.append({"config": 5, "switch": f"{frm} -> {to}", "device_us_all_96_layers": round(dev_us, 1), "kernels_enqueued": 96 if moved else 0,
+                    "host_us_all_96_layers": round(host_us, 1), "weight_bytes_written": moved})
+        _say(quiet, out[-1])
     fx.flexiq_check_status()
+    for L in layers:
+        L.close()
+    return out
 
 
-def run_deit_stack(dev, batch, replicas, iters):
+def oracle_free_n_low(ratio, n_g):
+    """Number of low-bit groups the library derives from a ratio (same rounding rule), for reporting only."""
+    import math
+    return max(0, min(n_g, math.ceil(float(np.float32(ratio)) * n_g - 1e-4)))
+
+
+def run_deit_stack(dev, batch, replicas, iters, quiet=False):
     """DeiT-S stack of linears (12 blocks x 4 layers = 48 layer instances, each with its own weights,
     input and output) captured in ONE CUDA graph per replica; `replicas` distinct copies of the whole
     stack are replayed in turn so that nothing a replay touches is still in L2 from the previous time
@@ -205,11 +283,12 @@ def run_deit_stack(dev, batch, replicas, iters):
                 x4 = torch.empty(M * K + 16, dtype=torch.uint8, device=dev)
                 Y = torch.empty((M, N), dtype=torch.int8, device=dev)
                 inst.append((L, c, X, x4, Y))
-                total_bytes += 4 * K * N + M * K * 5 + M * N  # w8, w8m, wf, w4 ~ 3.5 K N; X fp32 + slab; Y
+                total_bytes += int(2.5 * K * N) + M * K * 5 + M * N  # w8, w8m, w4; X fp32 + slab; Y
         stacks.append(inst)
     alg = sum(c.M * c.K * 4 + 2 * c.M * c.K + c.K * c.N + 8 * c.N + c.M * c.N for _, c, _, _, _ in stacks[0])
-    print(json.dumps({"setup_s": round(time.time() - t0, 1), "replicas": replicas, "instances": replicas * 48, "M": M,
-                      "resident_MB": round(total_bytes / 1e6, 1), "algorithmic_MB_per_pass": round(alg / 1e6, 2)}), flush=True)
+    out = [{"setup_s": round(time.time() - t0, 1), "replicas": replicas, "instances": replicas * 48, "M": M,
+            "resident_MB": round(total_bytes / 1e6, 1), "algorithmic_MB_per_pass": round(alg / 1e6, 2)}]
+    _say(quiet, out[-1])
     stream = torch.cuda.current_stream()
 
     def one_pass(inst):
@@ -222,7 +301,7 @@ def run_deit_stack(dev, batch, replicas, iters):
         for inst in stacks:
             for L, *_ in inst:
                 L.set_lowbit_ratio(ratio)
-            one_pass(inst)  # weight operands move to this ratio outside the capture
+            one_pass(inst)
             torch.cuda.synchronize()
             g = torch.cuda.CUDAGraph()
             side = torch.cuda.Stream()
@@ -245,9 +324,14 @@ def run_deit_stack(dev, batch, replicas, iters):
             torch.cuda.synchronize()
             us = e0.elapsed_time(e1) / (iters * len(order)) * 1e3
             res[label] = {"pass_us": round(us, 1), "us_per_layer": round(us / 48, 2), "alg_gbs": round(alg / us / 1e3, 1)}
-        print(json.dumps({"config": 4, "protocol": "48-layer graph per replica", "batch": batch, "ratio": ratio, **res}), flush=True)
+        out.append({"config": 4, "protocol": "48-layer graph per replica", "batch": batch, "ratio": ratio, **res})
+        _say(quiet, out[-1])
         del graphs
     fx.flexiq_check_status()
+    for inst in stacks:
+        for L, *_ in inst:
+            L.close()
+    return out
 
 
 def main():
