@@ -24,12 +24,12 @@
 #include <cuda_fp16.h>
 #include "sm100_ptx.cuh"
 #include "straddle.cuh"
+#include "role_timers.cuh"   // PROF_* expand to nothing in the product build
 
 namespace flexiq {
 
 __device__ unsigned int g_status_word = 0;
 
-#include "role_timers.cuh"   // PROF_* expand to nothing in the product build
 
 constexpr int BM = 128;
 constexpr int kNumWorkWarps = 16;                     // epilogue warps (+ expander warps on the packed path)
@@ -78,6 +78,13 @@ struct GemmParams {
     // weight tile is loaded once per CTA and stays in shared memory in front of the ring, whose stages then hold
     // activation taps only: half as many copies per tile for the producer lane, which bounds these layers.
     int b_res;
+    // Patch mode (KIND 2: 3x3-like convolutions of stride 1 whose channels fit one K block and whose output
+    // channels fit one tile): a tile is TH = 128 / PW whole output rows of one image, its 128 accumulator rows
+    // being the positions y * PW + x of a grid whose pitch PW (a power of two >= W + pad) leaves a few unused
+    // columns.  The input patch of TH + R - 1 rows x PW pixels is loaded ONCE per tile by a tiled 4-D copy
+    // (halo and padding arrive as zeros); filter tap (r, s) is the same patch read from row offset r * PW + s,
+    // so every input pixel crosses from L2 once instead of R * S times.
+    int pw_log2, TH, tiles_per_img, patch_stage;   // patch_stage: bytes of one ring stage (the patch, rounded up to 1 KB)
     // packed low-bit path only: positions the expander warps shift the 4-bit values back to
     const uint8_t *sx;   // [n_g] activation positions, slab order
     const uint8_t *sw;   // [n_g][N] weight positions
@@ -287,6 +294,25 @@ __device__ __forceinline__ void unpack16(uint32_t w0, uint32_t w1, int s, uint32
     }
 }
 
+// The 9 taps of a 3x3 filter on a halo patch, fully unrolled: tap (r, t) reads the patch from row offset
+// r * PW + t (ROW16 sixteen-byte units per pixel row, `down` units per patch row), KS K steps of 32 bytes each.
+template <int CG, int ROW16, int KS>
+__device__ __forceinline__ void patch_taps_3x3(uint32_t d_tmem, uint32_t a_lo, uint32_t down, uint32_t b_lo, uint32_t b_step,
+                                               uint32_t desc_hi, uint32_t idesc)
+{
+#pragma unroll
+    for (int r = 0; r < 3; ++r) {
+#pragma unroll
+        for (int t = 0; t < 3; ++t) {
+#pragma unroll
+            for (int k = 0; k < KS; ++k)
+                ptx::mma_i8_s<CG>(d_tmem, a_lo + (uint32_t)(t * ROW16 + 2 * k), b_lo + (uint32_t)(2 * k), desc_hi, idesc, (r | t | k) ? 1u : 0u);
+            b_lo += b_step;
+        }
+        a_lo += down;
+    }
+}
+
 struct EpilogueCtx {
     uint32_t tmem_base, buf_stride, cta_rank;
     uint64_t *tmem_full, *tmem_empty;
@@ -303,9 +329,10 @@ struct EpilogueCtx {
 // Per pass: fetch the columns' factors, read the whole slice of the accumulator into registers,
 // hand the accumulator back, then scale / round / clip; the results are staged in shared memory (32 rows
 // x 32 bytes: 32 int8, 16 half-precision or 8 four-byte columns) and leave through tiled bulk stores.
-template <int CG, int MODE, bool SPLIT>
+template <int CG, int MODE, bool SPLIT, int KIND>
 __device__ __forceinline__ void epilogue_role(const GemmParams &p, const EpilogueCtx &x, int quad, int part, int lane)
 {
+    constexpr bool kPatch = KIND == 2;
     constexpr bool kScaled = MODE != FLEXIQ_OUT_ACC_I32;
     constexpr bool kHalf = MODE == FLEXIQ_OUT_DEQUANT_F16 || MODE == FLEXIQ_OUT_DEQUANT_BF16;
     constexpr int kElem = (MODE == FLEXIQ_OUT_REQUANT_I8 || MODE == kOutNextSlab) ? 1 : (kHalf ? 2 : 4);  // output bytes per element
@@ -325,9 +352,28 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
     PROF_DECL(prof_math);
     PROF_T0(prof_start);
     const int passes = 4 / x.parts;              // 1 with sixteen epilogue warps, 2 with eight
+    // Patch mode keeps four accumulators, tile ti in accumulator ti mod 4.  With 64-column tiles only column
+    // slots 0 and 1 of a lane quadrant have columns, so slots 2 and 3 take the odd tiles instead of idling.
+    int ti = 0, tile_inc = 1;
+    if (kPatch && BN == 64) { tile_inc = 2; ti = part >> 1; part &= 1; }
     TileWalk tw;
-    for (tw.init(x.first_tile, x.tile_step, x.num_tiles, p.n_tiles); tw.left > 0; tw.next()) {
-        const long long row = ((long long)tw.m_blk * CG + x.cta_rank) * BM + quad * 32 + lane;
+    for (tw.init(x.first_tile + ti * x.tile_step, x.tile_step * tile_inc, x.num_tiles, p.n_tiles); tw.left > 0; tw.next(), ti += tile_inc) {
+        if (kPatch) { buf = ti & 3; buf_phase = (uint32_t)(ti >> 2) & 1u; }
+        long long row = ((long long)tw.m_blk * CG + x.cta_rank) * BM + quad * 32 + lane;
+        // where the warp's 32 accumulator rows go: rows row0.. of Y, or in patch mode a box of bx x by pixels
+        int st_x = 0, st_y = 0, st_n = 0;
+        bool box_live = true;
+        if (kPatch) {
+            const int pw = 1 << p.pw_log2;
+            st_n = tw.m_blk / p.tiles_per_img;
+            const int y0 = (tw.m_blk - st_n * p.tiles_per_img) * p.TH;
+            const int k = quad * 32 + lane;
+            const int yy = y0 + (k >> p.pw_log2), xx = k & (pw - 1);
+            row = (yy < p.P && xx < p.Q) ? ((long long)st_n * p.P + yy) * p.Q + xx : p.M;   // p.M: not an output pixel
+            st_y = y0 + ((quad * 32) >> p.pw_log2);
+            st_x = (quad * 32) & (pw - 1);
+            box_live = st_y < p.P && st_x < p.Q;
+        }
         bool waited = false;
         for (int pass = 0; pass < passes; ++pass) {
             const int col0 = (part * passes + pass) * cols;  // first tile column of this warp in this pass
@@ -395,7 +441,7 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                 // Each warp stages 32 rows x 32 columns (1 KB, 32-byte swizzle: no bank conflicts) and one
                 // lane hands them to a tiled bulk store, which writes whole sectors asynchronously and
                 // drops the rows and columns that lie outside Y.
-                const long long row0 = row - lane;
+                const long long row0 = kPatch ? (box_live ? 0 : p.M) : row - lane;
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     const uint32_t *r = h == 0 ? ra : rb;
@@ -426,14 +472,15 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                         ptx::fence_proxy_async_smem();
                         __syncwarp();
                         if (lane == 0) {
-                            ptx::tma_store_2d(both ? x.map_y : x.map_y16, x.store_stage, n, (int)row0);
+                            if (kPatch) ptx::tma_store_4d(both ? x.map_y : x.map_y16, x.store_stage, n, st_x, st_y, st_n);
+                            else ptx::tma_store_2d(both ? x.map_y : x.map_y16, x.store_stage, n, (int)row0);
                             ptx::bulk_commit_group();
                         }
                     }
                 }
             } else if (kHalf && p.tma_store) {
                 // 16-bit outputs: 32 rows x 16 columns (32 bytes per row: the same 1 KB swizzled box) per store
-                const long long row0 = row - lane;
+                const long long row0 = kPatch ? (box_live ? 0 : p.M) : row - lane;
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     const uint32_t *r = h == 0 ? ra : rb;
@@ -455,7 +502,8 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                             ptx::fence_proxy_async_smem();
                             __syncwarp();
                             if (lane == 0) {
-                                ptx::tma_store_2d(x.map_y, x.store_stage, 2 * n, (int)row0);
+                                if (kPatch) ptx::tma_store_4d(x.map_y, x.store_stage, 2 * n, st_x, st_y, st_n);
+                                else ptx::tma_store_2d(x.map_y, x.store_stage, 2 * n, (int)row0);
                                 ptx::bulk_commit_group();
                             }
                         }
@@ -463,7 +511,7 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                 }
             } else if (kElem == 4 && p.tma_store) {
                 // 4-byte outputs: 32 rows x 8 columns per store (the same 32-byte rows)
-                const long long row0 = row - lane;
+                const long long row0 = kPatch ? (box_live ? 0 : p.M) : row - lane;
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     const uint32_t *r = h == 0 ? ra : rb;
@@ -484,7 +532,8 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
                                 ptx::fence_proxy_async_smem();
                                 __syncwarp();
                                 if (lane == 0) {
-                                    ptx::tma_store_2d(x.map_y, x.store_stage, 4 * (n + 8 * b), (int)row0);
+                                    if (kPatch) ptx::tma_store_4d(x.map_y, x.store_stage, 4 * (n + 8 * b), st_x, st_y, st_n);
+                                    else ptx::tma_store_2d(x.map_y, x.store_stage, 4 * (n + 8 * b), (int)row0);
                                     ptx::bulk_commit_group();
                                 }
                             }
@@ -566,7 +615,7 @@ __device__ __forceinline__ void epilogue_role(const GemmParams &p, const Epilogu
             }
             PROF_ADD(prof_math, te1);
         }
-        if ((buf ^= 1) == 0) buf_phase ^= 1;
+        if (!kPatch && (buf ^= 1) == 0) buf_phase ^= 1;
     }
     if (p.tma_store && lane == 0) ptx::bulk_wait_all();  // the staged stores are performed
     if (quad == 2 && part == 0 && lane == 0) { PROF_STORE(8, prof_wait); PROF_STORE(9, clock64() - prof_start); PROF_STORE(10, prof_ld); PROF_STORE(11, prof_math); }
@@ -604,8 +653,8 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
     uint64_t *full_bar = reinterpret_cast<uint64_t *>(store_stage + kNumWorkWarps * kStoreStagePerWarp);
     uint64_t *empty_bar = full_bar + kMaxStages;
     uint64_t *tmem_full = empty_bar + kMaxStages;
-    uint64_t *tmem_empty = tmem_full + 2;
-    uint64_t *raw_full = tmem_empty + 2;
+    uint64_t *tmem_empty = tmem_full + 4;
+    uint64_t *raw_full = tmem_empty + 4;
     uint64_t *raw_empty = raw_full + kRawStages;
     uint64_t *turn_bar = raw_empty + kRawStages;     // hand-over between the two MMA warps: one phase per tile
     uint32_t *tmem_ptr_s = reinterpret_cast<uint32_t *>(turn_bar + 1);
@@ -618,10 +667,11 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
     const bool k_im2col = KIND != 0 && p.im2col;      // compile-time false for KIND 0: the branches below fold away
     const int k_tps = KIND != 0 ? p.tps : 1;
     const bool k_bres = KIND != 0 && p.b_res;
+    constexpr bool kPatch = KIND == 2;            // halo patch per tile, taps as row offsets (see GemmParams)
     const int b_rows = BN / CG;                       // rows of the B tile this CTA loads
     // one stage = tps sub-tiles of A (BM x BK each) followed by tps sub-tiles of B (b_rows x BK each)
     const int a_sub = BM * p.BK, b_sub = b_rows * p.BK, b_off = k_tps * a_sub;
-    const int stage_bytes = k_bres ? k_tps * a_sub : k_tps * (a_sub + b_sub);
+    const int stage_bytes = kPatch ? p.patch_stage : (k_bres ? k_tps * a_sub : k_tps * (a_sub + b_sub));
     const int ring_off = k_bres ? ((p.T * b_sub + 1023) & ~1023) : 0;   // resident weight tiles lie in front of the ring
     const int num_tiles = p.m_tiles * p.n_tiles;
     const uint32_t cta_rank = CG == 2 ? ptx::cluster_ctarank() : 0u;
@@ -629,16 +679,17 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
     const int first_tile = blockIdx.x / CG, tile_step = gridDim.x / CG;
     // two accumulators (tiles in turn); SPLIT: two per tile, four in all
     const uint32_t buf_stride = BN <= 64 ? 64u : (BN <= 128 ? 128u : 256u);  // column offset from one accumulator to the next
-    const uint32_t tmem_cols = (SPLIT ? 4u : 2u) * buf_stride;
+    const uint32_t tmem_cols = ((SPLIT || kPatch) ? 4u : 2u) * buf_stride;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
             ptx::mbar_init(&full_bar[s], PK ? kExpWarps : 1);  // packed path: every fill counts eight arrivals
             ptx::mbar_init(&empty_bar[s], 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < 4; ++b) {
             ptx::mbar_init(&tmem_full[b], SPLIT ? 2 : 1);   // SPLIT: both MMA warps commit a tile
-            ptx::mbar_init(&tmem_empty[b], CG * kEpiWarps);
+            // patch mode with 64-column tiles: half of the epilogue warps drain a tile (the others take the next one)
+            ptx::mbar_init(&tmem_empty[b], (kPatch && BN == 64) ? kEpiWarps / 2 : CG * kEpiWarps);
         }
         for (int r = 0; r < kRawStages; ++r) {
             ptx::mbar_init(&raw_full[r], 1);
@@ -712,6 +763,23 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                 pix_n = pw.n;
                 pix_h = pw.h * p.stride - p.pad;
                 pix_w = pw.w * p.stride - p.pad;
+            }
+            if (kPatch) {
+                // one copy per tile: TH + R - 1 input rows of PW pixels, starting one padding to the left of and above
+                // the tile's first output pixel; what lies outside the image arrives as zeros
+                PROF_T0(tq0);
+                if (!__all_sync(0xffffffffu, wait_bounded(empty0 + 8 * stage, phase ^ 1, abort_flag, 1))) { ok = false; break; }
+                PROF_ADD(prof_wait, tq0);
+                if (ptx::elect_one()) {
+                    const int img = tw.m_blk / p.tiles_per_img;
+                    const int y0 = (tw.m_blk - img * p.tiles_per_img) * p.TH;
+                    ptx::mbar_expect_tx_s(full0 + 8 * stage, (uint32_t)(((p.TH + p.T / p.S - 1) << p.pw_log2) * p.BK));
+                    ptx::tma_load_4d_s(stage0 + stage * stage_bytes, &mapA_hi, full0 + 8 * stage, 0, -p.pad, y0 - p.pad, img);
+                }
+                __syncwarp();
+                ++issued;
+                if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
+                continue;
             }
             if (k_tps > 1) {
                 // several filter taps per stage: one barrier round trip pays for all of them
@@ -850,7 +918,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             PROF_DECL(prof_wait_acc);
             PROF_DECL(prof_wait_full);
             PROF_T0(prof_start);
-            const int tile_slots = k_tps > 1 ? (p.T + k_tps - 1) / k_tps : p.T * (p.nb_lo + p.nb_hi);  // ring stages per tile
+            const int tile_slots = kPatch ? 1 : (k_tps > 1 ? (p.T + k_tps - 1) / k_tps : p.T * (p.nb_lo + p.nb_hi));  // ring stages per tile
             int ti = 0;                                          // index of the tile in this CTA's sequence
             TileWalk tw;
             for (tw.init(first_tile, tile_step, num_tiles, p.n_tiles); tw.left > 0 && ok; tw.next(), ++ti) {
@@ -861,6 +929,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                     continue;
                 }
                 int slot = 0;                                    // stages of this tile passed so far
+                if (kPatch) { buf = ti & 3; buf_phase = (uint32_t)(ti >> 2) & 1u; }   // four accumulators, tile ti in ti mod 4
                 PROF_T0(t0);
                 if (!__all_sync(0xffffffffu, wait_bounded(&tmem_empty[buf], buf_phase ^ 1, abort_flag, 2))) break;
                 PROF_ADD(prof_wait_acc, t0);
@@ -870,6 +939,55 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                 const uint32_t d_tmem = tmem_base + (uint32_t)(SPLIT ? 2 * buf + my : buf) * buf_stride;
                 const int g0 = ti * tile_slots;                  // SPLIT: number of this tile's first stage in the CTA's sequence
                 uint32_t acc = 0;
+                if (kPatch) {
+                    const int ks = (p.C + 31) >> 5;  // K steps of one tap (C <= BK)
+                    PROF_T0(tq1);
+                    if (!__all_sync(0xffffffffu, wait_bounded(full0 + 8 * stage, phase, abort_flag, 3))) { ok = false; break; }
+                    PROF_ADD(prof_wait_full, tq1);
+                    if (lane == 0) ptx::mbar_arrive(turn_bar);   // the tile's only stage: the other warp may go on
+                    if (!bres_ready) {
+                        if (!__all_sync(0xffffffffu, wait_bounded(&raw_full[0], 0, abort_flag, 6))) { ok = false; break; }
+                        bres_ready = true;
+                    }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t a_lo = a_lo0 + stage * stage_step;
+                    if (ptx::elect_one()) {
+                        const uint32_t b_step = (uint32_t)(b_sub >> 4);
+                        const uint32_t row16 = (uint32_t)(p.BK >> 4);              // one pixel row of the patch, in 16-byte units
+                        uint32_t b_lo = bres_lo, a_row = a_lo;
+                        const int R = p.T / p.S;
+                        if (R == 3 && p.S == 3 && (ks == 2 || ks == 4)) {
+                            // the usual case spelled out: the issuing lane's instruction stream bounds these small MMAs
+                            const uint32_t down = row16 << p.pw_log2;
+                            if (ks == 2) patch_taps_3x3<CG, 4, 2>(d_tmem, a_lo, down, b_lo, b_step, desc_hi, idesc);
+                            else patch_taps_3x3<CG, 8, 4>(d_tmem, a_lo, down, b_lo, b_step, desc_hi, idesc);
+                        } else
+                        for (int r = 0; r < R; ++r) {
+                            uint32_t a_tap = a_row;
+                            for (int t = 0; t < p.S; ++t) {
+                                if (ks == 2) {
+                                    ptx::mma_i8_s<CG>(d_tmem, a_tap, b_lo, desc_hi, idesc, acc);
+                                    ptx::mma_i8_s<CG>(d_tmem, a_tap + 2, b_lo + 2, desc_hi, idesc, 1);
+                                } else if (ks == 4) {
+                                    ptx::mma_i8_s<CG>(d_tmem, a_tap, b_lo, desc_hi, idesc, acc);
+                                    ptx::mma_i8_s<CG>(d_tmem, a_tap + 2, b_lo + 2, desc_hi, idesc, 1);
+                                    ptx::mma_i8_s<CG>(d_tmem, a_tap + 4, b_lo + 4, desc_hi, idesc, 1);
+                                    ptx::mma_i8_s<CG>(d_tmem, a_tap + 6, b_lo + 6, desc_hi, idesc, 1);
+                                } else {
+                                    uint32_t a2 = acc;
+                                    for (int k = 0; k < ks; ++k) { ptx::mma_i8_s<CG>(d_tmem, a_tap + 2 * k, b_lo + 2 * k, desc_hi, idesc, a2); a2 = 1; }
+                                }
+                                acc = 1;
+                                a_tap += row16;                                    // next tap of the filter row: one pixel to the right
+                                b_lo += b_step;
+                            }
+                            a_row += row16 << p.pw_log2;                           // next filter row: one patch row down
+                        }
+                        ptx::mma_commit_s<CG>(empty0 + 8 * stage);
+                    }
+                    __syncwarp();
+                    if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
+                } else
                 if (k_tps > 1) {
                     const int ks = (p.C + 31) >> 5;  // K steps of one tap (C <= BK)
                     for (int tap0 = 0; tap0 < p.T && ok; tap0 += k_tps) {
@@ -910,7 +1028,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                         if (++stage == (uint32_t)p.stages) { stage = 0; phase ^= 1; }
                     }
                 }
-                for (int part = 0; part < 2 && ok && k_tps == 1; ++part) {
+                for (int part = 0; part < 2 && ok && k_tps == 1 && !kPatch; ++part) {
                     const int nb = part ? p.nb_hi : p.nb_lo;
                     if (nb == 0) continue;
                     const int ks_last = part ? p.ks_last_hi : p.ks_last_lo;
@@ -957,7 +1075,8 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                 }
                 if (ok && ptx::elect_one()) ptx::mma_commit_s<CG>(ptx::smem_u32(&tmem_full[buf]));
                 __syncwarp();
-                if (duo && !SPLIT) buf_phase ^= 1;               // this warp's accumulator again at its next tile
+                if (kPatch) {}                                   // set from ti at the top of the loop
+                else if (duo && !SPLIT) buf_phase ^= 1;          // this warp's accumulator again at its next tile
                 else if ((buf ^= 1) == 0) buf_phase ^= 1;        // SPLIT: buf counts the tile's pair of accumulators
             }
             if (my == 0) {
@@ -980,12 +1099,12 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
             x.map_y = &mapY; x.map_y16 = &mapY16;
             x.first_tile = first_tile; x.tile_step = tile_step; x.num_tiles = num_tiles;
             x.parts = kEpiWarps / 4; x.arrivals_on = 1;
-            if (p.out_mode == FLEXIQ_OUT_REQUANT_I8) epilogue_role<CG, FLEXIQ_OUT_REQUANT_I8, SPLIT>(p, x, warp & 3, e >> 2, lane);
-            else if (p.out_mode == FLEXIQ_OUT_DEQUANT_F32) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_F32, SPLIT>(p, x, warp & 3, e >> 2, lane);
-            else if (p.out_mode == kOutNextSlab) epilogue_role<CG, kOutNextSlab, SPLIT>(p, x, warp & 3, e >> 2, lane);
-            else if (p.out_mode == FLEXIQ_OUT_DEQUANT_F16) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_F16, SPLIT>(p, x, warp & 3, e >> 2, lane);
-            else if (p.out_mode == FLEXIQ_OUT_DEQUANT_BF16) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_BF16, SPLIT>(p, x, warp & 3, e >> 2, lane);
-            else epilogue_role<CG, FLEXIQ_OUT_ACC_I32, SPLIT>(p, x, warp & 3, e >> 2, lane);
+            if (p.out_mode == FLEXIQ_OUT_REQUANT_I8) epilogue_role<CG, FLEXIQ_OUT_REQUANT_I8, SPLIT, KIND>(p, x, warp & 3, e >> 2, lane);
+            else if (p.out_mode == FLEXIQ_OUT_DEQUANT_F32) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_F32, SPLIT, KIND>(p, x, warp & 3, e >> 2, lane);
+            else if (p.out_mode == kOutNextSlab) epilogue_role<CG, kOutNextSlab, SPLIT, KIND>(p, x, warp & 3, e >> 2, lane);
+            else if (p.out_mode == FLEXIQ_OUT_DEQUANT_F16) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_F16, SPLIT, KIND>(p, x, warp & 3, e >> 2, lane);
+            else if (p.out_mode == FLEXIQ_OUT_DEQUANT_BF16) epilogue_role<CG, FLEXIQ_OUT_DEQUANT_BF16, SPLIT, KIND>(p, x, warp & 3, e >> 2, lane);
+            else epilogue_role<CG, FLEXIQ_OUT_ACC_I32, SPLIT, KIND>(p, x, warp & 3, e >> 2, lane);
         } else if (PK && warp < 2 + kNumWorkWarps) {
             // --------------------------------------------------------- expanders (packed path)
             // Widen each raw 4-bit tile into the operand ring: 8 packed bytes -> one 16-byte unit
@@ -1206,6 +1325,28 @@ static int make_map_im2col(CUtensorMap *map, const void *base, int Cpart, long l
     return FLEXIQ_OK;
 }
 
+// 4-D byte tensor map over an NHWC tensor: (row_bytes of channels, W, H, Nb), box (box_bytes, bx, by, 1).
+static int make_map_nhwc(CUtensorMap *map, const void *base, uint64_t row_bytes, int W, int H, int Nb, uint32_t box_bytes,
+                         uint32_t bx, uint32_t by, int swizzle_bytes)
+{
+    EncodeTiledFn enc = get_encode_tiled();
+    if (!enc) return set_error(FLEXIQ_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    if ((reinterpret_cast<uintptr_t>(base) & 15) != 0 || (row_bytes & 15) != 0)
+        return set_error(FLEXIQ_ERR_INVALID_ARG, "tensor base %p / pixel pitch %llu not 16-byte aligned", base, (unsigned long long)row_bytes);
+    cuuint64_t dims[4] = {row_bytes, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)Nb};
+    cuuint64_t strides[3] = {row_bytes, row_bytes * W, row_bytes * W * H};
+    cuuint32_t box[4] = {box_bytes, bx, by, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    const CUtensorMapSwizzle swz = swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                 : (swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+                                 : (swizzle_bytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE));
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void *>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+        return set_error(FLEXIQ_ERR_CUDA, "cuTensorMapEncodeTiled (4-D) failed with CUresult %d (box %u x %u x %u)", (int)r, box_bytes, bx, by);
+    return FLEXIQ_OK;
+}
+
 template <int CG, int PK, int KIND, bool SPLIT>
 static int launch_kernel(const CUtensorMap &a_lo, const CUtensorMap &a_hi, const CUtensorMap &b_lo, const CUtensorMap &b_hi,
                          const CUtensorMap &b_st, const CUtensorMap &y_map, const CUtensorMap &y_map16, const GemmParams &p, int sms, cudaStream_t st)
@@ -1389,15 +1530,33 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
             }
         }
     }
+    // Patch mode (see GemmParams): stride-1 filters of more than one tap whose channels fit one K block and whose
+    // output channels fit one tile, the weights of all taps resident in shared memory.
+    bool patch = false;
+    int patch_pw = 8;
+    if (!packed && !g_forced_tile.cg && p.im2col && L->stride == 1 && L->C <= p.BK && L->N <= 128 && W + L->pad <= 128) {
+        while (patch_pw < W + L->pad) patch_pw *= 2;
+        const int th = BM / patch_pw, bn_p = L->N <= 64 ? 64 : 128;
+        const int stage = (((th + L->R - 1) * patch_pw * p.BK) + 1023) & ~1023;
+        const int b_all = ((p.T * bn_p * p.BK) + 1023) & ~1023;
+        if (b_all + 2 * stage <= kStageRegion && th + L->R - 1 <= 256) {
+            patch = true;
+            tc.cg = 1; tc.bn = bn_p;
+            p.TH = th; p.patch_stage = stage;
+            p.pw_log2 = 0;
+            while ((1 << p.pw_log2) < patch_pw) ++p.pw_log2;
+            p.tiles_per_img = (p.P + th - 1) / th;
+        }
+    }
     const int bn = tc.bn, cg = tc.cg;
     p.sx = x_shift ? x_shift : L->sx;
     p.sw = L->sw;
     p.G = L->G;
-    p.m_tiles = (int)((M + (long long)BM * cg - 1) / ((long long)BM * cg));
+    p.m_tiles = patch ? Nb * p.tiles_per_img : (int)((M + (long long)BM * cg - 1) / ((long long)BM * cg));
     p.BN = bn;
     p.n_tiles = (L->N + bn - 1) / bn;
     p.tps = 1;
-    if (!packed && p.im2col && L->C <= p.BK && L->S > 1) {
+    if (!packed && !patch && p.im2col && L->C <= p.BK && L->S > 1) {
         // convolution whose channels fit one K block: a stage holds up to a filter row of taps
         const int per_tap = (BM + bn / cg) * p.BK;
         const int limit = 49152 / per_tap;
@@ -1409,6 +1568,10 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
         const int b_all = ((p.T * (bn / cg) * p.BK + 1023) / 1024) * 1024;
         const int st = (kStageRegion - b_all) / (p.tps * BM * p.BK);
         if (b_all <= 65536 && st >= 4) { p.b_res = 1; p.stages = st; }
+    }
+    if (patch) {
+        p.b_res = 1;
+        p.stages = (kStageRegion - (((p.T * bn * p.BK) + 1023) & ~1023)) / p.patch_stage;
     }
     if (p.stages > kMaxStages) p.stages = kMaxStages;
     if (packed) {  // room for the ring of raw 4-bit tiles behind the operand ring
@@ -1426,12 +1589,14 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     const void *slab = packed_path ? static_cast<const void *>(X8) : static_cast<const void *>(X4);
     Layer::CallMaps &cm = L->call_maps;
     const bool cached = !packed && cm.slab == slab && cm.M == M && cm.Nb == Nb && cm.H == H && cm.W == W && cm.bk == p.BK &&
-                        cm.im2col == (int)p.im2col && (!staged || (cm.staged && cm.Y == Y && cm.y_elem == y_elem));
+                        cm.im2col == (int)p.im2col + 2 * (int)patch && (!staged || (cm.staged && cm.Y == Y && cm.y_elem == y_elem));
     if (cached) {
         a_lo = a_hi = cm.a;
     } else if (!packed) {
         // one int8 slab [rows][C] (a packed-path layer at ratio 0 has it in X8_dev)
-        if (p.im2col) {
+        if (patch) {
+            if ((rc = make_map_nhwc(&a_hi, slab, (uint64_t)L->C, W, H, Nb, p.BK, 1u << p.pw_log2, p.TH + L->R - 1, p.BK))) return rc;
+        } else if (p.im2col) {
             if ((rc = make_map_im2col(&a_hi, slab, L->C, L->C, Nb, H, W, L->R, L->S, L->stride, L->pad, p.BK, p.BK))) return rc;
         } else {
             const long long rows = L->is_conv ? (long long)Nb * H * W : M;
@@ -1459,6 +1624,13 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     if (staged && cached) {
         y_map = cm.y;
         y_map16 = cm.y16;
+    } else if (staged && patch) {
+        // a warp's 32 accumulator rows are bx consecutive pixels of by consecutive output rows
+        const uint32_t bx = (1u << p.pw_log2) < 32u ? (1u << p.pw_log2) : 32u, by = 32u / bx;
+        const uint64_t rb = (uint64_t)L->N * y_elem;
+        if ((y_elem > 1 || L->N >= 32) && (rc = make_map_nhwc(&y_map, Y, rb, p.Q, p.P, Nb, 32, bx, by, 32))) return rc;
+        if (y_elem > 1) y_map16 = y_map;
+        else if ((rc = make_map_nhwc(&y_map16, Y, rb, p.Q, p.P, Nb, 16, bx, by, 0))) return rc;
     } else if (staged && y_elem > 1) {
         // rows of N 2- or 4-byte values addressed in bytes: a box is 32 bytes (16 or 8 columns) x 32 rows
         if ((rc = make_map_2d(&y_map, Y, (uint64_t)L->N * y_elem, (uint64_t)M, (uint64_t)L->N * y_elem, 32, 32, 32))) return rc;
@@ -1468,7 +1640,7 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
         if ((rc = make_map_2d(&y_map16, Y, (uint64_t)L->N, (uint64_t)M, (uint64_t)L->N, 16, 32, 0))) return rc;
     }
     if (!packed && !cached) {
-        cm.slab = slab; cm.Y = staged ? Y : nullptr; cm.M = M; cm.Nb = Nb; cm.H = H; cm.W = W; cm.bk = p.BK; cm.im2col = p.im2col;
+        cm.slab = slab; cm.Y = staged ? Y : nullptr; cm.M = M; cm.Nb = Nb; cm.H = H; cm.W = W; cm.bk = p.BK; cm.im2col = (int)p.im2col + 2 * (int)patch;
         cm.staged = staged; cm.y_elem = y_elem; cm.a = a_hi; cm.y = y_map; cm.y16 = y_map16;
     }
     const int bi = weight_map_index(bn / cg);  // box rows = the B rows one CTA loads
@@ -1476,13 +1648,15 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     // One narrow tile per CTA and a long K: nothing overlaps across tiles, so the MMA warps share the tile
     // (SPLIT).  With several tiles per CTA the warps already work side by side on tiles of their own, and the
     // second accumulator's extra read in the epilogue would only cost (measured: +4 to +6 % on short-K shapes).
-    const bool split = !packed && bn <= 128 && p.tps == 1 && p.T * (p.nb_lo + p.nb_hi) >= 8 &&
+    const bool split = !packed && !patch && bn <= 128 && p.tps == 1 && p.T * (p.nb_lo + p.nb_hi) >= 8 &&
                        (long long)p.m_tiles * p.n_tiles <= sms / cg;
     if (next) record_slab(const_cast<Layer *>(next), Y, next->K_lo);   // the fused boundary writes the next layer's slab at its current ratio
     if (packed) return launch_kernel<1, 1, 1, false>(a_lo, a_hi, L->map_w4[bi], L->map_w8[bi], L->map_w8[bi], y_map, y_map16, p, sms, st);
     // multi-tap stages hold every channel in one K block: the whole weight operand is one of the three forms
-    const CUtensorMap &b_hi_map = p.tps > 1 ? (b_whole == 0 ? L->map_w8[bi] : (b_whole == 1 ? L->map_w8m[bi] : L->map_wst[bi])) : L->map_w8[bi];
-    if (p.tps > 1 && b_whole == 2) p.b_tap_step = p.BK;
+    const bool one_block = p.tps > 1 || patch;   // every channel in one K block: the weight operand is one of the three forms as a whole
+    const CUtensorMap &b_hi_map = one_block ? (b_whole == 0 ? L->map_w8[bi] : (b_whole == 1 ? L->map_w8m[bi] : L->map_wst[bi])) : L->map_w8[bi];
+    if (one_block && b_whole == 2) p.b_tap_step = p.BK;
+    if (patch) return launch_kernel<1, 0, 2, false>(a_lo, a_hi, L->map_w8m[bi], b_hi_map, L->map_wst[bi], y_map, y_map16, p, sms, st);
 #define FLEXIQ_LAUNCH(CG_, KIND_, SPLIT_) launch_kernel<CG_, 0, KIND_, SPLIT_>(a_lo, a_hi, L->map_w8m[bi], b_hi_map, L->map_wst[bi], y_map, y_map16, p, sms, st)
     if (cg == 2) {
         if (conv_kind) return split ? FLEXIQ_LAUNCH(2, 1, true) : FLEXIQ_LAUNCH(2, 1, false);

@@ -108,6 +108,21 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap *m, uint32_t src,
                  ::"l"(reinterpret_cast<uint64_t>(m)), "r"(src), "r"(x), "r"(y)
                  : "memory");
 }
+// The same for a 4-D tensor (channel bytes, x, y, image); no coordinate may be negative.
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap *m, uint32_t src, int c, int x, int y, int n)
+{
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(src), "r"(c), "r"(x), "r"(y), "r"(n)
+                 : "memory");
+}
+// Tiled load of a 4-D box (channel bytes, x, y, image).  x, y and n may start outside the tensor
+// (negative or beyond the end): those elements arrive as zeros; c must keep the 16-byte rule.
+__device__ __forceinline__ void tma_load_4d_s(uint32_t dst, const CUtensorMap *m, uint32_t bar, int c, int x, int y, int n)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(c), "r"(x), "r"(y), "r"(n) : "memory");
+}
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // all of this thread's bulk groups have finished reading their shared-memory source
 __device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }

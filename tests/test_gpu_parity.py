@@ -249,6 +249,21 @@ def test_conv_shapes(dev, Nb, H, C, Cout, R, stride):
     _run_conv(case, dev, [0.0, 0.25, 0.5, 1.0], shifts=shifts)
 
 
+@pytest.mark.parametrize("Nb,H,C,Cout,R", [(3, 14, 128, 80, 3),    # 8 output rows per tile, 14 rows: a ragged second tile; 80 channels in a 128-column tile
+                                          (5, 7, 64, 64, 3),      # pitch 8: one tile holds a whole image and more
+                                          (2, 20, 48, 32, 3),     # fewer channels than the K block
+                                          (2, 33, 64, 48, 5),     # 5 x 5 taps (the generic tap loop), pitch 64, odd height
+                                          (1, 60, 32, 16, 3),     # widest image the 64-pixel pitch holds with its padding... and one K step
+                                          (2, 100, 64, 64, 3)])   # pitch 128: one output row per tile
+def test_conv_patch_mode_edges(dev, Nb, H, C, Cout, R):
+    """Stride-1 convolutions whose channels fit one K block take the patch path (one halo patch per tile, taps as row
+    offsets into it): image sizes that leave unused grid columns and ragged last tiles, narrow channel counts."""
+    case = inputs.resnet_conv("pm", Nb, H, C, Cout, R, seed=H + C + R)
+    rng = np.random.default_rng(H * C + R)
+    shifts = rng.integers(0, 5, C // case.G).astype(np.uint8)
+    _run_conv(case, dev, [0.0, 0.5, 1.0], shifts=shifts)
+
+
 def test_resnet50_conv_full_size_56(dev):
     # full-size 3x3 C=64 @56x56 at batch 4 (the bench runs batch 32; rows are independent)
     case = inputs.resnet_conv("c56", 4, 56, 64, 64, 3, seed=3000)
