@@ -264,6 +264,23 @@ def test_conv_patch_mode_edges(dev, Nb, H, C, Cout, R):
     _run_conv(case, dev, [0.0, 0.5, 1.0], shifts=shifts)
 
 
+@pytest.mark.parametrize("kind,shape", [("conv", (4, 7, 512, 256, 3)), ("conv", (2, 7, 256, 80, 3)), ("linear", (200, 2048, 256, 16)),
+                                        ("linear", (130, 1536, 384, 32)), ("linear", (64, 3072, 272, 16))])
+def test_small_m_long_k_shapes(dev, kind, shape):
+    """Small-M, long-K layers (one narrow tile per CTA: the two MMA warps share the tile's K blocks, an accumulator
+    each).  Odd numbers of K blocks, ragged M and N, every output type and several ratios (the boundary block included)."""
+    if kind == "conv":
+        Nb, H, C, Cout, R = shape
+        case = inputs.resnet_conv("ks", Nb, H, C, Cout, R, seed=H + C + Cout)
+        rng = np.random.default_rng(C + Cout)
+        _run_conv(case, dev, [0.0, 0.3, 1.0], shifts=rng.integers(0, 5, C // case.G).astype(np.uint8))
+    else:
+        M, K, N, G = shape
+        case = inputs.ranged_linear("ks", M, K, N, G, seed=M + K, group_structured=True)
+        rng = np.random.default_rng(K + N)
+        _run_linear(case, dev, [0.0, 0.3, 1.0], shifts=rng.integers(0, 5, K // G).astype(np.uint8))
+
+
 def test_resnet50_conv_full_size_56(dev):
     # full-size 3x3 C=64 @56x56 at batch 4 (the bench runs batch 32; rows are independent)
     case = inputs.resnet_conv("c56", 4, 56, 64, 64, 3, seed=3000)
