@@ -428,6 +428,13 @@ int flexiq_force_tile(int cta_group, int tile_n);
  * SMs.  Writes the CTAs per tile (1 or 2) and the tile width.  The paper has no counterpart. */
 int flexiq_choose_tile(int64_t M, int N, int k_blocks, int block_k, int sm_count, int *cta_group_out, int *tile_n_out);
 
+/* Test hook: runs the mainloop's bounded wait, with a limit of about a millisecond instead of two seconds, once on
+ * a barrier that completes and once on a barrier that nothing ever arrives on.  result_dev [3] int32 receives
+ * {1, 0, 1}: the first wait was served, the second gave up, and the CTA's give-up flag is set; the status word is
+ * raised as after any expired wait (flexiq_check_status then returns FLEXIQ_ERR_TIMEOUT once, and the context
+ * stays usable).  Nothing traps and nothing spins without bound.  The paper has no counterpart. */
+int flexiq_selftest_wait_expiry(int *result_dev, void *stream);
+
 /* Reads and clears the device status word raised by a bounded wait that expired.
  * Synchronises `stream`. */
 int flexiq_check_status(void *stream);

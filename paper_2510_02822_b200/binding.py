@@ -30,7 +30,7 @@ EXPORTS = [
     "flexiq_calib_weight_absmax", "flexiq_calib_prepare", "flexiq_calib_absmax_ema",
     "flexiq_controller_create", "flexiq_controller_destroy", "flexiq_controller_level", "flexiq_controller_update",
     "flexiq_serving_simulate", "flexiq_evo_init", "flexiq_evo_next_generation", "flexiq_sq_distance_i8",
-    "flexiq_layer_export", "flexiq_force_tile", "flexiq_choose_tile", "flexiq_check_status", "flexiq_last_error",
+    "flexiq_layer_export", "flexiq_selftest_wait_expiry", "flexiq_force_tile", "flexiq_choose_tile", "flexiq_check_status", "flexiq_last_error",
 ]
 
 _lib = None
@@ -78,6 +78,7 @@ def lib():
         L.flexiq_calib_absmax_ema.argtypes = [vp, i32, i64, f32, vp, vp]
         L.flexiq_layer_export.argtypes = [vp, vp, vp, vp]
         L.flexiq_check_status.argtypes = [vp]
+        L.flexiq_selftest_wait_expiry.argtypes = [vp, vp]
         f64 = C.c_double
         L.flexiq_controller_create.argtypes = [C.POINTER(vp), i32, i32, vp, vp, f64, f64, i32]
         L.flexiq_controller_destroy.argtypes = [vp]
@@ -244,6 +245,10 @@ def flexiq_choose_tile(M, N, k_blocks, block_k=128, sm_count=148):
     cg, bn = C.c_int(0), C.c_int(0)
     _check(lib().flexiq_choose_tile(C.c_int64(M), N, k_blocks, block_k, sm_count, C.byref(cg), C.byref(bn)))
     return cg.value, bn.value
+
+
+def flexiq_selftest_wait_expiry(result_dev):
+    _check(lib().flexiq_selftest_wait_expiry(_ptr(result_dev), _stream()))
 
 
 def flexiq_check_status():

@@ -94,13 +94,13 @@ struct GemmParams {
 // Bounded wait.  Returns false after the limit or when another role already gave up;
 // the caller then leaves its loops and the CTA drains.  The slow path stays out of line
 // so that the hot loops remain small.
-__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int where)
+__device__ __noinline__ bool wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int where, uint32_t limit = kSpinLimit)
 {
     // a few quick polls for the common short wait, then hardware-parked waits of up to a
     // microsecond each: they wake at once when the phase completes and issue nothing meanwhile
     for (uint32_t it = 0; it < 8; ++it)
         if (ptx::mbar_try_wait_s(bar, parity)) return true;
-    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+    for (uint32_t it = 0; it < limit; ++it) {
         if (ptx::mbar_try_wait_hint_s(bar, parity, 1000u)) return true;
         if (*abort_flag) return false;
     }
@@ -1253,6 +1253,30 @@ __global__ void scale_vectors_kernel(int N, float x_scale, float y_scale, int re
     beta[n] = requant ? __fdiv_rn(bv, y_scale) : bv;
 }
 
+// Test hook: one warp waits, with the mainloop's own bounded wait but a limit of about a millisecond, on a barrier
+// that nothing ever arrives on; a second barrier that IS arrived on shows the same routine returning at once.
+__global__ void wait_expiry_kernel(int *result)
+{
+    __shared__ uint64_t bars[2];
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&bars[0], 1);
+        ptx::mbar_init(&bars[1], 1);
+        abort_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) ptx::mbar_arrive(&bars[1]);
+    __syncwarp();
+    const bool served = wait_slow(ptx::smem_u32(&bars[1]), 0, &abort_flag, 15, 1024u);    // completes: returns true
+    const bool starved = wait_slow(ptx::smem_u32(&bars[0]), 0, &abort_flag, 15, 1024u);   // never completes: gives up
+    if (threadIdx.x == 0) {
+        result[0] = served ? 1 : 0;
+        result[1] = starved ? 1 : 0;
+        result[2] = abort_flag;
+    }
+}
+
 // The straddle block of the masked path (straddle.cuh) for a GEMM that no prologue launch precedes.
 __global__ void straddle_kernel(const StraddleJob job)
 {
@@ -1743,6 +1767,16 @@ extern "C" int flexiq_force_tile(int cta_group, int tile_n)
         (cta_group == 2 && tile_n < 128))
         return set_error(FLEXIQ_ERR_INVALID_ARG, "unsupported tile: cta_group %d, tile_n %d", cta_group, tile_n);
     g_forced_tile = TileChoice{cta_group, tile_n};
+    return FLEXIQ_OK;
+}
+
+extern "C" int flexiq_selftest_wait_expiry(int *result_dev, void *stream)
+{
+    if (!result_dev) return set_error(FLEXIQ_ERR_INVALID_ARG, "result_dev is NULL");
+    int rc = check_device_sm100();
+    if (rc) return rc;
+    wait_expiry_kernel<<<1, 32, 0, reinterpret_cast<cudaStream_t>(stream)>>>(result_dev);
+    FLEXIQ_CUDA_TRY(cudaGetLastError());
     return FLEXIQ_OK;
 }
 

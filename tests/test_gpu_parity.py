@@ -584,6 +584,19 @@ def test_slab_written_at_another_ratio_is_refused(dev):
         L.close()
 
 
+def test_bounded_wait_expires_and_the_context_stays_usable(dev):
+    """A device-side wait that nothing satisfies gives up after its limit (here a millisecond), raises the status word
+    that flexiq_check_status reports as a timeout -- once -- and leaves the context usable for the next launches."""
+    res = torch.zeros(3, dtype=torch.int32, device=dev)
+    fx.flexiq_selftest_wait_expiry(res)
+    with pytest.raises(fx.FlexiqError) as e:
+        fx.flexiq_check_status()
+    assert e.value.code == fx.ERR_TIMEOUT
+    assert res.cpu().tolist() == [1, 0, 1]
+    fx.flexiq_check_status()                       # cleared
+    _run_linear(inputs.ranged_linear("after", 130, 128, 48, 16, seed=77), dev, [0.5])   # the device still computes
+
+
 def test_two_layers_on_two_streams(dev):
     """Independent layer handles may run on different streams at the same time."""
     cases = [inputs.ranged_linear("a", 700, 256, 320, 16, seed=31), inputs.ranged_linear("b", 500, 512, 144, 32, seed=32)]
