@@ -16,8 +16,9 @@
  *     FLEXIQ_ERR_UNSUPPORTED.
  *   - A layer handle belongs to the device that was current when it was created.  Every call
  *     that enqueues work for a handle returns FLEXIQ_ERR_INVALID_ARG when another device is
- *     current (its pointers would not be valid there).  One handle is used from one stream at a
- *     time; different handles may run on different streams concurrently.
+ *     current (its pointers would not be valid there).  One handle is used from one stream and
+ *     one host thread at a time (it keeps host-side records of the calls it has enqueued);
+ *     different handles may run on different streams and threads concurrently.
  *   - Every device-side wait is bounded.  If one expires the kernel raises a status
  *     word that flexiq_check_status() reports as FLEXIQ_ERR_TIMEOUT; the context
  *     stays usable.
