@@ -64,12 +64,57 @@ __global__ void group_or_kernel(const void *__restrict__ X, long long M, int K, 
         if (or_s[i]) atomicOr(&or_words[i], or_s[i]);
 }
 
+// Phase 2 of the dynamic mode on the masked path: the low groups of the slab that phase 1 wrote are lowered in
+// place with the positions the OR words give -- clip to what four bits hold at the position, clear the bits below
+// it -- 16 bytes per thread; a group whose position is 0 is already what it should be and is not touched.  The
+// positions go to sx_out (slab order).  Blocks in front: the straddle block of the weights, as in the static kernel.
+__global__ void lower_inplace_kernel(int8_t *__restrict__ slab, long long M, int K, int G, int K_lo,
+                                     const unsigned *__restrict__ or_words, uint8_t *__restrict__ sx_out, StraddleJob wp)
+{
+    ptx::pdl_launch_dependents();
+    ptx::pdl_wait();  // phase 1 has written the slab and the OR words
+    if (blockIdx.x < wp.first_block) {
+        const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+        if (idx < (long long)wp.rows * (wp.BK >> 4)) straddle_write_unit(wp, idx);
+        return;
+    }
+    const unsigned qblock = blockIdx.x - wp.first_block, qblocks = gridDim.x - wp.first_block;
+    if (qblock == 0)
+        for (int j = threadIdx.x; j < K / G; j += blockDim.x) sx_out[j] = (uint8_t)position_from_or(or_words[j]);
+    const int lo_c16 = K_lo / 16, c_per_g = G / 16;
+    const long long total = M * lo_c16;
+    for (long long idx = (long long)qblock * blockDim.x + threadIdx.x; idx < total; idx += (long long)qblocks * blockDim.x) {
+        const long long m = idx / lo_c16;
+        const int c16 = (int)(idx - m * lo_c16);
+        const int s = position_from_or(or_words[c16 / c_per_g]);
+        if (s == 0) continue;
+        uint4 *ptr = reinterpret_cast<uint4 *>(slab + (size_t)m * K + (size_t)c16 * 16);
+        const uint4 u = *ptr;
+        const unsigned in[4] = {u.x, u.y, u.z, u.w};
+        unsigned w[4];
+        const int hi = (8 << s) - 1, lo = -(8 << s);
+        const unsigned mask = ((0xffu << s) & 0xffu) * 0x01010101u;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            int b[4];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) b[t] = max(lo, min(hi, (int)(signed char)((in[k] >> (8 * t)) & 0xff)));
+            w[k] = pack2_sat_s8(b[1], b[0], pack2_sat_s8(b[3], b[2], 0u)) & mask;
+        }
+        *ptr = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
 // Quantize + lower + gather.  Thread <-> (row m, 16-channel slab chunk c16).
 //   sx != nullptr : static positions (slab order);  else positions from or_words.
 // Lowering works on the packed int8 words: q is first clipped to the range the 4-bit value
 // at position s can hold, [-2^(s+3), 2^(s+3) - 1] (identical to clamping q >> s to [-8, 7],
 // the shift being monotone); then bits s..s+3 of every byte are the two's-complement nibble
 // (packed path), and clearing the s low bits of every byte is (q >> s) << s (masked path).
+// PACKED == 2 is phase 1 of the dynamic mode on the masked path: nothing is lowered yet (every group is written
+// at 8 bits, gathered into slab order) and the OR of the sign-folded values of every group is collected on the way
+// (or_acc; a thread keeps its chunk column from one grid stride to the next when the stride is a multiple of the
+// row's chunks, which the launch arranges, so it flushes its OR once), so that the input is read once.
 template <int DTYPE, int PACKED>
 __global__ void quantize_lower_kernel(const void *__restrict__ X, long long M, int K, int G, int K_lo, float S,
                                       const int32_t *__restrict__ perm, const uint8_t *__restrict__ sx,
@@ -91,6 +136,39 @@ __global__ void quantize_lower_kernel(const void *__restrict__ X, long long M, i
         return;
     }
     const unsigned qblock = blockIdx.x - wp.first_block, qblocks = gridDim.x - wp.first_block;
+    if (PACKED == 2) {
+        extern __shared__ unsigned or_s[];
+        unsigned *or_acc = const_cast<unsigned *>(or_words);
+        const int n_g = K / G;
+        for (int i = threadIdx.x; i < n_g; i += blockDim.x) or_s[i] = 0;
+        __syncthreads();
+        unsigned o = 0;
+        int oj = -1;
+        for (long long idx = (long long)qblock * blockDim.x + threadIdx.x; idx < total; idx += (long long)qblocks * blockDim.x) {
+            const long long m = idx / n_c16;
+            const int c16 = (int)(idx - m * n_c16);
+            const int j = c16 / c_per_g;
+            if (j != oj) {   // another group (only when the stride is not a multiple of a row's chunks)
+                if (o) atomicOr(&or_s[oj], (o | (o >> 8) | (o >> 16) | (o >> 24)) & 0xffu);
+                o = 0;
+                oj = j;
+            }
+            const int src_c = perm[j] * G + (c16 % c_per_g) * 16;
+            unsigned w[4];
+            quantize16<DTYPE>(reinterpret_cast<const char *>(X) + ((size_t)m * K + src_c) * elem_bytes<DTYPE>(), div, -128.f, 127.f, w);
+            *reinterpret_cast<uint4 *>(X4 + m * x4_pitch + (size_t)c16 * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {   // fold negatives per byte (q >= 0 ? q : ~q): xor with the byte's sign replicated
+                const unsigned sign = (w[k] >> 7) & 0x01010101u;
+                o |= w[k] ^ (sign * 0xffu);
+            }
+        }
+        if (o) atomicOr(&or_s[oj], (o | (o >> 8) | (o >> 16) | (o >> 24)) & 0xffu);
+        __syncthreads();
+        for (int i = threadIdx.x; i < n_g; i += blockDim.x)
+            if (or_s[i]) atomicOr(&or_acc[i], or_s[i]);
+        return;
+    }
     if (sx_out != nullptr && qblock == 0)
         for (int j = threadIdx.x; j < K / G; j += blockDim.x) sx_out[j] = (uint8_t)position_from_or(or_words[j]);
     for (long long idx = (long long)qblock * blockDim.x + threadIdx.x; idx < total;
@@ -188,6 +266,23 @@ static int launch_prologue(Layer *L, const void *X, long long M, float S, int dy
     const int n_c16 = K / 16;
     const int sms = device_sm_count(L->device);
     const int threads = 256;
+    const bool masked = L->lowbit_path == FLEXIQ_LOWBIT_MASKED_I8;
+    if (dynamic && masked) {
+        // the input is read once: phase 1 quantizes, gathers and collects the OR words, phase 2 lowers the low groups of
+        // the slab in place (from L2) with the positions those words give
+        FLEXIQ_CUDA_TRY(cudaMemsetAsync(scratch, 0, sizeof(unsigned) * L->n_g, st));
+        long long want1 = (M * n_c16 + threads - 1) / threads;
+        long long blocks1 = want1 < (long long)sms * 16 ? want1 : (long long)sms * 16;
+        // a grid stride that is a multiple of a row's chunks keeps every thread on its chunk column
+        int a = n_c16, b = threads;
+        while (b) { const int t = a % b; a = b; b = t; }
+        const long long unit = n_c16 / a;
+        if (blocks1 >= unit) blocks1 -= blocks1 % unit;
+        StraddleJob none{};
+        FLEXIQ_CUDA_TRY(launch_pdl(quantize_lower_kernel<DTYPE, 2>, (unsigned)blocks1, threads, sizeof(unsigned) * L->n_g, st, X, M, K, G, 0, S, L->perm,
+                                   static_cast<const uint8_t *>(nullptr), static_cast<const unsigned *>(scratch), X4, pitch, X8, pitch8,
+                                   static_cast<uint8_t *>(nullptr), none));
+    } else
     if (dynamic) {
         FLEXIQ_CUDA_TRY(cudaMemsetAsync(scratch, 0, sizeof(unsigned) * L->n_g, st));
         long long want = (M * n_c16 + threads - 1) / threads;
@@ -201,7 +296,6 @@ static int launch_prologue(Layer *L, const void *X, long long M, float S, int dy
     const uint8_t *sx = dynamic ? nullptr : L->sx;
     StraddleJob wp{};
     long long extra = 0;
-    const bool masked = L->lowbit_path == FLEXIQ_LOWBIT_MASKED_I8;
     if (straddle_in_use(L) && straddle_stale(L, st)) {
         // the GEMM that consumes these slabs reads the straddle block of the same max_4bit_ch
         wp.wst = L->wst; wp.w8m = L->w8m; wp.w8 = L->w8;
@@ -213,6 +307,16 @@ static int launch_prologue(Layer *L, const void *X, long long M, float S, int dy
         extra = ((long long)wp.rows * (wp.BK >> 4) + threads - 1) / threads;
     }
     wp.first_block = (unsigned)extra;   // the straddle blocks come first
+    if (dynamic && masked) {
+        long long want2 = (M * (L->K_lo / 16) + threads - 1) / threads;
+        long long blocks2 = want2 < (long long)sms * 16 ? want2 : (long long)sms * 16;
+        if (blocks2 < 1) blocks2 = 1;   // the positions are written even when no group is low
+        FLEXIQ_CUDA_TRY(launch_pdl(lower_inplace_kernel, (unsigned)(blocks2 + extra), threads, 0, st, reinterpret_cast<int8_t *>(X4), M, K, G, L->K_lo,
+                                   static_cast<const unsigned *>(scratch), sx_out, wp));
+        if (wp.wst) straddle_written(L, st);
+        record_slab(L, X4, L->K_lo);
+        return FLEXIQ_OK;
+    }
     const unsigned grid = (unsigned)(blocks + extra);
     if (!masked)
         FLEXIQ_CUDA_TRY(launch_pdl(quantize_lower_kernel<DTYPE, 1>, grid, threads, 0, st, X, M, K, G, L->K_lo, S, L->perm, sx, scratch, X4, pitch, X8, pitch8, dynamic ? sx_out : nullptr, wp));
