@@ -223,8 +223,8 @@ int flexiq_mixed_gemm(flexiq_layer_t layer, const uint8_t *X4_dev, const int8_t 
  * k = (r, s, c), x[image][p*stride + r - pad][q*stride + s - pad][c], zero outside; the
  * slabs are NHWC with the channel dimension laid out as in flexiq_quantize_lower
  * (X4_dev [Nb][H][W][pitch], and on the packed path X8_dev [Nb][H][W][C_hi]); Y_dev [Nb][P][Q][Cout].
- * Calls on one layer handle must be ordered on one stream (the handle's weight operand and
- * epilogue factors follow the ratio and the scales of the latest call). */
+ * Calls on one layer handle must be ordered on one stream (the handle's ratio-dependent weight
+ * block and its epilogue factor tables follow the ratio and the scales of the calls it has seen). */
 int flexiq_mixed_conv(flexiq_layer_t layer, const uint8_t *X4_dev, const int8_t *X8_dev,
                       const uint8_t *x_shift_dev, int Nb, int H, int W, float x_scale,
                       float y_scale, int out_mode, void *Y_dev, void *stream);

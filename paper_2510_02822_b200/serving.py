@@ -6,8 +6,8 @@ stack of quantized linears of a transformer.
 
 1. profile: the time of one pass over the model's 48 quantized linear layers (prologue + mixed GEMM
    per layer, through the library, ratio set by flexiq_set_lowbit_ratio) per level (0/25/50/75/100 %)
-   and batch size 1 .. max_batch; each (level, batch) pass is one CUDA graph, and a switch of the level
-   brings the weight operands along with flexiq_layer_sync_ratio before the replay.  `--service paper-shaped` replaces the measured table by one that
+   and batch size 1 .. max_batch; each (level, batch) pass is one CUDA graph that is complete in itself
+   (it holds the write of the ratio-dependent weight block where its ratio needs one), so the graphs replay in any order.  `--service paper-shaped` replaces the measured table by one that
    falls with the ratio as the paper's GPU does (1.43x faster at 100 % than at 0 %), to exercise the
    controller where the hardware gives it something to trade; it is labelled as such in the output.
 2. latency against request rate: Poisson arrivals at 100 .. 3000 requests/s through
@@ -58,8 +58,8 @@ class Stack:
         self.use_graphs = use_graphs
 
     def set_level(self, level: int):
-        """Run-time ratio switch: one host integer per layer; with graphs also the weight operands,
-        which a replayed graph does not bring up to date itself."""
+        """Run-time ratio switch: one host integer per layer (flexiq_layer_sync_ratio below is kept as a no-cost
+        precaution: a captured graph writes the ratio-dependent weight block itself)."""
         if level != self.level:
             for L, *_ in self.inst:
                 L.set_lowbit_ratio(level / (LEVELS - 1))
@@ -108,7 +108,7 @@ def profile_service(stack: Stack, max_batch: int, reps: int) -> np.ndarray:
         stack.timed(0, 1)
     for level in range(LEVELS):
         for b in range(1, max_batch + 1):
-            for _ in range(3):  # the weight operand follows the ratio (and the graph is captured) on the first pass
+            for _ in range(3):  # the graph is captured on the first pass
                 stack.timed(level, b)
             table[level, b - 1] = float(np.median([stack.timed(level, b) for _ in range(reps)]))
     return table

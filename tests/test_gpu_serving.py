@@ -18,8 +18,9 @@ def dev():
 
 
 def test_graphs_of_several_ratios_replay_in_any_order(dev):
-    """A graph captured at ratio r stays valid after other ratios ran, provided the weight operand
-    is brought back with flexiq_layer_sync_ratio before the replay (the run-time ratio switch)."""
+    """A graph captured at ratio r stays valid after other ratios ran (the run-time ratio switch): with the ratio set
+    again and flexiq_layer_sync_ratio called before the replay, as a deployment may do, and -- second loop -- with
+    nothing at all between the replays."""
     case = inputs.ranged_linear("srv", 333, 512, 304, 16, seed=77, group_structured=True)
     perm, sxg, sxs, sw = helpers.prepare_linear(case)
     L = fx.Layer(torch.from_numpy(case.Wq).to(dev), torch.from_numpy(case.w_scale).to(dev), torch.from_numpy(case.bias).to(dev), perm, sxg, case.G)
@@ -57,7 +58,12 @@ def test_graphs_of_several_ratios_replay_in_any_order(dev):
         graphs[r].replay()
         torch.cuda.synchronize()
         assert np.array_equal(Y.cpu().numpy(), want[r]), r
-    L.sync_ratio()  # nothing changed sides: a no-op
+    L.sync_ratio()  # nothing to write: a no-op
+    for r in [0.75, 0.25, 1.0, 0.5, 0.25, 0.0]:   # nothing between the replays: every graph is complete in itself
+        Y.zero_()
+        graphs[r].replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(Y.cpu().numpy(), want[r]), r
     fx.flexiq_check_status()
     L.close()
 
