@@ -83,8 +83,12 @@ struct GemmParams {
     // being the positions y * PW + x of a grid whose pitch PW (a power of two >= W + pad) leaves a few unused
     // columns.  The input patch of TH + R - 1 rows x PW pixels is loaded ONCE per tile by a tiled 4-D copy
     // (halo and padding arrive as zeros); filter tap (r, s) is the same patch read from row offset r * PW + s,
-    // so every input pixel crosses from L2 once instead of R * S times.
+    // so every input pixel crosses from L2 once instead of R * S times.  When W + 2 pad > PW the rightmost taps of the
+    // last pixels of an output row index a column beyond the pitch, i.e. the first columns of the NEXT patch row: that
+    // is its left padding, zeros, which is what the right padding should read -- provided the row exists, so the
+    // patch then carries one more row.
     int pw_log2, TH, tiles_per_img, patch_stage;   // patch_stage: bytes of one ring stage (the patch, rounded up to 1 KB)
+    int patch_rows;      // input rows of a patch: TH + R - 1, plus one when a tap's column index can pass the pitch (see above)
     // packed low-bit path only: positions the expander warps shift the 4-bit values back to
     const uint8_t *sx;   // [n_g] activation positions, slab order
     const uint8_t *sw;   // [n_g][N] weight positions
@@ -773,7 +777,7 @@ mixed_gemm_kernel(const __grid_constant__ CUtensorMap mapA_lo, const __grid_cons
                 if (ptx::elect_one()) {
                     const int img = tw.m_blk / p.tiles_per_img;
                     const int y0 = (tw.m_blk - img * p.tiles_per_img) * p.TH;
-                    ptx::mbar_expect_tx_s(full0 + 8 * stage, (uint32_t)(((p.TH + p.T / p.S - 1) << p.pw_log2) * p.BK));
+                    ptx::mbar_expect_tx_s(full0 + 8 * stage, (uint32_t)((p.patch_rows << p.pw_log2) * p.BK));
                     ptx::tma_load_4d_s(stage0 + stage * stage_bytes, &mapA_hi, full0 + 8 * stage, 0, -p.pad, y0 - p.pad, img);
                 }
                 __syncwarp();
@@ -1561,12 +1565,13 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     if (!packed && !g_forced_tile.cg && p.im2col && L->stride == 1 && L->C <= p.BK && L->N <= 128 && W + L->pad <= 128) {
         while (patch_pw < W + L->pad) patch_pw *= 2;
         const int th = BM / patch_pw, bn_p = L->N <= 64 ? 64 : 128;
-        const int stage = (((th + L->R - 1) * patch_pw * p.BK) + 1023) & ~1023;
+        const int rows = th + L->R - 1 + (W + 2 * L->pad > patch_pw ? 1 : 0);
+        const int stage = ((rows * patch_pw * p.BK) + 1023) & ~1023;
         const int b_all = ((p.T * bn_p * p.BK) + 1023) & ~1023;
-        if (b_all + 2 * stage <= kStageRegion && th + L->R - 1 <= 256) {
+        if (b_all + 2 * stage <= kStageRegion && rows <= 256) {
             patch = true;
             tc.cg = 1; tc.bn = bn_p;
-            p.TH = th; p.patch_stage = stage;
+            p.TH = th; p.patch_stage = stage; p.patch_rows = rows;
             p.pw_log2 = 0;
             while ((1 << p.pw_log2) < patch_pw) ++p.pw_log2;
             p.tiles_per_img = (p.P + th - 1) / th;
@@ -1619,7 +1624,7 @@ static int run_mixed(Layer *L, const uint8_t *X4, const int8_t *X8, const uint8_
     } else if (!packed) {
         // one int8 slab [rows][C] (a packed-path layer at ratio 0 has it in X8_dev)
         if (patch) {
-            if ((rc = make_map_nhwc(&a_hi, slab, (uint64_t)L->C, W, H, Nb, p.BK, 1u << p.pw_log2, p.TH + L->R - 1, p.BK))) return rc;
+            if ((rc = make_map_nhwc(&a_hi, slab, (uint64_t)L->C, W, H, Nb, p.BK, 1u << p.pw_log2, p.patch_rows, p.BK))) return rc;
         } else if (p.im2col) {
             if ((rc = make_map_im2col(&a_hi, slab, L->C, L->C, Nb, H, W, L->R, L->S, L->stride, L->pad, p.BK, p.BK))) return rc;
         } else {

@@ -254,7 +254,10 @@ def test_conv_shapes(dev, Nb, H, C, Cout, R, stride):
                                           (2, 20, 48, 32, 3),     # fewer channels than the K block
                                           (2, 33, 64, 48, 5),     # 5 x 5 taps (the generic tap loop), pitch 64, odd height
                                           (1, 60, 32, 16, 3),     # widest image the 64-pixel pitch holds with its padding... and one K step
-                                          (2, 100, 64, 64, 3)])   # pitch 128: one output row per tile
+                                          (2, 100, 64, 64, 3),    # pitch 128: one output row per tile
+                                          (2, 15, 32, 32, 3),     # W + pad == pitch: the right padding of a tile's last pixel is the
+                                          (3, 31, 16, 112, 3),    # next patch row's left padding, so the patch carries one more row
+                                          (4, 14, 32, 48, 5)])
 def test_conv_patch_mode_edges(dev, Nb, H, C, Cout, R):
     """Stride-1 convolutions whose channels fit one K block take the patch path (one halo patch per tile, taps as row
     offsets into it): image sizes that leave unused grid columns and ragged last tiles, narrow channel counts."""
