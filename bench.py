@@ -150,21 +150,14 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
     gemm_events = []
 
-    def step(record=False):
-        for ri, r in enumerate(RATIOS):
+    def step():
+        for r in RATIOS:
             for L in layers:
                 L.set_lowbit_ratio(r)
             for li, (L, c) in enumerate(zip(layers, cases)):
                 x4, x8 = slabs[li]
                 fx.flexiq_quantize_lower(L.h, Xd[li], fx.DTYPE_F32, c.M, c.x_scale, 0, x4, x8)
-                if record:
-                    e0 = torch.cuda.Event(enable_timing=True)
-                    e1 = torch.cuda.Event(enable_timing=True)
-                    e0.record(stream)
                 fx.flexiq_mixed_gemm(L.h, x4, x8, None, c.M, c.x_scale, c.y_scale, fx.OUT_REQUANT_I8, Yd[li])
-                if record:
-                    e1.record(stream)
-                    gemm_events.append((ri, li, e0, e1))
 
     for _ in range(max(args.warmup, 3)):
         step()
