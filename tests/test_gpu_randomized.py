@@ -325,3 +325,69 @@ def test_random_call_sequences_on_one_handle(dev):
         fx.flexiq_check_status()
         del graphs
         L.close()
+
+
+def test_random_auxiliary_kernels(dev):
+    """The kernels around the layer path on drawn shapes: calibration ranges (one or several batches), histogram
+    and coverage ranges, static preparation (positions, scores, greedy order), the residual reorder operator in
+    both directions and three element sizes, and the squared distance of the selection search."""
+    for i in range(30):
+        rng = np.random.default_rng(5100000 + i)
+        G = int(rng.choice([16, 32, 64]))
+        K = G * int(rng.integers(1, 70))
+        N = 16 * int(rng.integers(1, 20))
+        M = int(rng.integers(1, 900))
+        dt = [torch.float32, torch.float16, torch.bfloat16][int(rng.integers(0, 3))]
+        xs = float(rng.uniform(0.01, 0.2))
+        x = (rng.normal(0, 1, (M, K)) * rng.uniform(0.05, 8, (1, K))).astype(np.float32)
+        X = torch.from_numpy(x).to(dt).to(dev)
+        q = oracle.quantize(X.float().cpu().numpy(), xs)
+        # ranges, accumulated over two uneven parts
+        lo = torch.empty(K, dtype=torch.int32, device=dev)
+        hi = torch.empty(K, dtype=torch.int32, device=dev)
+        cut = int(rng.integers(0, M + 1))
+        code = fx._dtype_code(X)
+        if cut:
+            fx.flexiq_calib_channel_ranges(X[:cut], code, cut, K, xs, False, lo, hi)
+        if M - cut:
+            fx.flexiq_calib_channel_ranges(X[cut:], code, M - cut, K, xs, bool(cut), lo, hi)
+        elo, ehi = oracle.channel_ranges(q)
+        assert np.array_equal(lo.cpu().numpy(), elo) and np.array_equal(hi.cpu().numpy(), ehi), f"ranges {(M, K, dt)}"
+        # histogram and coverage ranges
+        hist = torch.empty((K, 256), dtype=torch.int32, device=dev)
+        fx.flexiq_calib_channel_histogram(X, code, M, K, xs, False, hist)
+        eh = oracle.channel_histogram(q)
+        assert np.array_equal(hist.cpu().numpy().view(np.uint32), eh), f"histogram {(M, K, dt)}"
+        tail = int(rng.integers(0, max(1, M // 8) + 1))
+        clo, chi = torch.empty_like(lo), torch.empty_like(hi)
+        fx.flexiq_calib_ranges_from_histogram(hist, K, tail, clo, chi)
+        e_clo, e_chi = oracle.ranges_from_histogram(eh, tail)
+        assert np.array_equal(clo.cpu().numpy(), e_clo) and np.array_equal(chi.cpu().numpy(), e_chi), f"coverage {(M, K, tail)}"
+        # weight ranges, positions, scores, greedy order
+        Wq = rng.integers(-127, 128, (K, N)).astype(np.int8)
+        Wq[rng.integers(0, K, K // 3)] //= 16   # some narrow input channels
+        perm, sx, info = calib.static_preparation_device(X, xs, torch.from_numpy(Wq).to(dev), G)
+        wmax = oracle.weight_absmax_linear(Wq)
+        perm_e, score_e = oracle.greedy_order(elo, ehi, wmax, G)
+        assert np.array_equal(info["wmax"].cpu().numpy(), wmax)
+        assert np.array_equal(sx, oracle.static_positions(elo, ehi, G))
+        assert np.array_equal(info["score"].cpu().numpy(), score_e) and np.array_equal(perm, perm_e), f"order {(K, N, G)}"
+        # residual reorder in the order just found
+        L = fx.Layer(torch.from_numpy(Wq).to(dev), torch.ones(N, device=dev), torch.zeros(N, device=dev), perm, sx, G)
+        rdt = [torch.int8, torch.float16, torch.float32][int(rng.integers(0, 3))]
+        R = torch.from_numpy(rng.integers(-120, 120, (M, K)).astype(np.int32)).to(rdt).to(dev)
+        Y, guard_ok = helpers.with_guard(torch, (M, K), rdt, dev)
+        L.reorder_channels(R, fx.REORDER_TO_SLAB, Y=Y)
+        torch.cuda.synchronize()
+        guard_ok()
+        assert np.array_equal(Y.cpu().numpy(), oracle.reorder_channels(R.cpu().numpy(), G, perm, True)), f"reorder {(M, K, G, rdt)}"
+        assert torch.equal(L.reorder_channels(Y, fx.REORDER_FROM_SLAB), R)
+        L.close()
+        # squared distance of two int8 tensors
+        n = int(rng.integers(0, 300000))
+        a = rng.integers(-128, 128, n).astype(np.int8)
+        b = rng.integers(-128, 128, n).astype(np.int8)
+        out = torch.full((1,), -5, dtype=torch.int64, device=dev)
+        fx.flexiq_sq_distance_i8(torch.from_numpy(a).to(dev), torch.from_numpy(b).to(dev), out)
+        assert int(out.item()) == int(((a.astype(np.int64) - b.astype(np.int64)) ** 2).sum())
+    fx.flexiq_check_status()
