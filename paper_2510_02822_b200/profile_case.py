@@ -47,6 +47,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=1)
     ap.add_argument("--path", default="masked", choices=["masked", "packed"])
     ap.add_argument("--out", default="i8", choices=["i8", "f32", "i32", "f16", "bf16"])
+    ap.add_argument("--dynamic", action="store_true", help="run-time extraction positions (Sec. 4.1): the prologue finds them from the call's own values")
     ap.add_argument("--aux", default="", choices=["", "reorder", "calib", "distance"], help="run an auxiliary kernel on the layer's input instead: the residual reorder operator, the calibration range kernels, or the squared-distance reduction (on the int8 view of the input and a shifted copy)")
     args = ap.parse_args()
     dev = torch.device("cuda:0")
@@ -97,22 +98,23 @@ def main():
 
     def mixed(x4, x8):
         if is_conv:
-            return L.mixed_conv(x4, x8, c.Nb, c.H, c.W, c.x_scale, c.y_scale, mode, Y=Ybuf)
-        return L.mixed_gemm(x4, x8, M, c.x_scale, c.y_scale, mode, Y=Ybuf)
+            return L.mixed_conv(x4, x8, c.Nb, c.H, c.W, c.x_scale, c.y_scale, mode, Y=Ybuf, x_shift=shifts)
+        return L.mixed_gemm(x4, x8, M, c.x_scale, c.y_scale, mode, Y=Ybuf, x_shift=shifts)
 
-    x4, x8, _ = L.quantize_lower(X, c.x_scale)
+    x4, x8, shifts = L.quantize_lower(X, c.x_scale, dynamic=args.dynamic)
+    slabs = (x4, x8)
     Ybuf = None
     Ybuf = mixed(x4, x8)
     ops = 2.0 * Ybuf.numel() * (c.R * c.S * c.C if is_conv else c.K)
     for _ in range(args.warmup):
-        L.quantize_lower(X, c.x_scale)
+        L.quantize_lower(X, c.x_scale, dynamic=args.dynamic, slabs=slabs)
         mixed(x4, x8)
     # back-to-back launches: the queue stays full, so launch latency is hidden
     e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
     torch.cuda.synchronize()
     e[0].record(stream)
     for _ in range(args.iters):
-        L.quantize_lower(X, c.x_scale)
+        L.quantize_lower(X, c.x_scale, dynamic=args.dynamic, slabs=slabs)
     e[1].record(stream)
     for _ in range(args.iters):
         mixed(x4, x8)
@@ -121,7 +123,7 @@ def main():
     fx.flexiq_check_status()
     tp = e[0].elapsed_time(e[1]) / args.iters
     tg = e[1].elapsed_time(e[2]) / args.iters
-    print(f"{args.layer} ratio={args.ratio} path={args.path}: prologue {tp * 1e3:.1f} us, mixed kernel {tg * 1e3:.1f} us, "
+    print(f"{args.layer} ratio={args.ratio} path={args.path}{' dynamic positions' if args.dynamic else ''}: prologue {tp * 1e3:.1f} us, mixed kernel {tg * 1e3:.1f} us, "
           f"{ops / tg / 1e9:.1f} TOPS")
     L.close()
 
