@@ -257,7 +257,10 @@ def test_conv_shapes(dev, Nb, H, C, Cout, R, stride):
                                           (2, 100, 64, 64, 3),    # pitch 128: one output row per tile
                                           (2, 15, 32, 32, 3),     # W + pad == pitch: the right padding of a tile's last pixel is the
                                           (3, 31, 16, 112, 3),    # next patch row's left padding, so the patch carries one more row
-                                          (4, 14, 32, 48, 5)])
+                                          (4, 14, 32, 48, 5),
+                                          (1, 127, 16, 32, 3),    # W + pad == 128: the widest image of the patch path, one row per tile, the extra row
+                                          (1, 126, 16, 32, 5),    # the same with two pixels of padding
+                                          (1, 128, 16, 32, 3)])   # one pixel too wide for it: im2col copies
 def test_conv_patch_mode_edges(dev, Nb, H, C, Cout, R):
     """Stride-1 convolutions whose channels fit one K block take the patch path (one halo patch per tile, taps as row
     offsets into it): image sizes that leave unused grid columns and ragged last tiles, narrow channel counts."""
