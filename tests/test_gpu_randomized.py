@@ -391,3 +391,36 @@ def test_random_auxiliary_kernels(dev):
         fx.flexiq_sq_distance_i8(torch.from_numpy(a).to(dev), torch.from_numpy(b).to(dev), out)
         assert int(out.item()) == int(((a.astype(np.int64) - b.astype(np.int64)) ** 2).sum())
     fx.flexiq_check_status()
+
+
+def test_random_large_linears_on_sampled_rows(dev):
+    """Linears of 2,000 to 30,000 rows, up to 4096 input and output channels: several waves of tiles per CTA, CTA pairs,
+    ragged last tiles in both directions.  The oracle computes 150 random rows, the first rows and the last 40;
+    a second launch must give the same bytes as the first everywhere."""
+    for i in range(10):
+        rng = np.random.default_rng(6100000 + i)
+        G = int(rng.choice([16, 32, 64]))
+        K = G * int(rng.integers(4, 4096 // G + 1))
+        N = 16 * int(rng.integers(8, 257))
+        M = int(rng.integers(2000, 30000))
+        case = inputs.vit_linear("rb", M, K, N, G, seed=i)
+        perm, sxg, sxs, sw = helpers.prepare_linear(case, rng.integers(0, 5, K // G).astype(np.uint8))
+        L = _mk(case, dev, perm, sxg)
+        X = torch.from_numpy(case.X).to(dev)
+        rows = np.unique(np.concatenate([rng.integers(0, M, 150), np.arange(M - 40, M), np.arange(0, 8)])).astype(np.int64)
+        ridx = torch.from_numpy(rows).to(dev)
+        q_rows = oracle.quantize(case.X[rows], case.x_scale)
+        for r in (float(rng.random()), float(rng.choice([0.0, 0.5, 1.0]))):
+            L.set_lowbit_ratio(r)
+            nl = oracle.n_low(r, K // G)
+            x4, x8, _ = L.quantize_lower(X, case.x_scale)
+            mode = int(rng.choice([fx.OUT_REQUANT_I8, fx.OUT_DEQUANT_F16, fx.OUT_ACC_I32]))
+            Y = L.mixed_gemm(x4, x8, M, case.x_scale, case.y_scale, mode)
+            Y2 = L.mixed_gemm(x4, x8, M, case.x_scale, case.y_scale, mode)
+            torch.cuda.synchronize()
+            fx.flexiq_check_status()
+            acc = oracle.mixed_gemm_acc(q_rows, case.Wq, G, perm, sxs, sw, nl)
+            what = f"linear {(M, K, N, G)} ratio {r} mode {mode}"
+            assert np.array_equal(_bits(Y[ridx], mode), _expected(acc, case, mode, case.y_scale)), what
+            assert torch.equal(Y.view(torch.uint8), Y2.view(torch.uint8)), what
+        L.close()
